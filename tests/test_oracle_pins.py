@@ -1,0 +1,525 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+Nothing here touches the CUDA path. Each test checks the oracle against a closed form,
+an invariant, a library routine it does not itself call (numpy/scipy/torch fp64), or
+brute force on tiny inputs, chosen so that a plausible slip in the oracle (dropped term,
+wrong sign or index, transposed operand) fails at least one of them.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as TF
+
+import oracle
+
+V = 4096
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ------------------------------------------------------------------ entropy (Eq. 4, 7)
+def test_entropy_uniform_is_ln_v():
+    z = np.full((1, 3, V), 0.37, np.float32)
+    ent, mean = oracle.scale_entropy(z)
+    assert np.allclose(ent, math.log(V), atol=1e-6)
+    assert abs(mean[0] - math.log(V)) < 1e-6
+    assert abs(math.log(V) - 8.317766) < 1e-6
+
+
+def test_entropy_one_hot_is_zero():
+    z = np.zeros((1, 2, V), np.float32)
+    z[0, 0, 17] = 1000.0          # exp(-1000) underflows to 0 in double: exactly 0
+    z[0, 1, 4095] = 100.0         # 4095 * e^-100 * ~100: far below fp32 resolution of 1
+    ent, _ = oracle.scale_entropy(z)
+    assert ent[0, 0] == 0.0
+    assert 0.0 <= ent[0, 1] < 1e-30
+
+
+def test_entropy_two_level_closed_form():
+    # m logits at value a, V-m at value b
+    for m, a, b in [(1, 3.0, 0.0), (100, 2.0, -1.0), (4000, -0.5, 0.25), (7, 9.0, 1.0)]:
+        z = np.full((1, 1, V), b, np.float32)
+        z[0, 0, :m] = a
+        Z = m * math.exp(a) + (V - m) * math.exp(b)
+        want = math.log(Z) - (m * a * math.exp(a) + (V - m) * b * math.exp(b)) / Z
+        ent, _ = oracle.scale_entropy(z)
+        assert abs(ent[0, 0] - want) < 1e-6 * max(1.0, want)
+
+
+def test_entropy_binary_matches_sigmoid_entropy():
+    z = np.array([[[0.3, -1.2]], [[5.0, 5.0]], [[-2.0, 4.0]]], np.float32)  # V = 2
+    ent, _ = oracle.scale_entropy(z)
+    for r in range(3):
+        p = 1.0 / (1.0 + math.exp(-(float(z[r, 0, 1]) - float(z[r, 0, 0]))))
+        want = -(p * math.log(p) + (1 - p) * math.log(1 - p))
+        assert abs(ent[r, 0] - want) < 1e-6
+
+
+def test_entropy_shift_invariance_bounds_and_library():
+    from scipy.special import softmax
+    from scipy.stats import entropy as sp_entropy
+    rng = np.random.default_rng(0)
+    z = (rng.standard_normal((2, 5, 512)) * rng.uniform(0.2, 6.0, (2, 5, 1))).astype(np.float32)
+    ent, mean = oracle.scale_entropy(z)
+    ent_shift, _ = oracle.scale_entropy(z + np.float32(8.0))   # exact shift in fp32 for these magnitudes? use tolerance
+    assert np.allclose(ent, ent_shift, atol=2e-5)
+    assert (ent >= 0).all() and (ent <= math.log(512) + 1e-6).all()
+    lib = sp_entropy(softmax(z.astype(np.float64), axis=-1), axis=-1)
+    assert np.allclose(ent, lib, atol=1e-6)
+    assert np.allclose(mean, lib.mean(axis=1), atol=1e-6)
+
+
+def test_entropy_neg_inf_logit_contributes_nothing():
+    z = np.zeros((1, 1, 8), np.float32)
+    z[0, 0, 4:] = -np.inf
+    ent, _ = oracle.scale_entropy(z)
+    assert abs(ent[0, 0] - math.log(4)) < 1e-7
+
+
+def test_mean_is_per_segment_and_permutation_invariant():
+    rng = np.random.default_rng(1)
+    z = rng.standard_normal((3, 16, 64)).astype(np.float32) * 3
+    ent, mean = oracle.scale_entropy(z)
+    perm = rng.permutation(16)
+    ent_p, mean_p = oracle.scale_entropy(z[:, perm])
+    assert np.array_equal(ent[:, perm], ent_p)
+    assert np.allclose(mean, mean_p, atol=1e-6)
+    assert np.allclose(mean, ent.astype(np.float64).mean(axis=1), atol=1e-6)
+
+
+# ------------------------------------------------------- trigger and ratios (Eq. 8-13)
+def _read_golden(name):
+    vals = {}
+    with open(os.path.join(GOLDEN, name)) as fh:
+        for line in fh:
+            line = line.split("#")[0].strip()
+            if "=" in line:
+                k, v = line.split("=")
+                vals[k.strip()] = v.strip()
+    return vals
+
+
+def test_schedule_worked_example_golden():
+    gold = _read_golden("schedule_worked_example.txt")
+    hbar = np.array([[float(x) for x in gold["hbar"].split()]], np.float32)
+    p = oracle.SchedParams()
+    assert (p.t_est, p.alpha, p.tau, p.lam) == (5, 0.5, 0.8, 0.1)   # paper's hyper-parameters
+    for t in range(1, 11):
+        r = oracle.keep_ratios(p, t, 1, 256, hbar[:, :t])
+        if t < 7:
+            assert r["t_star"][0] == 0 and r["act_scale"][0] == 0 and r["keep"][0] == 256
+        else:
+            assert r["t_star"][0] == int(gold["t_star"])
+            assert r["act_scale"][0] == int(gold["act_scale"])
+        if t == 7:
+            assert r["keep"][0] == 256 and r["ratio_scale"][0] == 0.0   # t* itself is not pruned
+        if t >= 8:
+            assert abs(r["ratio_scale"][0] - float(gold[f"ratio_{t}"])) < 1e-12
+            assert r["keep"][0] == int(gold[f"keep_{t}"])
+
+
+def test_trigger_telescoping_and_linear_growth_never_triggers():
+    p = oracle.SchedParams()
+    # linear growth: smoothed rate equals eta forever, alpha < 1 -> never triggers
+    hbar = (0.5 + 0.7 * np.arange(1, 14, dtype=np.float64))[None].astype(np.float32)
+    r = oracle.keep_ratios(p, 13, 1, 100, hbar)
+    assert r["t_star"][0] == 0 and r["keep"][0] == 100
+    # telescoping: eta = (H_5 - H_1)/4 and smoothed g_t = (H_t - H_{t-2})/2, checked via the
+    # trigger position on a random increasing-then-flat curve
+    rng = np.random.default_rng(3)
+    for _ in range(50):
+        H = np.cumsum(rng.uniform(0.0, 1.0, 12))
+        H[rng.integers(6, 12):] = H[5]
+        eta = (H[4] - H[0]) / 4.0
+        want = 0
+        for t in range(6, 13):
+            if (H[t - 1] - H[t - 3]) / 2.0 <= 0.5 * eta:
+                want = t
+                break
+        # skip cases within fp32 rounding of the threshold
+        margins = [abs((H[t - 1] - H[t - 3]) / 2.0 - 0.5 * eta) for t in range(6, 13)]
+        if min(margins) < 1e-5:
+            continue
+        r = oracle.keep_ratios(p, 12, 1, 64, H[None].astype(np.float32))
+        assert r["t_star"][0] == want
+
+
+def test_scale_ratio_monotone_and_lambda_term():
+    p0 = oracle.SchedParams(lam=0.0, force_act_scale=6)
+    hbar = np.linspace(1, 3, 12, dtype=np.float32)[None]
+    prev = -1.0
+    for t in range(6, 13):
+        r = oracle.keep_ratios(p0, t, 1, 1000, hbar[:, :t])["ratio_scale"][0]
+        assert abs(r - 1.0 / (1.0 + math.exp(-(t - 6) / 0.8))) < 1e-12
+        assert r > prev
+        prev = r
+    p1 = oracle.SchedParams(lam=0.1, force_act_scale=6)
+    g = float(hbar[0, 7]) - float(hbar[0, 6])
+    r = oracle.keep_ratios(p1, 8, 1, 1000, hbar[:, :8])["ratio_scale"][0]
+    assert abs(r - (1.0 / (1.0 + math.exp(-2 / 0.8)) - 0.1 * math.tanh(g))) < 1e-12
+    # growing entropy (g > 0) prunes less than a flat curve
+    flat = np.full((1, 8), 2.0, np.float32)
+    r_flat = oracle.keep_ratios(p1, 8, 1, 1000, flat)["ratio_scale"][0]
+    assert r < r_flat
+
+
+def test_layer_linkage_examples():
+    p = oracle.SchedParams(force_act_scale=2, lam=0.0)
+    hbar = np.array([[1.0, 1.0]], np.float32)          # t = 2 = activation -> Ratio_t = 0.5
+    base = oracle.keep_ratios(p, 2, 1, 1000, hbar)
+    assert base["ratio_scale"][0] == 0.5 and base["ratio_layer"][0] == 0.5
+    same = oracle.keep_ratios(p, 2, 3, 1000, hbar, np.array([[4.0, 4.0, 4.0]], np.float32))
+    assert same["ratio_layer"][0] == 0.5
+    r2 = oracle.keep_ratios(p, 2, 2, 1000, hbar, np.array([[4.0, 5.0]], np.float32))
+    assert abs(r2["ratio_layer"][0] - 0.75 * 0.5) < 1e-12      # Delta = 0.25
+    assert r2["keep"][0] == 1000 - 375
+    r3 = oracle.keep_ratios(p, 2, 3, 1000, hbar, np.array([[4.0, 5.0, 3.0]], np.float32))
+    assert abs(r3["ratio_layer"][0] - (4.0 / 3.0) * 0.5) < 1e-12  # mu = 4.5, Delta = -1/3
+    # a higher-entropy layer always prunes less
+    assert r2["ratio_layer"][0] < 0.5 < r3["ratio_layer"][0]
+    # mu == 0 -> Delta = 0
+    rz = oracle.keep_ratios(p, 2, 2, 1000, hbar, np.array([[0.0, 5.0]], np.float32))
+    assert rz["ratio_layer"][0] == 0.5
+
+
+def test_keep_count_clamps_and_overrides():
+    hbar = np.ones((2, 9), np.float32)
+    p = oracle.SchedParams(force_act_scale=9, force_keep_ratio=0.2)
+    r = oracle.keep_ratios(p, 9, 1, 16384, hbar)
+    assert (r["keep"] == 16384 - math.floor(0.8 * 16384)).all() and r["keep"][0] == 3277
+    p = oracle.SchedParams(force_act_scale=3, force_keep_ratio=0.0, k_min=5)
+    assert oracle.keep_ratios(p, 9, 1, 100, hbar)["keep"][0] == 5
+    p = oracle.SchedParams(force_act_scale=3, ratio_max=0.6, lam=0.0)
+    assert oracle.keep_ratios(p, 9, 1, 100, hbar)["keep"][0] == 40      # sigmoid(7.5) clamped to 0.6
+    # ratio driven above 1 or below 0 by the layer term is clamped
+    p = oracle.SchedParams(force_act_scale=9, lam=0.0)
+    hi = oracle.keep_ratios(p, 9, 2, 100, hbar, np.array([[4.0, 0.1], [1.0, 9.0]], np.float32))
+    assert hi["ratio_layer"][0] > 0.9 and hi["keep"][0] == 100 - math.floor(hi["ratio_layer"][0] * 100)
+    assert hi["ratio_layer"][1] < 0 and hi["keep"][1] == 100
+    # not yet activated -> nothing pruned
+    p = oracle.SchedParams(force_act_scale=10, force_keep_ratio=0.5)
+    assert oracle.keep_ratios(p, 9, 1, 100, hbar)["keep"][0] == 100
+
+
+# --------------------------------------------------------------------------- top-k
+def _brute_topk(e, k):
+    order = np.argsort(-e.astype(np.float64), kind="stable")   # descending, ties -> lower index
+    keep = np.sort(order[:k])
+    prune = np.sort(order[k:])
+    return keep, prune
+
+
+def test_topk_exhaustive_three_value_alphabet():
+    alphabet = (0.0, 1.5, 1.5000001)
+    for N in range(1, 8):
+        rows = np.array(list(itertools.product(alphabet, repeat=N)), np.float32)
+        for k in range(0, N + 1):
+            ks = np.full(len(rows), k, np.int32)
+            keep_idx, prune_idx, cu, pos = oracle.select_topk(rows, ks)
+            assert np.array_equal(cu, np.arange(len(rows) + 1) * k)
+            for s, e in enumerate(rows):
+                wk, wp = _brute_topk(e, k)
+                assert np.array_equal(keep_idx[s * k:(s + 1) * k], wk)
+                assert np.array_equal(prune_idx[s * (N - k):(s + 1) * (N - k)], wp)
+                inv = np.full(N, -1)
+                inv[wk] = np.arange(k)
+                assert np.array_equal(pos[s], inv)
+
+
+def test_topk_special_cases_and_ragged_k():
+    N = 97
+    same = np.full((1, N), 2.5, np.float32)
+    keep_idx, prune_idx, cu, _ = oracle.select_topk(same, [10])
+    assert np.array_equal(keep_idx, np.arange(10)) and np.array_equal(prune_idx, np.arange(10, N))
+    inc = np.arange(N, dtype=np.float32)[None]
+    assert np.array_equal(oracle.select_topk(inc, [5])[0], np.arange(N - 5, N))
+    assert np.array_equal(oracle.select_topk(inc, [N])[0], np.arange(N))
+    e = np.array([[1, 7, 7, 3]], np.float32)
+    assert oracle.select_topk(e, [1])[0][0] == 1            # first arg-max
+    # signed zeros compare equal: the tie goes to the lower index
+    z = np.array([[-0.0, 0.0, -0.0, 0.0]], np.float32)
+    assert np.array_equal(oracle.select_topk(z, [2])[0], [0, 1])
+    rng = np.random.default_rng(5)
+    ent = rng.standard_normal((4, 300)).astype(np.float32)
+    ent[:, ::7] = ent[:, 3:4]                                # many ties
+    ks = np.array([1, 150, 299, 300], np.int32)
+    keep_idx, prune_idx, cu, pos = oracle.select_topk(ent, ks)
+    assert np.array_equal(cu, np.concatenate([[0], np.cumsum(ks)]))
+    off_p = 0
+    for s in range(4):
+        wk, wp = _brute_topk(ent[s], ks[s])
+        assert np.array_equal(keep_idx[cu[s]:cu[s + 1]], wk)
+        assert np.array_equal(prune_idx[off_p:off_p + len(wp)], wp)
+        off_p += len(wp)
+
+
+# ------------------------------------------------------------------ block (Eq. 14)
+def _rand_weights(C, F, rng, scale=0.2):
+    w = {
+        "ln1_g": 1 + 0.1 * rng.standard_normal(C), "ln1_b": 0.1 * rng.standard_normal(C),
+        "w_qkv": scale * rng.standard_normal((3 * C, C)), "b_qkv": 0.1 * rng.standard_normal(3 * C),
+        "w_o": scale * rng.standard_normal((C, C)), "b_o": 0.1 * rng.standard_normal(C),
+        "ln2_g": 1 + 0.1 * rng.standard_normal(C), "ln2_b": 0.1 * rng.standard_normal(C),
+        "w_fc1": scale * rng.standard_normal((F, C)), "b_fc1": 0.1 * rng.standard_normal(F),
+        "w_fc2": scale * rng.standard_normal((C, F)), "b_fc2": 0.1 * rng.standard_normal(C),
+    }
+    return {k: v.astype(np.float32) for k, v in w.items()}
+
+
+def _torch_block(w, eps, heads, x_kept, k_old, v_old):
+    """One image, library ops only (torch fp64): x_kept [k, C], k_old/v_old [P, C]."""
+    t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    x = t(x_kept)
+    C = x.shape[1]
+    dh = C // heads
+    h = TF.layer_norm(x, (C,), t(w["ln1_g"]), t(w["ln1_b"]), eps)
+    qkv = TF.linear(h, t(w["w_qkv"]), t(w["b_qkv"]))
+    q, k, v = qkv.split(C, dim=1)
+    K = torch.cat([t(k_old), k])
+    Vv = torch.cat([t(v_old), v])
+    sh = lambda a: a.view(a.shape[0], heads, dh).transpose(0, 1)
+    o = TF.scaled_dot_product_attention(sh(q), sh(K), sh(Vv))
+    o = o.transpose(0, 1).reshape(x.shape[0], C)
+    x1 = x + TF.linear(o, t(w["w_o"]), t(w["b_o"]))
+    h2 = TF.layer_norm(x1, (C,), t(w["ln2_g"]), t(w["ln2_b"]), eps)
+    f = TF.linear(TF.gelu(TF.linear(h2, t(w["w_fc1"]), t(w["b_fc1"])), approximate="tanh"),
+                  t(w["w_fc2"]), t(w["b_fc2"]))
+    return (x1 + f).numpy(), k.numpy(), v.numpy()
+
+
+def _block_case(seed=0, B=2, N=12, C=16, heads=2, F=24, Lmax=20, P=(5, 0)):
+    rng = np.random.default_rng(seed)
+    w = _rand_weights(C, F, rng)
+    x = rng.standard_normal((B, N, C)).astype(np.float32)
+    kc = rng.standard_normal((B, Lmax, C)).astype(np.float32)
+    vc = rng.standard_normal((B, Lmax, C)).astype(np.float32)
+    return w, x, kc, vc, np.array(P, np.int32)
+
+
+def test_block_matches_library_composition_ragged():
+    w, x, kc, vc, kv_len = _block_case()
+    ent = np.random.default_rng(9).standard_normal((2, 12)).astype(np.float32)
+    keep_idx, _, cu, _ = oracle.select_topk(ent, [7, 3])
+    y, k_new, v_new = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len)
+    for b in range(2):
+        idx = keep_idx[cu[b]:cu[b + 1]]
+        wy, wk, wv = _torch_block(w, 1e-6, 2, x[b, idx], kc[b, :kv_len[b]], vc[b, :kv_len[b]])
+        assert np.allclose(y[cu[b]:cu[b + 1]], wy, atol=2e-5, rtol=1e-5)
+        assert np.allclose(k_new[cu[b]:cu[b + 1]], wk, atol=1e-5)
+        assert np.allclose(v_new[cu[b]:cu[b + 1]], wv, atol=1e-5)
+
+
+def test_block_keep_all_equals_dense_block_and_row_subset():
+    w, x, kc, vc, kv_len = _block_case(seed=2)
+    B, N, _ = x.shape
+    keep_idx = np.tile(np.arange(N, dtype=np.int32), B)
+    cu = np.arange(B + 1, dtype=np.int32) * N
+    y, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len)
+    for b in range(B):
+        wy, _, _ = _torch_block(w, 1e-6, 2, x[b], kc[b, :kv_len[b]], vc[b, :kv_len[b]])
+        assert np.allclose(y[b * N:(b + 1) * N], wy, atol=2e-5, rtol=1e-5)
+    rows = np.array([3, 17, 0], np.int32)
+    ys, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len, rows=rows)
+    assert np.array_equal(ys, y[rows])
+
+
+def test_block_attention_special_cases():
+    w, x, kc, vc, kv_len = _block_case(seed=3, P=(4, 6))
+    B, N, C = x.shape
+    # isolate attention: q = 0 -> uniform weights; W_o = I, FFN output zero, k/v = LN1 output
+    w["w_qkv"][:C] = 0
+    w["b_qkv"][:C] = 0
+    w["w_qkv"][2 * C:] = np.eye(C, dtype=np.float32)
+    w["b_qkv"][2 * C:] = 0
+    w["w_o"] = np.eye(C, dtype=np.float32)
+    w["b_o"][:] = 0
+    w["w_fc2"][:] = 0
+    w["b_fc2"][:] = 0
+    keep_idx = np.array([1, 4, 9, 0, 2], np.int32)
+    cu = np.array([0, 3, 5], np.int32)
+    y, k_new, v_new = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len)
+    for b in range(B):
+        allv = np.concatenate([vc[b, :kv_len[b]], v_new[cu[b]:cu[b + 1]]]).astype(np.float64)
+        for m in range(cu[b], cu[b + 1]):
+            assert np.allclose(y[m] - x[b, keep_idx[m]], allv.mean(axis=0), atol=1e-5)
+    # one key only (empty cache, one kept token): the output is that token's own value row
+    y1, _, v1 = oracle.pruned_block_forward(w, 1e-6, 2, x, np.array([5, 7], np.int32),
+                                            np.array([0, 1, 2], np.int32), kc, vc,
+                                            np.zeros(2, np.int32))
+    assert np.allclose(y1[0] - x[0, 5], v1[0], atol=1e-6)
+    assert np.allclose(y1[1] - x[1, 7], v1[1], atol=1e-6)
+
+
+def test_block_constant_query_softmax_per_head():
+    from scipy.special import softmax
+    w, x, kc, vc, kv_len = _block_case(seed=4, B=1, P=(9,))
+    C, heads, dh = 16, 2, 8
+    w["w_qkv"][:C] = 0                      # q = b_q for every token
+    w["w_o"] = np.eye(C, dtype=np.float32)
+    w["b_o"][:] = 0
+    w["w_fc2"][:] = 0
+    w["b_fc2"][:] = 0
+    keep_idx = np.array([2, 3], np.int32)
+    cu = np.array([0, 2], np.int32)
+    y, k_new, v_new = oracle.pruned_block_forward(w, 1e-6, heads, x, keep_idx, cu, kc, vc, kv_len)
+    K = np.concatenate([kc[0, :9], k_new]).astype(np.float64)
+    Vv = np.concatenate([vc[0, :9], v_new]).astype(np.float64)
+    q = w["b_qkv"][:C].astype(np.float64)
+    want = np.zeros(C)
+    for hd in range(heads):
+        sl = slice(hd * dh, (hd + 1) * dh)
+        pr = softmax(K[:, sl] @ q[sl] / math.sqrt(dh))
+        want[sl] = pr @ Vv[:, sl]
+    for m in range(2):
+        assert np.allclose(y[m] - x[0, keep_idx[m]], want, atol=1e-5)
+
+
+def test_block_layernorm_and_linear_probes():
+    w, x, kc, vc, kv_len = _block_case(seed=5, B=1, P=(0,))
+    C = 16
+    w["w_qkv"][C:2 * C] = np.eye(C, dtype=np.float32)   # k_new = LN1(x)
+    w["b_qkv"][C:2 * C] = 0
+    x[0, 0] = 3.25                                       # constant row -> LN gives beta
+    x[0, 2] = 7.0 * x[0, 1]                              # positive scaling leaves LN unchanged
+    keep_idx = np.arange(6, dtype=np.int32)
+    cu = np.array([0, 6], np.int32)
+    _, k_new, v_new = oracle.pruned_block_forward(w, 1e-12, 2, x, keep_idx, cu, kc, vc, kv_len)
+    assert np.allclose(k_new[0], w["ln1_b"], atol=1e-6)
+    assert np.allclose(k_new[1], k_new[2], atol=1e-5)
+    unit = (k_new[3].astype(np.float64) - w["ln1_b"]) / w["ln1_g"]
+    assert abs(unit.mean()) < 1e-6 and abs(unit.var() - 1.0) < 1e-5
+    # v_new = LN1(x) W_v^T + b_v with [out, in] weights: check with a numpy matmul
+    want_v = k_new.astype(np.float64) @ w["w_qkv"][2 * C:].astype(np.float64).T + w["b_qkv"][2 * C:]
+    assert np.allclose(v_new, want_v, atol=1e-5)
+
+
+def test_block_ffn_path_against_library():
+    w, x, kc, vc, kv_len = _block_case(seed=6, B=1, P=(3,))
+    C = 16
+    w["w_o"][:] = 0
+    w["b_o"][:] = 0                                      # x1 = x
+    keep_idx = np.array([0, 5, 6, 11], np.int32)
+    cu = np.array([0, 4], np.int32)
+    y, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len)
+    t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    xs = t(x[0, keep_idx])
+    h2 = TF.layer_norm(xs, (C,), t(w["ln2_g"]), t(w["ln2_b"]), 1e-6)
+    f = TF.linear(TF.gelu(TF.linear(h2, t(w["w_fc1"]), t(w["b_fc1"])), approximate="tanh"),
+                  t(w["w_fc2"]), t(w["b_fc2"]))
+    assert np.allclose(y, (xs + f).numpy(), atol=1e-5)
+
+
+def test_block_kept_set_permutation_equivariance():
+    # permuting the tokens of x_in together with keep_idx leaves every kept row's output unchanged
+    w, x, kc, vc, kv_len = _block_case(seed=7, B=1, P=(5,))
+    keep_idx = np.array([1, 3, 8, 10], np.int32)
+    cu = np.array([0, 4], np.int32)
+    y, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len)
+    perm = np.random.default_rng(0).permutation(12)
+    inv = np.argsort(perm)
+    x_p = x[:, perm]
+    keep_p = inv[keep_idx].astype(np.int32)              # same tokens, new positions, same order
+    y_p, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x_p, keep_p, cu, kc, vc, kv_len)
+    assert np.allclose(y, y_p, atol=1e-6)
+
+
+# ---------------------------------------------------------------- restore (Eq. 15-16)
+def _restore_case(seed, B, hp, wp, h, w, C, k):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((B, h * w, C)).astype(np.float32)
+    cache = rng.standard_normal((B, hp, wp, C)).astype(np.float32)
+    ent = rng.standard_normal((B, h * w)).astype(np.float32)
+    keep_idx, prune_idx, cu, _ = oracle.select_topk(ent, k)
+    y = rng.standard_normal((int(cu[-1]), C)).astype(np.float32)
+    return x, cache, keep_idx, prune_idx, cu, y
+
+
+def test_restore_matches_library_bilinear_and_cache_definition():
+    B, hp, wp, h, w, C = 2, 5, 5, 8, 8, 6
+    x, cache, keep_idx, prune_idx, cu, y = _restore_case(0, B, hp, wp, h, w, C, [20, 33])
+    x_out, cache_out = oracle.restore_from_cache(x, y, keep_idx, prune_idx, cu, cache, h, w)
+    up = TF.interpolate(torch.from_numpy(cache.astype(np.float64)).permute(0, 3, 1, 2), size=(h, w),
+                        mode="bilinear", align_corners=False).permute(0, 2, 3, 1).reshape(B, h * w, C).numpy()
+    off = 0
+    for b in range(B):
+        kept = keep_idx[cu[b]:cu[b + 1]]
+        npr = h * w - len(kept)
+        pruned = prune_idx[off:off + npr]
+        off += npr
+        assert np.array_equal(x_out[b, kept], y[cu[b]:cu[b + 1]])          # kept rows bit-equal y
+        assert np.allclose(cache_out[b, kept], y[cu[b]:cu[b + 1]] - x[b, kept], atol=1e-6)
+        assert np.allclose(x_out[b, pruned], x[b, pruned] + up[b, pruned], atol=1e-5)
+        assert np.allclose(cache_out[b, pruned], up[b, pruned], atol=1e-6)
+        assert np.allclose(x_out[b] - x[b], cache_out[b], atol=1e-5)        # Eq. 15 on every row
+
+
+def test_restore_non_square_and_downscale_factor_library():
+    B, hp, wp, h, w, C = 1, 13, 13, 16, 16, 3
+    x, cache, keep_idx, prune_idx, cu, y = _restore_case(1, B, hp, wp, h, w, C, [0])
+    x_out, cache_out = oracle.restore_from_cache(x, y, keep_idx, prune_idx, cu, cache, h, w)
+    up = TF.interpolate(torch.from_numpy(cache.astype(np.float64)).permute(0, 3, 1, 2), size=(h, w),
+                        mode="bilinear", align_corners=False).permute(0, 2, 3, 1).reshape(B, h * w, C).numpy()
+    assert np.allclose(cache_out, up, atol=1e-6)
+    # rectangular source grid
+    rng = np.random.default_rng(2)
+    cache = rng.standard_normal((1, 3, 7, 2)).astype(np.float32)
+    x = np.zeros((1, 6 * 9, 2), np.float32)
+    pr = np.arange(54, dtype=np.int32)
+    _, co = oracle.restore_from_cache(x, np.zeros((0, 2), np.float32), np.zeros(0, np.int32), pr,
+                                      np.array([0, 0], np.int32), cache, 6, 9)
+    up = TF.interpolate(torch.from_numpy(cache.astype(np.float64)).permute(0, 3, 1, 2), size=(6, 9),
+                        mode="bilinear", align_corners=False).permute(0, 2, 3, 1).reshape(1, 54, 2).numpy()
+    assert np.allclose(co, up, atol=1e-6)
+
+
+def test_restore_closed_forms():
+    z0 = np.zeros(0, np.int32)
+    cu0 = np.array([0, 0], np.int32)
+    # 1-D 2 -> 4: (a, .75a+.25b, .25a+.75b, b)
+    a, b = 2.0, 10.0
+    cache = np.array([a, b], np.float32).reshape(1, 1, 2, 1)
+    x = np.zeros((1, 4, 1), np.float32)
+    _, co = oracle.restore_from_cache(x, np.zeros((0, 1), np.float32), z0, np.arange(4, dtype=np.int32),
+                                      cu0, cache, 1, 4)
+    assert np.allclose(co.ravel(), [a, .75 * a + .25 * b, .25 * a + .75 * b, b], atol=1e-6)
+    # same size -> identity; constant -> constant; 1x1 -> broadcast
+    rng = np.random.default_rng(3)
+    cache = rng.standard_normal((1, 4, 4, 2)).astype(np.float32)
+    x = rng.standard_normal((1, 16, 2)).astype(np.float32)
+    xo, co = oracle.restore_from_cache(x, np.zeros((0, 2), np.float32), z0, np.arange(16, dtype=np.int32),
+                                       cu0, cache, 4, 4)
+    assert np.array_equal(co, cache.reshape(1, 16, 2))
+    assert np.allclose(xo, x + cache.reshape(1, 16, 2), atol=1e-6)
+    const = np.full((1, 3, 3, 2), 1.75, np.float32)
+    _, co = oracle.restore_from_cache(x, np.zeros((0, 2), np.float32), z0, np.arange(16, dtype=np.int32),
+                                      cu0, const, 4, 4)
+    assert np.allclose(co, 1.75, atol=1e-7)
+    one = rng.standard_normal((1, 1, 1, 2)).astype(np.float32)
+    _, co = oracle.restore_from_cache(x, np.zeros((0, 2), np.float32), z0, np.arange(16, dtype=np.int32),
+                                      cu0, one, 4, 4)
+    assert np.allclose(co, np.broadcast_to(one.reshape(1, 1, 2), (1, 16, 2)), atol=1e-7)
+    # zero cache -> pruned rows pass through unchanged
+    xo, _ = oracle.restore_from_cache(x, np.zeros((0, 2), np.float32), z0, np.arange(16, dtype=np.int32),
+                                      cu0, np.zeros((1, 2, 2, 2), np.float32), 4, 4)
+    assert np.array_equal(xo, x)
+
+
+# ------------------------------------------------------------------- whole step
+def test_whole_step_keep_all_reproduces_dense_layer():
+    w, x, kc, vc, kv_len = _block_case(seed=8, B=2, N=16, P=(5, 2))
+    B, N, C = x.shape
+    ent, _ = oracle.scale_entropy(np.random.default_rng(0).standard_normal((B, N, 32)).astype(np.float32))
+    r = oracle.keep_ratios(oracle.SchedParams(), 3, 1, N, np.ones((B, 3), np.float32))
+    assert (r["keep"] == N).all()                       # before t_est nothing is pruned
+    keep_idx, prune_idx, cu, _ = oracle.select_topk(ent, r["keep"])
+    assert len(prune_idx) == 0
+    y, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len)
+    cache = np.random.default_rng(1).standard_normal((B, 3, 3, C)).astype(np.float32)
+    x_out, cache_out = oracle.restore_from_cache(x, y, keep_idx, prune_idx, cu, cache, 4, 4)
+    for b in range(B):
+        wy, _, _ = _torch_block(w, 1e-6, 2, x[b], kc[b, :kv_len[b]], vc[b, :kv_len[b]])
+        assert np.allclose(x_out[b], wy, atol=2e-5, rtol=1e-5)
+        assert np.allclose(cache_out[b], wy - x[b], atol=3e-5)
