@@ -1,0 +1,210 @@
+/*
+ * nova.h - C ABI of the NOVA pruned-scale step for one NVIDIA B200 (sm_100a).
+ *
+ * The library runs the work that NOVA (training-free acceleration of next-scale
+ * visual autoregressive generation) adds to, and removes from, one transformer layer
+ * at an accelerated scale:
+ *
+ *   nova_scale_entropy      Eq. 4, Eq. 7   per-token entropy and per-image mean
+ *   nova_keep_ratios        Eq. 8-13       inflection trigger, scale/layer ratios, keep counts
+ *   nova_select_topk        text after Eq. 3 / Eq. 13: keep the highest-entropy tokens
+ *   nova_pruned_block_forward   Eq. 14     the layer on the kept tokens only
+ *   nova_restore_from_cache     Eq. 15-16  fill pruned rows from the residual cache
+ *
+ * General rules
+ *  - Plain C ABI. No call throws, aborts or traps the GPU. Every call returns a
+ *    nova_status; nova_last_error() gives a text for the last failure on a context.
+ *  - "device" pointers are CUDA device pointers owned by the caller; "host" pointers
+ *    are ordinary host memory owned by the caller. The library never frees or keeps
+ *    a caller pointer beyond the call, except the workspace given to
+ *    nova_set_workspace(), which it uses until replaced or the context is destroyed.
+ *  - All device work is enqueued on the `stream` argument (a cudaStream_t passed as
+ *    void*; NULL is the legacy default stream) and is asynchronous with respect to
+ *    the host. Calls on one context must not overlap on the GPU: they share the
+ *    workspace and the device status word.
+ *  - bf16 tensors are row-major with the last dimension contiguous; device pointers to
+ *    bf16/f32 tensors must be 16-byte aligned. Index tensors are int32.
+ *  - Scales t and layers j are 1-based as in the paper.
+ *  - Device-side waits are bounded. If one expires the kernel records
+ *    NOVA_ERR_TIMEOUT in the context's device status word and returns; non-finite
+ *    logits record NOVA_ERR_NONFINITE. nova_device_status() reads that word.
+ */
+#ifndef NOVA_H
+#define NOVA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct nova_ctx nova_ctx;
+
+typedef enum nova_status {
+    NOVA_OK = 0,
+    NOVA_ERR_INVALID_ARG = 1,  /* null pointer, negative count, bad enum            */
+    NOVA_ERR_SHAPE = 2,        /* size outside what the kernels support             */
+    NOVA_ERR_ALIGNMENT = 3,    /* pointer or stride not 16-byte aligned             */
+    NOVA_ERR_WORKSPACE = 4,    /* workspace missing or too small                    */
+    NOVA_ERR_NONFINITE = 5,    /* +inf or NaN logit seen (device status)            */
+    NOVA_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired (device status)*/
+    NOVA_ERR_CUDA = 7          /* a CUDA runtime/driver call failed                 */
+} nova_status;
+
+typedef enum nova_dtype { NOVA_BF16 = 0, NOVA_F32 = 1 } nova_dtype;
+
+/* ---- context ------------------------------------------------------------------ */
+
+/* Creates a context bound to CUDA device `device`. Allocates a few bytes of device
+ * memory for the status word (the only allocation the library ever makes). */
+nova_status nova_create(nova_ctx** out, int device);
+void        nova_destroy(nova_ctx* ctx);
+const char* nova_last_error(const nova_ctx* ctx);
+const char* nova_status_string(nova_status s);
+
+/* Synchronises `stream`, returns the device status word (NOVA_OK, NOVA_ERR_TIMEOUT or
+ * NOVA_ERR_NONFINITE) and clears it. */
+nova_status nova_device_status(nova_ctx* ctx, void* stream);
+
+/* ---- Eq. 4 and Eq. 7: entropy ------------------------------------------------- */
+/*
+ * logits: device, [S, N, V], dtype dt, row r = s*N + i starts at element r*row_stride
+ *         (row_stride >= V; a multiple of 8 for bf16, 4 for f32).
+ * ent:    device f32 [S, N]   ent[s,i] = -sum_v p(v) ln p(v), p = softmax(row), natural log.
+ * mean:   device f32 [S] or NULL   mean[s] = (1/N) sum_i ent[s,i], summed in a fixed order.
+ * A -inf logit contributes 0. A +inf or NaN logit makes the row's entropy NaN and records
+ * NOVA_ERR_NONFINITE in the device status word. Negative zeros are returned as +0.
+ * Errors: S,N < 0 or V < 1 -> INVALID_ARG; misaligned pointer/stride -> ALIGNMENT.
+ * S*N == 0 is a no-op.
+ */
+nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nova_dtype dt,
+                               int S, int N, int V, int64_t row_stride,
+                               float* ent, float* mean, void* stream);
+
+/* ---- Eq. 8-13: trigger, ratios, keep counts (host arithmetic, double) ---------- */
+typedef struct nova_sched_params {
+    int    t_est;            /* scales kept dense to estimate the growth baseline (paper: 5) */
+    double alpha;            /* Eq. 10 fraction of the baseline (paper: 0.5)                 */
+    double tau;              /* Eq. 11 sigmoid temperature (paper: 0.8)                      */
+    double lambda;           /* Eq. 11 weight of tanh(g_t) (paper: 0.1)                      */
+    int    k_min;            /* lower bound of a keep count (default 1)                      */
+    double ratio_max;        /* upper clamp of a reduction ratio (default 1)                 */
+    int    force_act_scale;  /* 0: adaptive trigger; >0: fixed activation scale              */
+    double force_keep_ratio; /* <0: Eq. 11-13; in [0,1]: reduction ratio = 1 - this          */
+} nova_sched_params;
+
+/* Fills *p with the paper's hyper-parameters and this library's default clamps. */
+void nova_sched_params_default(nova_sched_params* p);
+
+/*
+ * All pointers are host memory. hbar_scale [B, t]: mean entropies of scales 1..t
+ * (current included); hbar_layer [B, j]: mean entropies of layers 1..j of scale t
+ * (may be NULL when j == 1).
+ * Per image b:
+ *   g_u = H_u - H_{u-1}; eta = mean(g_2..g_{t_est}); t_star[b] = first u in [t_est+1, t]
+ *   with (g_u + g_{u-1})/2 <= alpha*eta, or 0; act_scale[b] = t_star+1 or 0 (Eq. 8-10).
+ *   If t >= act_scale > 0: ratio_scale = sigmoid((t-act_scale)/tau) - lambda*tanh(g_t)
+ *   (Eq. 11); ratio_layer = ratio_scale for j == 1, else ratio_scale - Delta*ratio_scale with
+ *   Delta = (H_{t,j} - mu)/mu, mu = mean of layers 1..j-1 (mu == 0 -> Delta = 0) (Eq. 12-13).
+ *   Otherwise both ratios are 0.
+ *   keep[b] = N_t - floor(clamp(ratio_layer, 0, ratio_max) * N_t), clamped to [k_min, N_t].
+ * Ratios are reduction ratios (fraction pruned). Errors: null pointer, B < 0, t < 1,
+ * j < 1, N_t < 1, t_est < 2, tau <= 0 -> INVALID_ARG.
+ */
+nova_status nova_keep_ratios(const nova_sched_params* p, int B, int t, int j, int N_t,
+                             const float* hbar_scale, const float* hbar_layer,
+                             int32_t* t_star, int32_t* act_scale,
+                             double* ratio_scale, double* ratio_layer, int32_t* keep);
+
+/* ---- keep the highest-entropy tokens ------------------------------------------- */
+/*
+ * ent:  device f32 [S, N] (finite).   k: HOST int32 [S], 0 <= k[s] <= N.
+ * Token i of segment s is kept iff fewer than k[s] tokens j of the segment have
+ * ent[j] > ent[i] or (ent[j] == ent[i] and j < i)   (+0 and -0 compare equal).
+ * keep_idx:  device int32 [sum k]        kept in-segment indices, ascending, segments concatenated
+ * prune_idx: device int32 [S*N - sum k]  pruned in-segment indices, ascending, concatenated
+ * cu_keep:   device int32 [S+1]          cu_keep[s] = k[0] + ... + k[s-1]
+ * pos:       device int32 [S, N] or NULL position of i in its segment's kept list, -1 if pruned
+ * Errors: N > 16384 -> SHAPE; k[s] outside [0, N] -> INVALID_ARG. S*N == 0 writes only cu_keep.
+ */
+nova_status nova_select_topk(nova_ctx* ctx, const float* ent, int S, int N, const int32_t* k,
+                             int32_t* keep_idx, int32_t* prune_idx, int32_t* cu_keep,
+                             int32_t* pos, void* stream);
+
+/* ---- Eq. 14: the layer on the kept tokens -------------------------------------- */
+typedef struct nova_block_weights {  /* device bf16; matrices are [out, in] row-major */
+    const void *ln1_g, *ln1_b;       /* [C]            */
+    const void *w_qkv, *b_qkv;       /* [3C, C], [3C]  rows 0..C-1 -> q, C..2C-1 -> k, 2C.. -> v */
+    const void *w_o, *b_o;           /* [C, C], [C]    */
+    const void *ln2_g, *ln2_b;       /* [C]            */
+    const void *w_fc1, *b_fc1;       /* [F, C], [F]    */
+    const void *w_fc2, *b_fc2;       /* [C, F], [C]    */
+    float eps;                       /* LayerNorm epsilon */
+} nova_block_weights;
+
+typedef struct nova_block_shape {
+    int B;        /* images                                         */
+    int N;        /* tokens per image at this scale                 */
+    int C;        /* width; multiple of 64                          */
+    int n_heads;  /* C / n_heads must be 64 or 128                  */
+    int F;        /* MLP hidden width; multiple of 64               */
+    int Lmax;     /* rows per image of the K/V caches               */
+    int M;        /* total kept tokens = cu_keep[B] (host knows it) */
+} nova_block_shape;
+
+/* Bytes of workspace nova_pruned_block_forward needs for this shape (0 on bad shape). */
+size_t      nova_block_workspace_bytes(const nova_block_shape* s);
+/* Gives the context a device buffer (256-byte aligned) used as scratch by later calls. */
+nova_status nova_set_workspace(nova_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/*
+ * Pre-LayerNorm transformer block on the compacted kept rows:
+ *   Xc = rows keep_idx of x_in;  h = LN(Xc);  [q|k|v] = h W_qkv^T + b_qkv;
+ *   keys/values of image b = k_cache[b, 0:kv_len[b]] followed by the kept tokens' own k, v;
+ *   o = softmax(q K^T / sqrt(dh)) V per head (no mask);  x1 = Xc + o W_o^T + b_o;
+ *   y = x1 + GELU_tanh(LN(x1) W_fc1^T + b_fc1) W_fc2^T + b_fc2.
+ * x_in:     device bf16 [B, N, C]
+ * keep_idx: device int32 [M], cu_keep: device int32 [B+1] (as written by nova_select_topk)
+ * k_cache, v_cache: device bf16 [B, Lmax, C]; rows [0, kv_len[b]) are valid. The kept
+ *           tokens' k and v are always written to rows kv_len[b] .. kv_len[b]+k_b-1
+ *           (so kv_len[b] + k_b <= Lmax is required and is checked on the device:
+ *           an overflowing image records NOVA_ERR_SHAPE in the device status word and
+ *           its rows are not written).
+ * kv_len:   device int32 [B]; if append_kv != 0 it is advanced by k_b at the end.
+ * y_kept:   device bf16 [M, C], compacted order.
+ * Arithmetic: bf16 operands, fp32 accumulation on the tensor cores; LayerNorm, softmax,
+ * GELU and residual adds in fp32; activations between stages stored as bf16.
+ * Errors: bad shape -> SHAPE; workspace smaller than nova_block_workspace_bytes ->
+ * WORKSPACE; misaligned pointers -> ALIGNMENT. M == 0 is a no-op.
+ */
+nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block_weights* w,
+                                      const nova_block_shape* s, const void* x_in,
+                                      const int32_t* keep_idx, const int32_t* cu_keep,
+                                      void* k_cache, void* v_cache, int32_t* kv_len,
+                                      int append_kv, void* y_kept, void* stream);
+
+/* ---- Eq. 15-16: residual cache reuse -------------------------------------------- */
+/*
+ * x_in:       device bf16 [B, h*w, C]   layer input
+ * y_kept:     device bf16 [M, C]        layer output on the kept rows (compacted)
+ * keep_idx / prune_idx / cu_keep: device int32, as written by nova_select_topk (S = B, N = h*w)
+ * cache_prev: device bf16 [B, hp, wp, C]  previous scale's residual cache of this layer;
+ *             may be NULL only if nothing is pruned.
+ * x_out:      device bf16 [B, h*w, C]:  kept rows = y_kept; pruned rows = x_in + U, where U is
+ *             cache_prev resized to (h, w) bilinearly with half-pixel centres
+ *             (src = (dst + 0.5) * hp / h - 0.5, clamped at the borders)            (Eq. 16)
+ * cache_out:  device bf16 [B, h*w, C] or NULL:  x_out - x_in on kept rows (computed in fp32
+ *             from y and x_in), U on pruned rows                                    (Eq. 15)
+ * x_out must not alias x_in. C must be a multiple of 8.
+ */
+nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, const void* y_kept,
+                                    const int32_t* keep_idx, const int32_t* prune_idx,
+                                    const int32_t* cu_keep, const void* cache_prev,
+                                    int hp, int wp, int h, int w, int C, int B, int M,
+                                    void* x_out, void* cache_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NOVA_H */

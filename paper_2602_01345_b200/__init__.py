@@ -1,0 +1,12 @@
+"""B200-native NOVA pruned-scale step: thin Python binding over the C-ABI library libnova.so.
+
+The binding only marshals arguments (torch tensors -> raw pointers and sizes); every step of
+the path runs in the library's CUDA kernels. There is no CPU fallback: if libnova.so is
+missing or cannot be loaded, importing this package fails.
+"""
+from .binding import (  # noqa: F401
+    NovaError, Context, SchedParams, BlockWeights, BlockShape,
+    nova_scale_entropy, nova_keep_ratios, nova_select_topk,
+    nova_pruned_block_forward, nova_restore_from_cache, nova_block_workspace_bytes,
+    lib_path, STATUS_NAMES,
+)

@@ -1,0 +1,247 @@
+"""ctypes binding of include/nova.h. Names and argument order follow the C ABI."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libnova.so")
+
+STATUS_NAMES = {0: "NOVA_OK", 1: "NOVA_ERR_INVALID_ARG", 2: "NOVA_ERR_SHAPE", 3: "NOVA_ERR_ALIGNMENT",
+                4: "NOVA_ERR_WORKSPACE", 5: "NOVA_ERR_NONFINITE", 6: "NOVA_ERR_TIMEOUT", 7: "NOVA_ERR_CUDA"}
+NOVA_BF16, NOVA_F32 = 0, 1
+
+
+class NovaError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} not found: build it with `python -m paper_2602_01345_b200.build` "
+        "(there is no CPU fallback for the NOVA kernels)")
+_lib = C.CDLL(_LIB_PATH)
+
+
+class _SchedParams(C.Structure):
+    _fields_ = [("t_est", C.c_int), ("alpha", C.c_double), ("tau", C.c_double), ("lam", C.c_double),
+                ("k_min", C.c_int), ("ratio_max", C.c_double), ("force_act_scale", C.c_int),
+                ("force_keep_ratio", C.c_double)]
+
+
+_WEIGHT_FIELDS = ("ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o",
+                  "ln2_g", "ln2_b", "w_fc1", "b_fc1", "w_fc2", "b_fc2")
+
+
+class _BlockWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _WEIGHT_FIELDS] + [("eps", C.c_float)]
+
+
+class _BlockShape(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("B", "N", "C", "n_heads", "F", "Lmax", "M")]
+
+
+_vp, _i, _i64 = C.c_void_p, C.c_int, C.c_int64
+_lib.nova_create.argtypes = [C.POINTER(_vp), _i]
+_lib.nova_create.restype = _i
+_lib.nova_destroy.argtypes = [_vp]
+_lib.nova_destroy.restype = None
+_lib.nova_last_error.argtypes = [_vp]
+_lib.nova_last_error.restype = C.c_char_p
+_lib.nova_status_string.argtypes = [_i]
+_lib.nova_status_string.restype = C.c_char_p
+_lib.nova_device_status.argtypes = [_vp, _vp]
+_lib.nova_device_status.restype = _i
+_lib.nova_set_workspace.argtypes = [_vp, _vp, C.c_size_t]
+_lib.nova_set_workspace.restype = _i
+_lib.nova_block_workspace_bytes.argtypes = [C.POINTER(_BlockShape)]
+_lib.nova_block_workspace_bytes.restype = C.c_size_t
+_lib.nova_sched_params_default.argtypes = [C.POINTER(_SchedParams)]
+_lib.nova_sched_params_default.restype = None
+_lib.nova_scale_entropy.argtypes = [_vp, _vp, _i, _i, _i, _i, _i64, _vp, _vp, _vp]
+_lib.nova_scale_entropy.restype = _i
+_lib.nova_keep_ratios.argtypes = [C.POINTER(_SchedParams), _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.nova_keep_ratios.restype = _i
+_lib.nova_select_topk.argtypes = [_vp, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.nova_select_topk.restype = _i
+_lib.nova_pruned_block_forward.argtypes = [_vp, C.POINTER(_BlockWeights), C.POINTER(_BlockShape), _vp, _vp, _vp,
+                                           _vp, _vp, _vp, _i, _vp, _vp]
+_lib.nova_pruned_block_forward.restype = _i
+_lib.nova_restore_from_cache.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp]
+_lib.nova_restore_from_cache.restype = _i
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors passed to the NOVA library must be contiguous"
+    return t.data_ptr() if t.numel() > 0 else None
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+@dataclass
+class SchedParams:
+    """Hyper-parameters of the activation trigger and ratio functions (paper defaults)."""
+    t_est: int = 5
+    alpha: float = 0.5
+    tau: float = 0.8
+    lam: float = 0.1
+    k_min: int = 1
+    ratio_max: float = 1.0
+    force_act_scale: int = 0
+    force_keep_ratio: float = -1.0
+
+    def _c(self):
+        return _SchedParams(self.t_est, self.alpha, self.tau, self.lam, self.k_min, self.ratio_max,
+                            self.force_act_scale, self.force_keep_ratio)
+
+
+@dataclass
+class BlockShape:
+    B: int
+    N: int
+    C: int
+    n_heads: int
+    F: int
+    Lmax: int
+    M: int
+
+    def _c(self):
+        return _BlockShape(self.B, self.N, self.C, self.n_heads, self.F, self.Lmax, self.M)
+
+
+class BlockWeights:
+    """Holds the twelve bf16 device tensors of one block and the C struct that points to them."""
+
+    def __init__(self, tensors: dict, eps: float = 1e-6):
+        self.tensors = {n: tensors[n] for n in _WEIGHT_FIELDS}
+        for n, t in self.tensors.items():
+            assert t.dtype == torch.bfloat16 and t.is_cuda and t.is_contiguous(), n
+        self.eps = float(eps)
+        self.c = _BlockWeights(*[self.tensors[n].data_ptr() for n in _WEIGHT_FIELDS], self.eps)
+
+
+class Context:
+    """Owns one nova_ctx (one CUDA device) and, optionally, a workspace tensor."""
+
+    def __init__(self, device: int = 0):
+        self.device = int(device)
+        h = _vp()
+        with torch.cuda.device(self.device):
+            st = _lib.nova_create(C.byref(h), self.device)
+        if st != 0:
+            raise NovaError(st, "nova_create failed")
+        self.handle = h
+        self._workspace = None
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.nova_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def check(self, status: int):
+        if status != 0:
+            raise NovaError(status, _lib.nova_last_error(self.handle).decode())
+
+    def set_workspace(self, tensor):
+        """Gives the library a device scratch buffer (kept alive by this object)."""
+        self._workspace = tensor
+        self.check(_lib.nova_set_workspace(self.handle, _ptr(tensor), tensor.numel() * tensor.element_size()
+                                           if tensor is not None else 0))
+
+    def ensure_workspace(self, shape: BlockShape):
+        need = nova_block_workspace_bytes(shape)
+        if self._workspace is None or self._workspace.numel() < need:
+            self.set_workspace(torch.empty(need + 256, dtype=torch.uint8, device=f"cuda:{self.device}"))
+
+    def device_status(self, stream=None) -> int:
+        """Synchronises the stream and returns (and clears) the device status word as a status code."""
+        return int(_lib.nova_device_status(self.handle, _stream(stream)))
+
+
+def nova_block_workspace_bytes(shape: BlockShape) -> int:
+    c = shape._c()
+    return int(_lib.nova_block_workspace_bytes(C.byref(c)))
+
+
+def nova_scale_entropy(ctx: Context, logits, ent, mean=None, stream=None):
+    """logits [S, N, V] (bf16 or f32, last dim contiguous) -> ent [S, N] f32, mean [S] f32."""
+    S, N, V = logits.shape
+    assert logits.stride(2) == 1 and logits.stride(0) == N * logits.stride(1)
+    dt = {torch.bfloat16: NOVA_BF16, torch.float32: NOVA_F32}[logits.dtype]
+    assert ent.dtype == torch.float32 and ent.is_contiguous() and ent.numel() == S * N
+    ctx.check(_lib.nova_scale_entropy(ctx.handle, logits.data_ptr() if logits.numel() else None, dt, S, N, V,
+                                      logits.stride(1), _ptr(ent), _ptr(mean), _stream(stream)))
+
+
+def nova_keep_ratios(p: SchedParams, t: int, j: int, N_t: int, hbar_scale, hbar_layer=None):
+    """Host arithmetic of the trigger and ratio functions. hbar_* are CPU float32 tensors.
+
+    Returns dict of CPU tensors: t_star, act_scale (int32), ratio_scale, ratio_layer (float64), keep (int32).
+    """
+    hs = hbar_scale.to("cpu", torch.float32).contiguous()
+    B = hs.shape[0]
+    assert hs.shape == (B, t)
+    hl = None
+    if hbar_layer is not None:
+        hl = hbar_layer.to("cpu", torch.float32).contiguous()
+        assert hl.shape == (B, j)
+    out = dict(t_star=torch.zeros(B, dtype=torch.int32), act_scale=torch.zeros(B, dtype=torch.int32),
+               ratio_scale=torch.zeros(B, dtype=torch.float64), ratio_layer=torch.zeros(B, dtype=torch.float64),
+               keep=torch.zeros(B, dtype=torch.int32))
+    c = p._c()
+    st = _lib.nova_keep_ratios(C.byref(c), B, t, j, N_t, _ptr(hs), _ptr(hl), _ptr(out["t_star"]),
+                               _ptr(out["act_scale"]), _ptr(out["ratio_scale"]), _ptr(out["ratio_layer"]),
+                               _ptr(out["keep"]))
+    if st != 0:
+        raise NovaError(st, "nova_keep_ratios")
+    return out
+
+
+def nova_select_topk(ctx: Context, ent, k, keep_idx, prune_idx, cu_keep, pos=None, stream=None):
+    """ent [S, N] f32 device; k: CPU int32 tensor [S]; outputs are device int32 tensors."""
+    S, N = ent.shape
+    assert ent.dtype == torch.float32 and ent.is_contiguous()
+    kk = k.to("cpu", torch.int32).contiguous()
+    assert kk.numel() == S
+    ctx.check(_lib.nova_select_topk(ctx.handle, _ptr(ent), S, N, _ptr(kk), _ptr(keep_idx), _ptr(prune_idx),
+                                    _ptr(cu_keep), _ptr(pos), _stream(stream)))
+
+
+def nova_pruned_block_forward(ctx: Context, w: BlockWeights, shape: BlockShape, x_in, keep_idx, cu_keep,
+                              k_cache, v_cache, kv_len, append_kv, y_kept, stream=None):
+    c = shape._c()
+    ctx.check(_lib.nova_pruned_block_forward(ctx.handle, C.byref(w.c), C.byref(c), _ptr(x_in), _ptr(keep_idx),
+                                             _ptr(cu_keep), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len),
+                                             int(bool(append_kv)), _ptr(y_kept), _stream(stream)))
+
+
+def nova_restore_from_cache(ctx: Context, x_in, y_kept, keep_idx, prune_idx, cu_keep, cache_prev, h, w,
+                            x_out, cache_out=None, stream=None):
+    B, N, Cc = x_in.shape
+    assert N == h * w
+    M = int(keep_idx.numel())
+    hp, wp = (cache_prev.shape[1], cache_prev.shape[2]) if cache_prev is not None else (0, 0)
+    ctx.check(_lib.nova_restore_from_cache(ctx.handle, _ptr(x_in), _ptr(y_kept), _ptr(keep_idx), _ptr(prune_idx),
+                                           _ptr(cu_keep), _ptr(cache_prev), hp, wp, h, w, Cc, B, M,
+                                           _ptr(x_out), _ptr(cache_out), _stream(stream)))

@@ -1,0 +1,174 @@
+// Context management and the host-side schedule arithmetic (Eq. 8-13).
+#include "common.cuh"
+
+#include <math.h>
+#include <new>
+
+extern "C" {
+
+const char* nova_status_string(nova_status s)
+{
+    switch (s) {
+        case NOVA_OK: return "ok";
+        case NOVA_ERR_INVALID_ARG: return "invalid argument";
+        case NOVA_ERR_SHAPE: return "unsupported shape";
+        case NOVA_ERR_ALIGNMENT: return "misaligned pointer or stride";
+        case NOVA_ERR_WORKSPACE: return "workspace missing or too small";
+        case NOVA_ERR_NONFINITE: return "non-finite logit";
+        case NOVA_ERR_TIMEOUT: return "device-side wait expired";
+        case NOVA_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+nova_status nova_create(nova_ctx** out, int device)
+{
+    if (!out) return NOVA_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess || device < 0 || device >= count) return NOVA_ERR_CUDA;
+    nova_ctx* ctx = new (std::nothrow) nova_ctx();
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    memset(ctx, 0, sizeof(*ctx));
+    ctx->device = device;
+    if (cudaSetDevice(device) != cudaSuccess ||
+        cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
+        cudaMemset(ctx->dev_status, 0, 256) != cudaSuccess) {
+        delete ctx;
+        return NOVA_ERR_CUDA;
+    }
+    cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device);
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn) {
+        cudaFree(ctx->dev_status);
+        delete ctx;
+        return NOVA_ERR_CUDA;
+    }
+    ctx->encode_tiled = fn;
+    *out = ctx;
+    return NOVA_OK;
+}
+
+void nova_destroy(nova_ctx* ctx)
+{
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->dev_status);
+    delete ctx;
+}
+
+const char* nova_last_error(const nova_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+nova_status nova_device_status(nova_ctx* ctx, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned int word = 0;
+    NOVA_CUDA_CHECK(ctx, cudaMemcpyAsync(&word, ctx->dev_status, sizeof(word), cudaMemcpyDeviceToHost, st));
+    NOVA_CUDA_CHECK(ctx, cudaStreamSynchronize(st));
+    if (word) NOVA_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->dev_status, 0, sizeof(word), st));
+    if (word & NOVA_DEV_TIMEOUT) return nova_fail(ctx, NOVA_ERR_TIMEOUT, "a device-side wait expired");
+    if (word & NOVA_DEV_SHAPE) return nova_fail(ctx, NOVA_ERR_SHAPE, "K/V cache overflow on the device");
+    if (word & NOVA_DEV_NONFINITE) return nova_fail(ctx, NOVA_ERR_NONFINITE, "non-finite logit");
+    return NOVA_OK;
+}
+
+nova_status nova_set_workspace(nova_ctx* ctx, void* dev_ptr, size_t bytes)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if (dev_ptr && (((uintptr_t)dev_ptr) & 255u)) return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "workspace must be 256-byte aligned");
+    ctx->workspace = dev_ptr;
+    ctx->workspace_bytes = dev_ptr ? bytes : 0;
+    return NOVA_OK;
+}
+
+void nova_sched_params_default(nova_sched_params* p)
+{
+    if (!p) return;
+    p->t_est = 5;
+    p->alpha = 0.5;
+    p->tau = 0.8;
+    p->lambda = 0.1;
+    p->k_min = 1;
+    p->ratio_max = 1.0;
+    p->force_act_scale = 0;
+    p->force_keep_ratio = -1.0;
+}
+
+// Eq. 8-13 for one image. hs[u-1] is the mean entropy of scale u; hl[k-1] that of layer k.
+static void schedule_one(const nova_sched_params& p, int t, int j, int n_tokens, const float* hs,
+                         const float* hl, int32_t* t_star, int32_t* act_scale, double* ratio_scale,
+                         double* ratio_layer, int32_t* keep)
+{
+    // growth rates g[u] for u = 2..t (Eq. 8)
+    double growth_now = 0.0;
+    int found = 0;
+    if (t > p.t_est) {
+        // baseline: the growth rates up to t_est telescope, but are summed one by one so the
+        // rounding matches a term-by-term evaluation of Eq. 9
+        double base = 0.0;
+        for (int u = 2; u <= p.t_est; ++u) base += (double)hs[u - 1] - (double)hs[u - 2];
+        base /= (double)(p.t_est - 1);
+        const double threshold = p.alpha * base;
+        for (int u = p.t_est + 1; u <= t && !found; ++u) {
+            const double gu = (double)hs[u - 1] - (double)hs[u - 2];
+            const double gprev = (double)hs[u - 2] - (double)hs[u - 3];
+            if ((gu + gprev) / 2.0 <= threshold) found = u;   // Eq. 10
+        }
+    }
+    int act = found ? found + 1 : 0;
+    if (p.force_act_scale > 0) {
+        act = p.force_act_scale;
+        found = act - 1;
+    }
+    *t_star = found;
+    *act_scale = act;
+
+    double rs = 0.0, rl = 0.0;
+    if (act > 0 && t >= act) {
+        if (p.force_keep_ratio >= 0.0) {
+            rs = rl = 1.0 - p.force_keep_ratio;
+        } else {
+            if (t >= 2) growth_now = (double)hs[t - 1] - (double)hs[t - 2];
+            const double arg = ((double)t - (double)act) / p.tau;
+            rs = 1.0 / (1.0 + exp(-arg)) - p.lambda * tanh(growth_now);   // Eq. 11
+            rl = rs;
+            if (j >= 2) {                                                // Eq. 12-13
+                double mu = 0.0;
+                for (int k = 1; k < j; ++k) mu += (double)hl[k - 1];
+                mu /= (double)(j - 1);
+                const double delta = (mu != 0.0) ? ((double)hl[j - 1] - mu) / mu : 0.0;
+                rl = rs - delta * rs;
+            }
+        }
+    }
+    *ratio_scale = rs;
+    *ratio_layer = rl;
+    double r = rl < 0.0 ? 0.0 : rl;
+    if (r > p.ratio_max) r = p.ratio_max;
+    long kept = (long)n_tokens - (long)floor(r * (double)n_tokens);
+    if (kept < p.k_min) kept = p.k_min;
+    if (kept > n_tokens) kept = n_tokens;
+    *keep = (int32_t)kept;
+}
+
+nova_status nova_keep_ratios(const nova_sched_params* p, int B, int t, int j, int N_t,
+                             const float* hbar_scale, const float* hbar_layer,
+                             int32_t* t_star, int32_t* act_scale,
+                             double* ratio_scale, double* ratio_layer, int32_t* keep)
+{
+    if (!p || B < 0 || t < 1 || j < 1 || N_t < 1 || p->t_est < 2 || !(p->tau > 0.0)) return NOVA_ERR_INVALID_ARG;
+    if (B == 0) return NOVA_OK;
+    if (!hbar_scale || !t_star || !act_scale || !ratio_scale || !ratio_layer || !keep) return NOVA_ERR_INVALID_ARG;
+    if (j >= 2 && !hbar_layer && p->force_keep_ratio < 0.0) return NOVA_ERR_INVALID_ARG;
+    for (int b = 0; b < B; ++b)
+        schedule_one(*p, t, j, N_t, hbar_scale + (size_t)b * t,
+                     hbar_layer ? hbar_layer + (size_t)b * j : nullptr,
+                     t_star + b, act_scale + b, ratio_scale + b, ratio_layer + b, keep + b);
+    return NOVA_OK;
+}
+
+}  // extern "C"

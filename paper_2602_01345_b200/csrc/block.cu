@@ -1,0 +1,253 @@
+// Eq. 14 on the kept tokens: gather + LayerNorm, QKV projection with K/V cache append,
+// attention, output projection + residual, LayerNorm, MLP with tanh-GELU + residual.
+// This file holds the small memory-bound kernels (row maps, LayerNorm, kv_len update), the
+// workspace layout and the launch sequence; the contractions live in gemm.cu / attention.cu.
+#include "common.cuh"
+
+namespace {
+
+// ---- row maps ---------------------------------------------------------------------------
+// src_row[r] = b*N + keep_idx[r]            row of x_in feeding compacted row r
+// kv_row[r]  = b*Lmax + kv_len[b] + (r - cu_keep[b])   cache row receiving r's k and v
+//              (-1 and a SHAPE flag if the image's cache would overflow)
+__global__ void build_row_maps(const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ cu_keep,
+                               const int32_t* __restrict__ kv_len, int B, int N, int Lmax, int M,
+                               int32_t* __restrict__ src_row, int32_t* __restrict__ kv_row,
+                               unsigned int* status)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= M) return;
+    int lo = 0, hi = B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (cu_keep[mid] <= r) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    src_row[r] = b * N + keep_idx[r];
+    const int k_b = cu_keep[b + 1] - cu_keep[b];
+    if (kv_len[b] + k_b > Lmax) {
+        kv_row[r] = -1;
+        atomicOr(status, NOVA_DEV_SHAPE);
+    } else {
+        kv_row[r] = b * Lmax + kv_len[b] + (r - cu_keep[b]);
+    }
+}
+
+__global__ void advance_kv_len(const int32_t* __restrict__ cu_keep, int32_t* __restrict__ kv_len, int B, int Lmax)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int k_b = cu_keep[b + 1] - cu_keep[b];
+    if (kv_len[b] + k_b <= Lmax) kv_len[b] += k_b;
+}
+
+// ---- LayerNorm ----------------------------------------------------------------------------
+// One warp per row; the row (C <= 32*8*VEC bf16) stays in registers between the mean, the
+// variance and the normalisation, so x is read once and out written once.
+constexpr int kLnWarps = 8;
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <int VEC>
+__global__ void __launch_bounds__(kLnWarps * 32)
+layernorm_rows(const uint4* __restrict__ x, const int32_t* __restrict__ src_row, const uint4* __restrict__ gamma,
+               const uint4* __restrict__ beta, float eps, int M, int vec_per_row, uint4* __restrict__ out)
+{
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
+    if (r >= M) return;
+    const long src = src_row ? (long)src_row[r] : (long)r;
+    const uint4* xr = x + src * vec_per_row;
+    float v[VEC][8];
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) {
+        const int c = i * 32 + lane;
+        uint4 raw = make_uint4(0, 0, 0, 0);
+        if (c < vec_per_row) raw = xr[c];
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            v[i][2 * q] = __uint_as_float(w[q] << 16);
+            v[i][2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
+            sum += v[i][2 * q] + v[i][2 * q + 1];
+        }
+    }
+    const float n = (float)(vec_per_row * 8);
+    const float mean = warp_sum(sum) / n;
+    float sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) {
+        if (i * 32 + lane < vec_per_row) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { const float d = v[i][q] - mean; sq += d * d; }
+        }
+    }
+    const float rstd = rsqrtf(warp_sum(sq) / n + eps);
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) {
+        const int c = i * 32 + lane;
+        if (c < vec_per_row) {
+            const uint4 g = gamma[c], bt = beta[c];
+            const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, bw[4] = {bt.x, bt.y, bt.z, bt.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float y0 = (v[i][2 * q] - mean) * rstd * __uint_as_float(gw[q] << 16) + __uint_as_float(bw[q] << 16);
+                const float y1 = (v[i][2 * q + 1] - mean) * rstd * __uint_as_float(gw[q] & 0xffff0000u) +
+                                 __uint_as_float(bw[q] & 0xffff0000u);
+                __nv_bfloat162 t = __floats2bfloat162_rn(y0, y1);
+                o[q] = *reinterpret_cast<uint32_t*>(&t);
+            }
+            out[(long)r * vec_per_row + c] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
+}
+
+struct Workspace {
+    int32_t* src_row;
+    int32_t* kv_row;
+    __nv_bfloat16 *h, *q, *o, *x1, *f;
+    size_t bytes;
+};
+
+inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+Workspace carve(void* base, int M, int C, int F)
+{
+    Workspace w;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { void* p = base ? (char*)base + off : nullptr; off += align_up(bytes); return p; };
+    const size_t Mp = (size_t)((M + 127) / 128) * 128;   // whole 128-row tiles
+    w.src_row = (int32_t*)take(Mp * 4);
+    w.kv_row = (int32_t*)take(Mp * 4);
+    w.h = (__nv_bfloat16*)take(Mp * C * 2);
+    w.q = (__nv_bfloat16*)take(Mp * C * 2);
+    w.o = (__nv_bfloat16*)take(Mp * C * 2);
+    w.x1 = (__nv_bfloat16*)take(Mp * C * 2);
+    w.f = (__nv_bfloat16*)take(Mp * (size_t)F * 2);
+    w.bytes = off;
+    return w;
+}
+
+bool shape_ok(const nova_block_shape* s)
+{
+    if (!s || s->B < 1 || s->N < 1 || s->C < 64 || s->n_heads < 1 || s->F < 64 || s->Lmax < 1 || s->M < 0) return false;
+    if (s->C % 64 || s->F % 64 || s->C % s->n_heads) return false;
+    const int dh = s->C / s->n_heads;
+    if (dh != 64 && dh != 128) return false;
+    if (s->C > 8192) return false;
+    if ((long)s->M > (long)s->B * s->N) return false;
+    return true;
+}
+
+}  // namespace
+
+nova_status nova_launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const int32_t* src_row,
+                           const __nv_bfloat16* g, const __nv_bfloat16* b, float eps, int M, int C,
+                           __nv_bfloat16* out, cudaStream_t st)
+{
+    if (M <= 0) return NOVA_OK;
+    const int vec = C / 8;
+    const int per_lane = (vec + 31) / 32;
+    const dim3 grid((M + kLnWarps - 1) / kLnWarps), block(kLnWarps * 32);
+#define NOVA_LN_CASE(V) layernorm_rows<V><<<grid, block, 0, st>>>((const uint4*)x, src_row, (const uint4*)g, (const uint4*)b, eps, M, vec, (uint4*)out)
+    if (per_lane <= 2) NOVA_LN_CASE(2);
+    else if (per_lane <= 4) NOVA_LN_CASE(4);
+    else if (per_lane <= 8) NOVA_LN_CASE(8);
+    else if (per_lane <= 16) NOVA_LN_CASE(16);
+    else if (per_lane <= 32) NOVA_LN_CASE(32);
+    else return nova_fail(ctx, NOVA_ERR_SHAPE, "layernorm: C > 8192");
+#undef NOVA_LN_CASE
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    return NOVA_OK;
+}
+
+extern "C" size_t nova_block_workspace_bytes(const nova_block_shape* s)
+{
+    if (!shape_ok(s)) return 0;
+    return carve(nullptr, s->M, s->C, s->F).bytes;
+}
+
+extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block_weights* w,
+                                                 const nova_block_shape* s, const void* x_in,
+                                                 const int32_t* keep_idx, const int32_t* cu_keep,
+                                                 void* k_cache, void* v_cache, int32_t* kv_len,
+                                                 int append_kv, void* y_kept, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if (!w || !s) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward: null weights or shape");
+    if (!shape_ok(s)) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_pruned_block_forward: unsupported shape");
+    if (s->M == 0) return NOVA_OK;
+    if (!x_in || !keep_idx || !cu_keep || !k_cache || !v_cache || !kv_len || !y_kept)
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward: null tensor");
+    const void* wp[] = {w->ln1_g, w->ln1_b, w->w_qkv, w->b_qkv, w->w_o, w->b_o,
+                        w->ln2_g, w->ln2_b, w->w_fc1, w->b_fc1, w->w_fc2, w->b_fc2};
+    for (const void* ptr : wp) {
+        if (!ptr) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward: null weight");
+        if (!nova_aligned16(ptr)) return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_pruned_block_forward: weight not 16-byte aligned");
+    }
+    if (!nova_aligned16(x_in) || !nova_aligned16(k_cache) || !nova_aligned16(v_cache) || !nova_aligned16(y_kept))
+        return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_pruned_block_forward: tensor not 16-byte aligned");
+    Workspace ws = carve(ctx->workspace, s->M, s->C, s->F);
+    if (!ctx->workspace || ctx->workspace_bytes < ws.bytes)
+        return nova_fail(ctx, NOVA_ERR_WORKSPACE, "nova_pruned_block_forward: workspace missing or too small");
+
+    cudaStream_t st = (cudaStream_t)stream;
+    const int M = s->M, C = s->C, F = s->F;
+    typedef const __nv_bfloat16* cbf;
+    typedef __nv_bfloat16* bf;
+
+    build_row_maps<<<(M + 255) / 256, 256, 0, st>>>(keep_idx, cu_keep, kv_len, s->B, s->N, s->Lmax, M,
+                                                    ws.src_row, ws.kv_row, ctx->dev_status);
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+
+    nova_status rc;
+    // h = LN1(gathered rows)
+    rc = nova_launch_ln(ctx, (cbf)x_in, ws.src_row, (cbf)w->ln1_g, (cbf)w->ln1_b, w->eps, M, C, ws.h, st);
+    if (rc) return rc;
+    // [q | k | v] = h W_qkv^T + b; k, v go straight to their cache rows
+    nova_gemm_args g;
+    memset(&g, 0, sizeof(g));
+    g.A = ws.h; g.W = (cbf)w->w_qkv; g.bias = (cbf)w->b_qkv; g.M = M; g.N = 3 * C; g.K = C;
+    g.epilogue = NOVA_EPI_QKV; g.out = ws.q; g.C = C; g.k_cache = (bf)k_cache; g.v_cache = (bf)v_cache; g.kv_row = ws.kv_row;
+    rc = nova_launch_gemm(ctx, g, st);
+    if (rc) return rc;
+    // o = softmax(q K^T / sqrt(dh)) V
+    nova_attn_args a;
+    a.q = ws.q; a.k_cache = (cbf)k_cache; a.v_cache = (cbf)v_cache; a.cu_keep = cu_keep; a.kv_len = kv_len;
+    a.o = ws.o; a.B = s->B; a.C = C; a.n_heads = s->n_heads; a.Lmax = s->Lmax; a.M = M;
+    rc = nova_launch_attention(ctx, a, st);
+    if (rc) return rc;
+    // x1 = Xc + o W_o^T + b_o
+    memset(&g, 0, sizeof(g));
+    g.A = ws.o; g.W = (cbf)w->w_o; g.bias = (cbf)w->b_o; g.M = M; g.N = C; g.K = C;
+    g.epilogue = NOVA_EPI_BIAS_RES; g.out = ws.x1; g.res = (cbf)x_in; g.res_row = ws.src_row;
+    rc = nova_launch_gemm(ctx, g, st);
+    if (rc) return rc;
+    // h = LN2(x1)
+    rc = nova_launch_ln(ctx, ws.x1, nullptr, (cbf)w->ln2_g, (cbf)w->ln2_b, w->eps, M, C, ws.h, st);
+    if (rc) return rc;
+    // f = GELU(h W_fc1^T + b_fc1)
+    memset(&g, 0, sizeof(g));
+    g.A = ws.h; g.W = (cbf)w->w_fc1; g.bias = (cbf)w->b_fc1; g.M = M; g.N = F; g.K = C;
+    g.epilogue = NOVA_EPI_BIAS_GELU; g.out = ws.f;
+    rc = nova_launch_gemm(ctx, g, st);
+    if (rc) return rc;
+    // y = x1 + f W_fc2^T + b_fc2
+    memset(&g, 0, sizeof(g));
+    g.A = ws.f; g.W = (cbf)w->w_fc2; g.bias = (cbf)w->b_fc2; g.M = M; g.N = C; g.K = F;
+    g.epilogue = NOVA_EPI_BIAS_RES; g.out = (bf)y_kept; g.res = ws.x1; g.res_row = nullptr;
+    rc = nova_launch_gemm(ctx, g, st);
+    if (rc) return rc;
+    if (append_kv) {
+        advance_kv_len<<<(s->B + 127) / 128, 128, 0, st>>>(cu_keep, kv_len, s->B, s->Lmax);
+        NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    }
+    return NOVA_OK;
+}

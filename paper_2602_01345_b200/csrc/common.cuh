@@ -1,0 +1,92 @@
+// Shared host/device declarations of the NOVA CUDA library (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/nova.h"
+
+// Device status word: kernels OR these bits in; nova_device_status() maps them to a status.
+#define NOVA_DEV_NONFINITE 1u
+#define NOVA_DEV_TIMEOUT   2u
+#define NOVA_DEV_SHAPE     4u
+
+struct nova_ctx {
+    int device;
+    unsigned int* dev_status;   // one word of device memory
+    void* workspace;            // caller-owned device scratch
+    size_t workspace_bytes;
+    void* encode_tiled;         // cuTensorMapEncodeTiled, resolved through the runtime
+    int num_sms;
+    bool attr_select, attr_gemm, attr_attn;   // dynamic shared memory opt-in done on this device
+    char err[256];
+};
+
+static inline nova_status nova_fail(nova_ctx* ctx, nova_status s, const char* msg)
+{
+    if (ctx) {
+        strncpy(ctx->err, msg, sizeof(ctx->err) - 1);
+        ctx->err[sizeof(ctx->err) - 1] = 0;
+    }
+    return s;
+}
+
+static inline nova_status nova_cuda_fail(nova_ctx* ctx, cudaError_t e, const char* where)
+{
+    if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s: %s", where, cudaGetErrorString(e));
+    return NOVA_ERR_CUDA;
+}
+
+#define NOVA_CUDA_CHECK(ctx, expr)                                            \
+    do {                                                                      \
+        cudaError_t e__ = (expr);                                             \
+        if (e__ != cudaSuccess) return nova_cuda_fail((ctx), e__, #expr);     \
+    } while (0)
+
+static inline bool nova_aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
+
+// Kernel launchers implemented in the other translation units.
+nova_status nova_launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const int32_t* src_row,
+                           const __nv_bfloat16* g, const __nv_bfloat16* b, float eps, int M, int C,
+                           __nv_bfloat16* out, cudaStream_t st);
+
+enum nova_epilogue {
+    NOVA_EPI_QKV = 0,       // +bias; columns [0,C) -> q, [C,2C) -> k cache rows, [2C,3C) -> v cache rows
+    NOVA_EPI_BIAS_RES = 1,  // +bias + residual[res_row[r]] -> out
+    NOVA_EPI_BIAS_GELU = 2  // GELU_tanh(+bias) -> out
+};
+
+struct nova_gemm_args {
+    const __nv_bfloat16* A;     // [M, K] row-major
+    const __nv_bfloat16* W;     // [N, K] row-major
+    const __nv_bfloat16* bias;  // [N]
+    int M, N, K;
+    int epilogue;
+    __nv_bfloat16* out;         // [M, N] (QKV: q buffer [M, C])
+    // residual epilogue
+    const __nv_bfloat16* res;   // residual rows of width N
+    const int32_t* res_row;     // row map into res, or NULL for identity
+    // QKV epilogue
+    int C;
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    const int32_t* kv_row;      // [M] destination cache row (b*Lmax + kv_len[b] + m), -1 = skip
+};
+
+nova_status nova_launch_gemm(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st);
+
+struct nova_attn_args {
+    const __nv_bfloat16* q;        // [M, C]
+    const __nv_bfloat16* k_cache;  // [B, Lmax, C] already holding the new rows
+    const __nv_bfloat16* v_cache;
+    const int32_t* cu_keep;        // [B+1]
+    const int32_t* kv_len;         // [B] length before this call's rows
+    __nv_bfloat16* o;              // [M, C]
+    int B, C, n_heads, Lmax, M;
+};
+
+nova_status nova_launch_attention(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st);

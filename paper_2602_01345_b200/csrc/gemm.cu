@@ -1,0 +1,240 @@
+// out[M, N] = epilogue(A[M, K] * W[N, K]^T + bias) on the sm_100a tensor cores.
+//
+// Both operands are K-major bf16, so one TMA box of 64 K-elements (128 bytes, 128-byte
+// swizzle) per row feeds tcgen05.mma directly. One CTA computes one 128 x BN output tile:
+//   warp 0      TMA producer: fills a ring of kStages {A tile, W tile} buffers
+//   warp 1      allocates TMEM, issues tcgen05.mma (one elected thread), commits to mbarriers
+//   warps 2-5   epilogue: tcgen05.ld the fp32 accumulator (one row per thread), add bias,
+//               apply GELU / residual / QKV routing, store bf16
+// Every mbarrier wait is bounded; on expiry the CTA records a timeout and tears down.
+#include "tc_common.cuh"
+
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kThreads = 192;
+
+template <int BN, int STAGES>
+struct GemmSmem {
+    static constexpr int kABytes = BM * BK * 2;
+    static constexpr int kBBytes = BN * BK * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kTotal = STAGES * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+__device__ __forceinline__ float gelu_tanh(float x)
+{
+    const float c = 0.7978845608028654f;
+    const float inner = c * (x + 0.044715f * x * x * x);
+    // tanh(y) = 1 - 2 / (exp(2y) + 1); exp through ex2 keeps the error near 1e-6 relative
+    const float e = __expf(2.f * inner);
+    const float t = 1.f - __fdividef(2.f, e + 1.f);
+    return 0.5f * x * (1.f + t);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+
+struct GemmParams {
+    const __nv_bfloat16* bias;
+    int M, N, K;
+    int epilogue;
+    __nv_bfloat16* out;
+    const __nv_bfloat16* res;
+    const int32_t* res_row;
+    int C;
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    const int32_t* kv_row;
+    unsigned int* status;
+};
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(kThreads)
+gemm_bf16_tn(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+             const GemmParams p)
+{
+    using L = GemmSmem<BN, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* full_bar = (uint64_t*)(smem + STAGES * L::kStageBytes);
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* acc_bar = empty_bar + STAGES;
+    uint32_t* tmem_slot = (uint32_t*)(acc_bar + 1);
+    __shared__ int abort_flag_s;
+    volatile int* abort_flag = &abort_flag_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int num_kb = p.K / BK;
+
+    if (threadIdx.x == 0) {
+        abort_flag_s = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(acc_bar, 1);
+        fence_barrier_init();
+        prefetch_tmap(&tmap_a);
+        prefetch_tmap(&tmap_w);
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, BN);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES;
+                if (kb >= STAGES && !mbar_wait(&empty_bar[s], ((kb / STAGES) - 1) & 1, abort_flag, p.status)) break;
+                uint8_t* a_dst = smem + s * L::kStageBytes;
+                uint8_t* b_dst = a_dst + L::kABytes;
+                mbar_arrive_expect_tx(&full_bar[s], L::kStageBytes);
+                tma_load_2d(a_dst, &tmap_a, &full_bar[s], kb * BK, m0);
+                tma_load_2d(b_dst, &tmap_w, &full_bar[s], kb * BK, n0);
+                issued = kb + 1;
+            }
+            if (*abort_flag) {
+                // let the copies already issued land before the CTA's shared memory is released
+                for (int kb = max(0, issued - STAGES); kb < issued; ++kb)
+                    mbar_drain(&full_bar[kb % STAGES], (kb / STAGES) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(BM, BN, 0);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % STAGES;
+                ok = mbar_wait(&full_bar[s], (kb / STAGES) & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(smem + s * L::kStageBytes);
+                const uint32_t b_addr = a_addr + L::kABytes;
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; ++kk) {
+                    const uint64_t adesc = smem_desc_sw128(a_addr + kk * 32, 16, 1024);
+                    const uint64_t bdesc = smem_desc_sw128(b_addr + kk * 32, 16, 1024);
+                    mma_bf16_ss(tmem_acc, adesc, bdesc, idesc, (kb | kk) ? 1u : 0u);
+                }
+                mma_commit(&empty_bar[s]);   // frees the stage when these MMAs have read it
+            }
+            if (ok) mma_commit(acc_bar);     // accumulator complete
+        }
+    } else {
+        // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31
+        const int q = warp & 3;
+        const int row = m0 + q * 32 + lane;
+        if (mbar_wait_warp(acc_bar, 0, abort_flag, p.status)) {
+            tc_fence_after();
+            const bool row_ok = row < p.M;
+            long res_base = 0;
+            long kv_base = -1;
+            if (row_ok) {
+                if (p.epilogue == NOVA_EPI_BIAS_RES) res_base = (long)(p.res_row ? p.res_row[row] : row) * p.N;
+                if (p.epilogue == NOVA_EPI_QKV) kv_base = (long)p.kv_row[row];
+            }
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col0 = n0 + c * 32;
+                uint32_t acc[32];
+                tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), acc);
+                tmem_ld_wait();
+                if (!row_ok || col0 >= p.N) continue;
+                float v[32];
+                const uint4* bias4 = (const uint4*)(p.bias + col0);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 b = bias4[i];
+                    const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        v[i * 8 + j * 2] = __uint_as_float(acc[i * 8 + j * 2]) + __uint_as_float(bw[j] << 16);
+                        v[i * 8 + j * 2 + 1] = __uint_as_float(acc[i * 8 + j * 2 + 1]) + __uint_as_float(bw[j] & 0xffff0000u);
+                    }
+                }
+                __nv_bfloat16* dst;
+                if (p.epilogue == NOVA_EPI_BIAS_GELU) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = gelu_tanh(v[i]);
+                    dst = p.out + (long)row * p.N + col0;
+                } else if (p.epilogue == NOVA_EPI_BIAS_RES) {
+                    const uint4* r4 = (const uint4*)(p.res + res_base + col0);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint4 r = r4[i];
+                        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            v[i * 8 + j * 2] += __uint_as_float(rw[j] << 16);
+                            v[i * 8 + j * 2 + 1] += __uint_as_float(rw[j] & 0xffff0000u);
+                        }
+                    }
+                    dst = p.out + (long)row * p.N + col0;
+                } else {
+                    // QKV routing: this 32-column chunk lies entirely in q, k or v (C % 32 == 0)
+                    const int which = col0 / p.C, cc = col0 - which * p.C;
+                    if (which == 0) dst = p.out + (long)row * p.C + cc;
+                    else {
+                        if (kv_base < 0) continue;   // cache overflow: flagged when the row map was built
+                        dst = (which == 1 ? p.k_cache : p.v_cache) + kv_base * p.C + cc;
+                    }
+                }
+                uint4* d4 = (uint4*)dst;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    d4[i] = make_uint4(pack_bf16(v[i * 8], v[i * 8 + 1]), pack_bf16(v[i * 8 + 2], v[i * 8 + 3]),
+                                       pack_bf16(v[i * 8 + 4], v[i * 8 + 5]), pack_bf16(v[i * 8 + 6], v[i * 8 + 7]));
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_acc, BN);
+    }
+}
+
+template <int BN, int STAGES>
+nova_status launch(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
+{
+    using L = GemmSmem<BN, STAGES>;
+    CUtensorMap ta, tw;
+    const uint64_t da[2] = {(uint64_t)a.K, (uint64_t)a.M}, sa[1] = {(uint64_t)a.K * 2};
+    const uint64_t dw[2] = {(uint64_t)a.K, (uint64_t)a.N}, sw[1] = {(uint64_t)a.K * 2};
+    if (!make_tmap_bf16(ctx, &ta, a.A, 2, da, sa, BM) || !make_tmap_bf16(ctx, &tw, a.W, 2, dw, sw, BN))
+        return nova_fail(ctx, NOVA_ERR_CUDA, "gemm: cuTensorMapEncodeTiled failed");
+    auto kern = gemm_bf16_tn<BN, STAGES>;
+    if (!ctx->attr_gemm) {
+        NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+        ctx->attr_gemm = true;
+    }
+    GemmParams p;
+    p.bias = a.bias; p.M = a.M; p.N = a.N; p.K = a.K; p.epilogue = a.epilogue; p.out = a.out;
+    p.res = a.res; p.res_row = a.res_row; p.C = a.C; p.k_cache = a.k_cache; p.v_cache = a.v_cache;
+    p.kv_row = a.kv_row; p.status = ctx->dev_status;
+    dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM);
+    kern<<<grid, kThreads, L::kTotal, st>>>(ta, tw, p);
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    return NOVA_OK;
+}
+
+}  // namespace
+
+nova_status nova_launch_gemm(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
+{
+    if (a.M <= 0) return NOVA_OK;
+    if (a.K % BK || a.N % 32 || a.K < BK) return nova_fail(ctx, NOVA_ERR_SHAPE, "gemm: K must be a multiple of 64 and N of 32");
+    return launch<128, 3>(ctx, a, st);
+}

@@ -1,0 +1,400 @@
+"""GPU parity: every C-ABI call against the CPU oracle on the same seeded inputs.
+
+Index outputs, keep counts and cumulative offsets must match bit for bit (the oracle's
+selection is run on the entropies the GPU produced, so both decide in the same precision);
+entropies within 1e-3 absolute; block outputs within 2e-2 of the output's maximum magnitude
+(bf16 operands and bf16 storage between stages against the fp32/fp64 oracle); restored rows
+within one bf16 unit in the last place.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import nova_synth as synth
+import oracle
+import paper_2602_01345_b200 as nova
+
+pytestmark = pytest.mark.gpu
+
+ENT_TOL = 1e-3
+BLOCK_TOL = 2e-2
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = nova.Context(0)
+    yield c
+    assert c.device_status() == 0
+    c.close()
+
+
+def f32(t):
+    return synth.to_f32_numpy(t)
+
+
+def gpu_entropy(ctx, logits):
+    S, N, _ = logits.shape
+    ent = torch.empty((S, N), dtype=torch.float32, device=DEV)
+    mean = torch.empty((S,), dtype=torch.float32, device=DEV)
+    nova.nova_scale_entropy(ctx, logits, ent, mean)
+    return ent, mean
+
+
+def gpu_select(ctx, ent, k, with_pos=True):
+    S, N = ent.shape
+    k = torch.as_tensor(k, dtype=torch.int32)
+    M = int(k.sum())
+    keep_idx = torch.full((M,), -7, dtype=torch.int32, device=DEV)
+    prune_idx = torch.full((S * N - M,), -7, dtype=torch.int32, device=DEV)
+    cu = torch.full((S + 1,), -7, dtype=torch.int32, device=DEV)
+    pos = torch.full((S, N), -7, dtype=torch.int32, device=DEV) if with_pos else None
+    nova.nova_select_topk(ctx, ent, k, keep_idx, prune_idx, cu, pos)
+    return keep_idx, prune_idx, cu, pos
+
+
+# --------------------------------------------------------------------------- entropy
+@pytest.mark.parametrize("S,N,V,dtype", [
+    (3, 37, 4096, torch.bfloat16),      # several blocks of 8 rows and a ragged last block
+    (2, 16, 4096, torch.float32),
+    (1, 9, 1000, torch.bfloat16),       # V below one full register tile
+    (2, 5, 8192, torch.bfloat16),       # wider than the register path for bf16 -> streaming kernel
+    (1, 3, 24, torch.float32),
+])
+def test_entropy_matches_oracle(ctx, S, N, V, dtype):
+    a = synth.smooth_temperature_field(S, 1, N, seed=3, device=DEV)
+    logits = synth.logits_from_temperature(a, V, seed=11, dtype=dtype)
+    ent, mean = gpu_entropy(ctx, logits)
+    want_ent, want_mean = oracle.scale_entropy(f32(logits))
+    assert np.abs(ent.cpu().numpy() - want_ent).max() <= ENT_TOL
+    assert np.abs(mean.cpu().numpy() - want_mean).max() <= ENT_TOL
+    if V >= 1000 and N >= 9:
+        assert want_ent.max() - want_ent.min() > 2.0   # the field really spans low and high entropy
+
+
+def test_entropy_ragged_v_and_row_stride(ctx):
+    V, stride = 1003, 1008
+    buf = torch.zeros((2, 6, stride), dtype=torch.bfloat16, device=DEV)
+    buf[:, :, :V] = synth.randn_bf16((2, 6, V), 5, DEV, std=3.0)
+    buf[:, :, V:] = 50.0                                # padding must be ignored
+    logits = buf[:, :, :V]
+    ent = torch.empty((2, 6), dtype=torch.float32, device=DEV)
+    nova.nova_scale_entropy(ctx, logits, ent, None)
+    want, _ = oracle.scale_entropy(f32(logits))
+    assert np.abs(ent.cpu().numpy() - want).max() <= ENT_TOL
+
+
+def test_entropy_closed_forms_on_gpu(ctx):
+    V = 4096
+    z = torch.zeros((1, 4, V), dtype=torch.bfloat16, device=DEV)
+    z[0, 0] = 0.5                                       # uniform -> ln V
+    z[0, 1, 100] = 100.0                                # one hot -> 0
+    z[0, 2, :7] = 3.0                                   # two-level
+    z[0, 3, 2048:] = float("-inf")                      # -inf logits contribute nothing -> ln 2048
+    ent, _ = gpu_entropy(ctx, z)
+    e = ent.cpu().numpy()[0]
+    assert abs(e[0] - math.log(V)) <= ENT_TOL
+    assert e[1] == 0.0
+    Z = 7 * math.exp(3.0) + (V - 7)
+    assert abs(e[2] - (math.log(Z) - 7 * 3.0 * math.exp(3.0) / Z)) <= ENT_TOL
+    assert abs(e[3] - math.log(2048)) <= ENT_TOL
+    assert ctx.device_status() == 0
+
+
+def test_entropy_flags_nonfinite(ctx):
+    z = synth.randn_bf16((1, 8, 256), 1, DEV)
+    z[0, 3, 17] = float("nan")
+    z[0, 5, 9] = float("inf")
+    ent, _ = gpu_entropy(ctx, z)
+    e = ent.cpu().numpy()[0]
+    assert np.isnan(e[3]) and np.isnan(e[5]) and np.isfinite(np.delete(e, [3, 5])).all()
+    assert ctx.device_status() == 5                     # NOVA_ERR_NONFINITE, then cleared
+    assert ctx.device_status() == 0
+
+
+def test_entropy_empty_and_bad_args(ctx):
+    ent = torch.empty((0, 4), dtype=torch.float32, device=DEV)
+    nova.nova_scale_entropy(ctx, torch.empty((0, 4, 64), dtype=torch.bfloat16, device=DEV), ent, None)
+    base = torch.zeros(4 * 64 + 8, dtype=torch.bfloat16, device=DEV)
+    mis = base[1:1 + 4 * 64].view(1, 4, 64)             # 2-byte offset: not 16-byte aligned
+    with pytest.raises(nova.NovaError) as ei:
+        nova.nova_scale_entropy(ctx, mis, torch.empty((1, 4), dtype=torch.float32, device=DEV), None)
+    assert ei.value.status == 3
+
+
+# ---------------------------------------------------------------------------- select
+@pytest.mark.parametrize("S,N", [(1, 1), (3, 33), (2, 256), (5, 1000), (2, 4096), (2, 16384)])
+def test_select_bit_exact(ctx, S, N):
+    g = torch.Generator(device="cpu").manual_seed(S * 100003 + N)
+    ent = torch.rand((S, N), generator=g) * 8.0
+    if N > 1:
+        ent[:, ::5] = ent[:, 1:2]                      # many exact ties
+    if N > 8:
+        ent[0, 3] = -0.0
+        ent[0, 7] = 0.0
+    ks = [int(x) for x in torch.randint(0, N + 1, (S,), generator=g)]
+    ks[0] = N // 2 if N > 1 else 1
+    ent_d = ent.to(DEV)
+    keep_idx, prune_idx, cu, pos = gpu_select(ctx, ent_d, ks)
+    w_keep, w_prune, w_cu, w_pos = oracle.select_topk(ent.numpy(), ks)
+    assert np.array_equal(cu.cpu().numpy(), w_cu)
+    assert np.array_equal(keep_idx.cpu().numpy(), w_keep)
+    assert np.array_equal(prune_idx.cpu().numpy(), w_prune)
+    assert np.array_equal(pos.cpu().numpy(), w_pos)
+
+
+def test_select_edge_counts_and_many_segments(ctx):
+    N = 300
+    S = 300                                             # more segments than one launch carries
+    g = torch.Generator(device="cpu").manual_seed(9)
+    ent = torch.randn((S, N), generator=g)
+    ks = [0, N, 1, N - 1] + [int(x) for x in torch.randint(0, N + 1, (S - 4,), generator=g)]
+    keep_idx, prune_idx, cu, _ = gpu_select(ctx, ent.to(DEV), ks, with_pos=False)
+    w_keep, w_prune, w_cu, _ = oracle.select_topk(ent.numpy(), ks)
+    assert np.array_equal(cu.cpu().numpy(), w_cu)
+    assert np.array_equal(keep_idx.cpu().numpy(), w_keep)
+    assert np.array_equal(prune_idx.cpu().numpy(), w_prune)
+
+
+def test_select_teacher_forced_on_gpu_entropy(ctx):
+    # the selection is decided on the entropies the GPU computed; the oracle ranks those same values
+    B, h, w = 2, 16, 16
+    a = synth.smooth_temperature_field(B, h, w, seed=0, device=DEV)
+    logits = synth.logits_from_temperature(a, synth.V_CODEBOOK, seed=1)
+    ent, mean = gpu_entropy(ctx, logits)
+    r = nova.nova_keep_ratios(nova.SchedParams(force_act_scale=10, force_keep_ratio=0.5), 10, 1, h * w,
+                              mean.cpu().view(B, 1).expand(B, 10).contiguous())
+    assert r["keep"].tolist() == [128, 128]
+    keep_idx, prune_idx, cu, pos = gpu_select(ctx, ent, r["keep"])
+    w_keep, w_prune, w_cu, w_pos = oracle.select_topk(ent.cpu().numpy(), r["keep"].numpy())
+    assert np.array_equal(keep_idx.cpu().numpy(), w_keep)
+    assert np.array_equal(prune_idx.cpu().numpy(), w_prune)
+    assert np.array_equal(cu.cpu().numpy(), w_cu)
+    # and the kept tokens are the high-entropy half of the field
+    kept_mean = ent.cpu().numpy()[0][w_keep[:128]].mean()
+    assert kept_mean > ent.cpu().numpy()[0].mean()
+
+
+def test_select_bad_args(ctx):
+    ent = torch.zeros((1, 8), dtype=torch.float32, device=DEV)
+    out = torch.zeros(16, dtype=torch.int32, device=DEV)
+    with pytest.raises(nova.NovaError) as ei:
+        nova.nova_select_topk(ctx, ent, torch.tensor([9], dtype=torch.int32), out, out, out, None)
+    assert ei.value.status == 1
+    big = torch.zeros((1, 16385), dtype=torch.float32, device=DEV)
+    with pytest.raises(nova.NovaError) as ei:
+        nova.nova_select_topk(ctx, big, torch.tensor([5], dtype=torch.int32), out, out, out, None)
+    assert ei.value.status == 2
+
+
+# --------------------------------------------------------------------------- restore
+def _bf16_ulp_ok(got, want):
+    """|got - want| within one bf16 unit in the last place of the larger magnitude, plus the
+    fp32 evaluation error of a four-term weighted sum of O(1) values (about 8 * 2^-24 * 5),
+    which dominates only where the interpolated value cancels to nearly zero."""
+    mag = np.maximum(np.abs(got), np.abs(want))
+    return (np.abs(got - want) <= mag * 2.0 ** -7 + 4e-6).all()
+
+
+@pytest.mark.parametrize("B,hp,wp,h,w,C,keep_frac", [
+    (2, 13, 13, 16, 16, 1024, 0.5),     # config-1 restore
+    (3, 5, 7, 9, 11, 64, 0.3),          # ragged everything, rectangular
+    (1, 4, 4, 4, 4, 256, 0.0),          # nothing kept, same-size resize
+    (2, 3, 3, 8, 8, 128, 1.0),          # everything kept
+])
+def test_restore_matches_oracle(ctx, B, hp, wp, h, w, C, keep_frac):
+    N = h * w
+    x = synth.activations(B, N, C, seed=1, device=DEV)
+    cache = synth.residual_cache(B, hp, wp, C, seed=2, device=DEV)
+    g = torch.Generator(device="cpu").manual_seed(4)
+    ent = torch.rand((B, N), generator=g)
+    ks = [int(round(keep_frac * N))] * B
+    if 0 < keep_frac < 1 and B > 1:
+        ks[1] = max(1, ks[1] // 3)
+    keep_idx, prune_idx, cu, _ = gpu_select(ctx, ent.to(DEV), ks)
+    M = sum(ks)
+    y = synth.randn_bf16((M, C), 7, DEV)
+    x_out = torch.full_like(x, float("nan"))
+    cache_out = torch.full_like(x, float("nan"))
+    nova.nova_restore_from_cache(ctx, x, y, keep_idx, prune_idx, cu, cache, h, w, x_out, cache_out)
+    wx, wc = oracle.restore_from_cache(f32(x), f32(y), keep_idx.cpu().numpy(), prune_idx.cpu().numpy(),
+                                       cu.cpu().numpy(), f32(cache), h, w)
+    gx, gc = f32(x_out), f32(cache_out)
+    assert np.isfinite(gx).all() and np.isfinite(gc).all()       # every row was written
+    kk, cuu = keep_idx.cpu().numpy(), cu.cpu().numpy()
+    for b in range(B):
+        kept = kk[cuu[b]:cuu[b + 1]]
+        assert np.array_equal(gx[b, kept], f32(y)[cuu[b]:cuu[b + 1]])   # kept rows bit-equal y
+    assert _bf16_ulp_ok(gx, wx)
+    assert _bf16_ulp_ok(gc, wc)
+    # no cache output requested
+    x_out2 = torch.empty_like(x)
+    nova.nova_restore_from_cache(ctx, x, y, keep_idx, prune_idx, cu, cache, h, w, x_out2, None)
+    assert torch.equal(x_out2, x_out)
+
+
+# ----------------------------------------------------------------------------- block
+def _run_block(ctx, shape, weights, x, keep_idx, cu, k_cache, v_cache, kv_len, append=True):
+    ctx.ensure_workspace(shape)
+    y = torch.full((shape.M, shape.C), float("nan"), dtype=torch.bfloat16, device=DEV)
+    nova.nova_pruned_block_forward(ctx, weights, shape, x, keep_idx, cu, k_cache, v_cache, kv_len, append, y)
+    return y
+
+
+def _rel_err(got, want):
+    return float(np.abs(got - want).max() / np.abs(want).max())
+
+
+def _block_case(ctx, B, N, C, heads, F, Lmax, ks, kv_lens, seed, rows=None):
+    wt = synth.block_weights(C, F, seed, DEV)
+    x = synth.activations(B, N, C, seed + 1, DEV)
+    k_cache, v_cache, _ = synth.kv_cache(B, Lmax, max(kv_lens), C, seed + 2, DEV)
+    kv_len = torch.tensor(kv_lens, dtype=torch.int32, device=DEV)
+    # rows past each image's own length hold garbage the kernels must never use
+    for b, n in enumerate(kv_lens):
+        k_cache[b, n:] = float("nan")
+        v_cache[b, n:] = float("nan")
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    ent = torch.rand((B, N), generator=g)
+    keep_idx, prune_idx, cu, _ = gpu_select(ctx, ent.to(DEV), ks)
+    M = sum(ks)
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, M)
+    k0, v0 = k_cache.clone(), v_cache.clone()
+    y = _run_block(ctx, shape, nova.BlockWeights(wt, 1e-6), x, keep_idx, cu, k_cache, v_cache, kv_len)
+    assert ctx.device_status() == 0
+    wts = {n: f32(t) for n, t in wt.items()}
+    kc = np.nan_to_num(f32(k0))
+    vc = np.nan_to_num(f32(v0))
+    wy, wk, wv = oracle.pruned_block_forward(wts, 1e-6, heads, f32(x), keep_idx.cpu().numpy(), cu.cpu().numpy(),
+                                             kc, vc, np.array(kv_lens, np.int32), rows=rows)
+    gy = f32(y)
+    if rows is not None:
+        gy = gy[np.asarray(rows)]
+    assert np.isfinite(gy).all()
+    assert _rel_err(gy, wy) <= BLOCK_TOL
+    # appended cache rows and the advanced lengths
+    cuu = cu.cpu().numpy()
+    gk, gv = f32(k_cache), f32(v_cache)
+    for b in range(B):
+        n0, kb = kv_lens[b], ks[b]
+        if kb == 0:
+            continue
+        assert _rel_err(gk[b, n0:n0 + kb], wk[cuu[b]:cuu[b + 1]]) <= BLOCK_TOL
+        assert _rel_err(gv[b, n0:n0 + kb], wv[cuu[b]:cuu[b + 1]]) <= BLOCK_TOL
+        # rows before the append are untouched
+        assert torch.equal(k_cache[b, :n0], k0[b, :n0])
+    assert kv_len.cpu().tolist() == [a + b for a, b in zip(kv_lens, ks)]
+    return _rel_err(gy, wy)
+
+
+def test_block_config1_shape(ctx):
+    # width 1024, 16 heads x 64, MLP 4096, batch 2, 128 of 256 tokens kept, 424 prior tokens
+    _block_case(ctx, B=2, N=256, C=1024, heads=16, F=4096, Lmax=680, ks=[128, 128], kv_lens=[424, 424], seed=0)
+
+
+def test_block_ragged_small_dh64(ctx):
+    # kept counts that are not multiples of the 128-row tile, an empty image, ragged key tails
+    _block_case(ctx, B=4, N=200, C=128, heads=2, F=256, Lmax=512, ks=[200, 77, 0, 1],
+                kv_lens=[0, 130, 17, 300], seed=3)
+
+
+def test_block_dh128_several_key_tiles(ctx):
+    _block_case(ctx, B=2, N=300, C=256, heads=2, F=512, Lmax=1024, ks=[300, 129], kv_lens=[517, 5], seed=5)
+
+
+def test_block_keep_all_equals_dense(ctx):
+    # keep ratio 1: the compacted call is the dense block on every token
+    _block_case(ctx, B=1, N=256, C=128, heads=2, F=256, Lmax=512, ks=[256], kv_lens=[100], seed=7)
+
+
+def test_block_without_append_leaves_kv_len(ctx):
+    B, N, C, heads, F, Lmax = 1, 64, 128, 2, 256, 256
+    wt = synth.block_weights(C, F, 1, DEV)
+    x = synth.activations(B, N, C, 2, DEV)
+    k_cache, v_cache, kv_len = synth.kv_cache(B, Lmax, 10, C, 3, DEV)
+    keep_idx, _, cu, _ = gpu_select(ctx, torch.rand((B, N)).to(DEV), [32])
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, 32)
+    _run_block(ctx, shape, nova.BlockWeights(wt), x, keep_idx, cu, k_cache, v_cache, kv_len, append=False)
+    assert kv_len.cpu().tolist() == [10]
+    assert ctx.device_status() == 0
+
+
+def test_block_cache_overflow_is_reported_not_written(ctx):
+    B, N, C, heads, F, Lmax = 1, 64, 128, 2, 256, 40
+    wt = synth.block_weights(C, F, 1, DEV)
+    x = synth.activations(B, N, C, 2, DEV)
+    k_cache, v_cache, kv_len = synth.kv_cache(B, Lmax, 30, C, 3, DEV)
+    k0 = k_cache.clone()
+    keep_idx, _, cu, _ = gpu_select(ctx, torch.rand((B, N)).to(DEV), [32])   # 30 + 32 > 40
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, 32)
+    _run_block(ctx, shape, nova.BlockWeights(wt), x, keep_idx, cu, k_cache, v_cache, kv_len)
+    assert ctx.device_status() == 2                      # NOVA_ERR_SHAPE
+    assert torch.equal(k_cache, k0) and kv_len.cpu().tolist() == [30]
+
+
+def test_block_bad_args(ctx):
+    wt = synth.block_weights(128, 256, 1, DEV)
+    x = synth.activations(1, 8, 128, 2, DEV)
+    k_cache, v_cache, kv_len = synth.kv_cache(1, 16, 0, 128, 3, DEV)
+    idx = torch.arange(8, dtype=torch.int32, device=DEV)
+    cu = torch.tensor([0, 8], dtype=torch.int32, device=DEV)
+    y = torch.empty((8, 128), dtype=torch.bfloat16, device=DEV)
+    w = nova.BlockWeights(wt)
+    with pytest.raises(nova.NovaError) as ei:            # head dim 32 unsupported
+        nova.nova_pruned_block_forward(ctx, w, nova.BlockShape(1, 8, 128, 4, 256, 16, 8), x, idx, cu,
+                                       k_cache, v_cache, kv_len, True, y)
+    assert ei.value.status == 2
+    ctx.set_workspace(torch.empty(256, dtype=torch.uint8, device=DEV))
+    with pytest.raises(nova.NovaError) as ei:            # workspace too small
+        nova.nova_pruned_block_forward(ctx, w, nova.BlockShape(1, 8, 128, 2, 256, 16, 8), x, idx, cu,
+                                       k_cache, v_cache, kv_len, True, y)
+    assert ei.value.status == 4
+
+
+# ------------------------------------------------------------------------ whole step
+def test_whole_pruned_step_config1(ctx):
+    """entropy -> keep ratios -> top-k -> block on kept rows -> restore, config-1 shapes, each
+    stage checked against the oracle fed with the GPU's inputs to that stage."""
+    B, h, w, C, heads, F, P = 2, 16, 16, 1024, 16, 4096, 424
+    N, Lmax = h * w, 680
+    a = synth.smooth_temperature_field(B, h, w, seed=0, device=DEV)
+    logits = synth.logits_from_temperature(a, synth.V_CODEBOOK, seed=1)
+    wt = synth.block_weights(C, F, 0, DEV)
+    x = synth.activations(B, N, C, 1, DEV)
+    k_cache, v_cache, kv_len = synth.kv_cache(B, Lmax, P, C, 2, DEV)
+    cache_prev = synth.residual_cache(B, 13, 13, C, 3, DEV)
+    k0, v0 = k_cache.clone(), v_cache.clone()
+
+    ent, mean = gpu_entropy(ctx, logits)
+    w_ent, w_mean = oracle.scale_entropy(f32(logits))
+    assert np.abs(ent.cpu().numpy() - w_ent).max() <= ENT_TOL
+
+    hbar = mean.cpu().view(B, 1).expand(B, 10).contiguous()
+    sp = dict(force_act_scale=10, force_keep_ratio=0.5)
+    r = nova.nova_keep_ratios(nova.SchedParams(**sp), 10, 1, N, hbar)
+    wr = oracle.keep_ratios(oracle.SchedParams(**sp), 10, 1, N, hbar.numpy())
+    assert np.array_equal(r["keep"].numpy(), wr["keep"]) and np.array_equal(r["act_scale"].numpy(), wr["act_scale"])
+
+    keep_idx, prune_idx, cu, _ = gpu_select(ctx, ent, r["keep"])
+    w_keep, w_prune, w_cu, _ = oracle.select_topk(ent.cpu().numpy(), wr["keep"])
+    assert np.array_equal(keep_idx.cpu().numpy(), w_keep) and np.array_equal(prune_idx.cpu().numpy(), w_prune)
+    assert np.array_equal(cu.cpu().numpy(), w_cu)
+
+    M = int(r["keep"].sum())
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, M)
+    y = _run_block(ctx, shape, nova.BlockWeights(wt, 1e-6), x, keep_idx, cu, k_cache, v_cache, kv_len)
+    wy, _, _ = oracle.pruned_block_forward({n: f32(t) for n, t in wt.items()}, 1e-6, heads, f32(x), w_keep, w_cu,
+                                           f32(k0), f32(v0), np.full(B, P, np.int32))
+    assert _rel_err(f32(y), wy) <= BLOCK_TOL
+
+    x_out = torch.empty_like(x)
+    cache_out = torch.empty_like(x)
+    nova.nova_restore_from_cache(ctx, x, y, keep_idx, prune_idx, cu, cache_prev, h, w, x_out, cache_out)
+    wx, wc = oracle.restore_from_cache(f32(x), f32(y), w_keep, w_prune, w_cu, f32(cache_prev), h, w)
+    assert _bf16_ulp_ok(f32(x_out), wx) and _bf16_ulp_ok(f32(cache_out), wc)
+    # free-running end to end (oracle block output instead of the GPU's): still within the block tolerance
+    fx, _ = oracle.restore_from_cache(f32(x), wy, w_keep, w_prune, w_cu, f32(cache_prev), h, w)
+    assert _rel_err(f32(x_out), fx) <= BLOCK_TOL
+    assert ctx.device_status() == 0
