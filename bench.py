@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the NOVA pruned-scale step on B200.
+
+A step is one pass of the whole hot path over one accelerated scale: for each of the L layers,
+entropy of that layer's logits -> keep counts (host) -> top-k -> block on the kept tokens ->
+restore from the residual cache. The default workload is the 1024x1024 large-model shape
+(32 layers, width 2048, 16 heads x 128, MLP 8192, last scale 64x64 = 4096 tokens attending to
+6425 prior tokens, batch 4, keep ratio 0.5). Prints one JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import nova_synth as synth  # noqa: E402
+
+METRIC = "pruned_scale_images_per_s"
+UNIT = "images/s"
+# DRAM bytes per attention launch from the committed ncu capture (profiles/), or None.
+ATTENTION_TRAFFIC_BYTES = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4_1024", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--keep", type=float, default=0.5)
+    ap.add_argument("--scale", type=int, default=None, help="1-based scale index (default: last)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def workload_desc(args):
+    ms = synth.CONFIGS[args.workload]
+    t = args.scale or len(ms.scales)
+    B = args.batch or ms.B
+    side = ms.scales[t - 1]
+    prev = ms.scales[t - 2] if t >= 2 else side
+    return dict(ms=ms, t=t, B=B, h=side, w=side, hp=prev, wp=prev, N=side * side,
+                P=ms.prior_tokens(t), Lmax=ms.total_tokens, keep=args.keep)
+
+
+def config_json(wd, n_gpus):
+    ms = wd["ms"]
+    return {
+        "workload": f"{ms.name}: scale {wd['t']} ({wd['h']}x{wd['w']} = {wd['N']} tokens, {wd['P']} prior tokens), "
+                    f"{ms.L} layers, width {ms.C}, {ms.heads} heads x {ms.dh}, MLP {ms.F}, V={synth.V_CODEBOOK}, "
+                    f"batch {wd['B']} per GPU, keep ratio {wd['keep']}",
+        "batch_per_gpu": wd["B"], "layers": ms.L, "tokens": wd["N"], "prior_tokens": wd["P"],
+        "keep_ratio": wd["keep"], "l2": "inputs_larger_than_l2", "parallelism": f"replicas x{n_gpus}",
+    }
+
+
+# ------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.proc = None
+        try:
+            self.fh = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-i", str(device_index), "-lms", "100"], stdout=self.fh,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.fh.close()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------ state
+def build_state(wd, device, seed=0):
+    """Random-init weights, prior K/V caches, previous residual caches and per-layer logits."""
+    ms, B, N = wd["ms"], wd["B"], wd["N"]
+    weights = [synth.block_weights(ms.C, ms.F, seed * 100 + j, device) for j in range(ms.L)]
+    k_caches, v_caches = [], []
+    for j in range(ms.L):
+        k, v, _ = synth.kv_cache(B, wd["Lmax"], wd["P"], ms.C, seed * 1000 + 2 * j, device)
+        k_caches.append(k)
+        v_caches.append(v)
+    kv_len0 = torch.full((ms.L, B), wd["P"], dtype=torch.int32, device=device)
+    cache_prev = [synth.residual_cache(B, wd["hp"], wd["wp"], ms.C, seed * 10 + j, device) for j in range(ms.L)]
+    a = synth.smooth_temperature_field(B, wd["h"], wd["w"], seed, a_lo=0.5, a_hi=6.0, device=device)
+    beta = synth.layer_inverse_temperatures(ms.L, seed)
+    logits = [synth.logits_from_temperature(a * float(beta[j]), synth.V_CODEBOOK, seed * 7 + j) for j in range(ms.L)]
+    x_in = synth.activations(B, N, ms.C, seed + 5, device)
+    return dict(weights=weights, k_caches=k_caches, v_caches=v_caches, kv_len0=kv_len0,
+                kv_len=kv_len0.clone(), cache_prev=cache_prev, logits=logits, x_in=x_in)
+
+
+def attention_flops(keeps, P, C):
+    """4 * sum_b k_b * (P + k_b) * C for one layer (QK^T and PV, 2 flops per multiply-add)."""
+    return sum(4.0 * int(k) * (P + int(k)) * C for k in keeps.tolist())
+
+
+def peaks():
+    try:
+        p = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        return dict(hbm=float(p["hbm_gbs"]), tensor=float(p["bf16_tflops_sustained"]), source="measured")
+    except Exception:
+        return dict(hbm=6650.0, tensor=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------ ours
+def run_ours(args):
+    import paper_2602_01345_b200 as nova
+    from paper_2602_01345_b200 import pipeline
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    wd = workload_desc(args)
+    ms, B, N = wd["ms"], wd["B"], wd["N"]
+
+    ctx = nova.Context(local)
+    st = build_state(wd, dev)
+    runner = pipeline.PrunedScaleRunner(ctx, st["weights"], ms.heads, B, wd["h"], wd["w"], wd["Lmax"],
+                                        st["k_caches"], st["v_caches"], st["kv_len"], st["cache_prev"])
+    sched = nova.SchedParams(force_act_scale=wd["t"], force_keep_ratio=wd["keep"])
+    hbar_scale = torch.linspace(2.0, 7.0, wd["t"]).repeat(B, 1).contiguous()
+    stream = torch.cuda.current_stream()
+
+    def one_step():
+        st["kv_len"].copy_(st["kv_len0"])          # every step starts from the same cache state
+        return runner.run_scale(st["x_in"], st["logits"], sched, wd["t"], hbar_scale, stream=stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+    assert ctx.device_status() == 0, "device status after warm-up"
+
+    clocks = ClockSampler(local)
+    launches0 = pipeline.launch_count(ctx)
+    pipeline.profile_begin(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        x_out, keeps = one_step()
+    e1.record(stream)
+    barrier()
+    total_ms = e0.elapsed_time(e1)
+    prof = pipeline.profile_end(ctx)
+    launches = pipeline.launch_count(ctx) - launches0
+    clk = clocks.stop()
+    if dist is not None:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * B / (ms_per_step / 1e3)
+    assert ctx.device_status() == 0, "device status after the timed region"
+
+    # ---- roofline of the dominant kernel (attention), from the events recorded in the timed region
+    pk = peaks()
+    attn_ms, attn_n = prof["attention"]
+    flops_per_launch = attention_flops(keeps[0], wd["P"], ms.C)
+    achieved = flops_per_launch / (attn_ms / attn_n * 1e-3) / 1e12 if attn_n else 0.0
+    roofline = {"kernel": "attention", "bound": "tensor", "achieved": round(achieved, 2), "peak": pk["tensor"],
+                "unit": "TFLOP/s", "frac": round(achieved / pk["tensor"], 4), "traffic": ATTENTION_TRAFFIC_BYTES,
+                "peak_source": pk["source"] + " (bf16 sustained)"}
+    kernels = {k: {"ms_per_step": round(v[0] / args.steps, 4), "launches_per_step": v[1] / args.steps}
+               for k, v in prof.items() if v[1]}
+    M = int(keeps[0].sum())
+    gemm_flops = {"gemm_qkv": 2.0 * M * 3 * ms.C * ms.C, "gemm_proj": 2.0 * M * ms.C * ms.C,
+                  "gemm_fc1": 2.0 * M * ms.F * ms.C, "gemm_fc2": 2.0 * M * ms.F * ms.C}
+    for k, fl in gemm_flops.items():
+        if k in kernels and prof[k][1]:
+            kernels[k]["tflops"] = round(fl / (prof[k][0] / prof[k][1] * 1e-3) / 1e12, 1)
+    rows = B * N
+    ent_bytes = rows * (synth.V_CODEBOOK * 2 + 4)
+    if prof["entropy_rows"][1]:
+        kernels["entropy_rows"]["gbs"] = round(ent_bytes / (prof["entropy_rows"][0] / prof["entropy_rows"][1] * 1e-3) / 1e9, 1)
+    restore_bytes = (M * 4 + (rows - M) * 3) * ms.C * 2 + B * wd["hp"] * wd["wp"] * ms.C * 2
+    if prof["restore"][1]:
+        kernels["restore"]["gbs"] = round(restore_bytes / (prof["restore"][0] / prof["restore"][1] * 1e-3) / 1e9, 1)
+
+    out = {
+        "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": config_json(wd, world), "clocks": clk, "gpu_launches": int(launches),
+        "tokens_per_s": round(world * B * N / (ms_per_step / 1e3), 1),
+        "roofline": roofline, "kernels": kernels,
+    }
+
+    # ---- end to end: inputs start in pinned host memory, result read back every step
+    if not args.no_e2e:
+        out["e2e"] = run_e2e(args, wd, st, runner, sched, hbar_scale, barrier, dist, dev, world)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(wd, st, keeps)
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, wd, st, runner, sched, hbar_scale, barrier, dist, dev, world):
+    ms, B, N = wd["ms"], wd["B"], wd["N"]
+    L = ms.L
+    host_x = st["x_in"].cpu().pin_memory()
+    host_logits = [t.cpu().pin_memory() for t in st["logits"]]
+    host_out = torch.empty_like(host_x).pin_memory()
+    dev_x = torch.empty_like(st["x_in"])
+    dev_logits = [torch.empty_like(t) for t in st["logits"]]
+    copy_stream = torch.cuda.Stream()
+    main = torch.cuda.current_stream()
+    h2d = host_x.numel() * 2 + sum(t.numel() * 2 for t in host_logits)
+    d2h = host_out.numel() * 2
+
+    def e2e_step():
+        st["kv_len"].copy_(st["kv_len0"])
+        copy_stream.wait_stream(main)               # the previous step no longer reads the device buffers
+        ready = []
+        with torch.cuda.stream(copy_stream):
+            dev_x.copy_(host_x, non_blocking=True)
+            x_ready = torch.cuda.Event()
+            x_ready.record(copy_stream)
+            for j in range(L):
+                dev_logits[j].copy_(host_logits[j], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(copy_stream)
+                ready.append(ev)
+        main.wait_event(x_ready)
+        x_out, _ = runner.run_scale(dev_x, dev_logits, sched, wd["t"], hbar_scale, stream=main, logits_ready=ready)
+        host_out.copy_(x_out, non_blocking=True)
+        main.synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(main)
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record(main)
+    barrier()
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    dev_ms = e0.elapsed_time(e1)
+    t_ms = max(wall_ms, dev_ms)
+    if dist is not None:
+        tt = torch.tensor([t_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_ms = float(tt.item())
+    per = t_ms / args.steps
+    return {"value": round(world * B / (per / 1e3), 3), "unit": UNIT, "ms_per_step": round(per, 3),
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "note": "pinned host x_in and per-layer logits uploaded on a copy stream overlapped with compute; x_out read back"}
+
+
+# ---------------------------------------------------------------------- CPU baseline (oracle)
+def oracle_sample(wd, st, keeps, rows_entropy=1024, rows_block=8):
+    """Times the oracle, as it stands, on one layer of one image and extrapolates to the whole
+    pruned scale: entropy on a row sample, selection on the full map, K/V of every kept token
+    (exact), attention + MLP on a row sample, restore on the full map."""
+    import numpy as np
+
+    import oracle
+    ms, N = wd["ms"], wd["N"]
+    f32 = synth.to_f32_numpy
+    t = {}
+    logits = f32(st["logits"][0][0:1, :rows_entropy])
+    t0 = time.perf_counter()
+    oracle.scale_entropy(logits)
+    t["entropy"] = (time.perf_counter() - t0) * (N / rows_entropy)
+    ent_full = np.random.default_rng(0).random((1, N)).astype(np.float32)
+    k = int(keeps[0][0])
+    t0 = time.perf_counter()
+    keep_idx, prune_idx, cu, _ = oracle.select_topk(ent_full, [k])
+    t["select"] = time.perf_counter() - t0
+    wts = {n: f32(v) for n, v in st["weights"][0].items()}
+    x = f32(st["x_in"][0:1])
+    kc, vc = f32(st["k_caches"][0][0:1]), f32(st["v_caches"][0][0:1])
+    kv_len = np.array([wd["P"]], np.int32)
+    t0 = time.perf_counter()
+    oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=np.zeros(0, np.int32))
+    t["block_kv"] = time.perf_counter() - t0
+    rows = np.linspace(0, k - 1, rows_block).astype(np.int32)
+    t0 = time.perf_counter()
+    y, _, _ = oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=rows)
+    t["block_rows"] = max(time.perf_counter() - t0 - t["block_kv"], 0.0) * (k / rows_block)
+    y_full = np.zeros((k, ms.C), np.float32)
+    t0 = time.perf_counter()
+    oracle.restore_from_cache(x, y_full, keep_idx, prune_idx, cu, f32(st["cache_prev"][0][0:1]), wd["h"], wd["w"])
+    t["restore"] = time.perf_counter() - t0
+    per_image_layer = sum(t.values())
+    return per_image_layer, t, oracle.num_threads()
+
+
+def cpu_baseline(wd, st, keeps):
+    per_image_layer, parts, cores = oracle_sample(wd, st, keeps)
+    ms = wd["ms"]
+    sec_per_image = per_image_layer * ms.L
+    return {"value": round(1.0 / sec_per_image, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "one layer of one image: entropy on 1024 of the rows, top-k on the full map, K/V of all kept "
+                      "tokens, attention+MLP on 8 kept rows, restore on the full map; each part scaled to the full "
+                      f"row count, then x{ms.L} layers",
+            "seconds_per_image_layer": {k: round(v, 3) for k, v in parts.items()}}
+
+
+def run_reference(args):
+    """The oracle as the reference arm: same metric and workload, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wd = workload_desc(args)
+    ms = wd["ms"]
+    wd_small = dict(wd, B=1)
+    st = build_state_cpu_one_layer(wd_small)
+    k = wd["N"] - int((1.0 - wd["keep"]) * wd["N"])
+    keeps = [torch.tensor([k], dtype=torch.int32)]
+    times = []
+    cores = 1
+    for i in range(args.warmup + args.steps):
+        per_image_layer, _, cores = oracle_sample(wd_small, st, keeps, rows_entropy=256, rows_block=2)
+        if i >= args.warmup:
+            times.append(per_image_layer * ms.L)
+    sec_per_image = sum(times) / len(times)
+    value = 1.0 / sec_per_image
+    sample = ("per step: one layer of one image (entropy on 256 rows, full top-k, K/V of all kept tokens, "
+              f"attention+MLP on 2 kept rows, full restore), parts scaled to full row counts, x{ms.L} layers")
+    out = {"impl": "reference", "metric": METRIC, "value": round(value, 6), "unit": UNIT,
+           "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": round(sec_per_image * wd["B"] * 1e3, 1), "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config_json(wd, 1),
+           "cpu_baseline": {"value": round(value, 6), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+           "e2e": {"value": round(value, 6), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def build_state_cpu_one_layer(wd):
+    """Layer-0 inputs of the workload for one image, generated on the CPU."""
+    ms, N = wd["ms"], wd["N"]
+    a = synth.smooth_temperature_field(1, wd["h"], wd["w"], 0)
+    k, v, _ = synth.kv_cache(1, wd["Lmax"], wd["P"], ms.C, 0, "cpu")
+    return dict(weights=[synth.block_weights(ms.C, ms.F, 0, "cpu")], k_caches=[k], v_caches=[v],
+                cache_prev=[synth.residual_cache(1, wd["hp"], wd["wp"], ms.C, 0, "cpu")],
+                logits=[synth.logits_from_temperature(a[:, :256].contiguous(), synth.V_CODEBOOK, 0)],
+                x_in=synth.activations(1, N, ms.C, 5, "cpu"))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

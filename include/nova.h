@@ -67,6 +67,18 @@ const char* nova_status_string(nova_status s);
  * NOVA_ERR_NONFINITE) and clears it. */
 nova_status nova_device_status(nova_ctx* ctx, void* stream);
 
+/* ---- measurement (no counterpart in the paper) --------------------------------- */
+/* Kernels launched by this context since nova_create. */
+unsigned long long nova_launch_count(const nova_ctx* ctx);
+/* Per-kernel timing: between nova_profile_begin and nova_profile_end every kernel launch is
+ * bracketed by CUDA events on its stream. nova_profile_end waits for them and fills
+ * ms[c] / launches[c] (host arrays of n >= nova_profile_categories() entries) with the summed
+ * device time and the launch count of category c; nova_profile_category_name(c) names it. */
+int         nova_profile_categories(void);
+const char* nova_profile_category_name(int cat);
+nova_status nova_profile_begin(nova_ctx* ctx);
+nova_status nova_profile_end(nova_ctx* ctx, double* ms, long long* launches, int n);
+
 /* ---- Eq. 4 and Eq. 7: entropy ------------------------------------------------- */
 /*
  * logits: device, [S, N, V], dtype dt, row r = s*N + i starts at element r*row_stride

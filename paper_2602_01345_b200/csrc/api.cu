@@ -30,8 +30,17 @@ nova_status nova_create(nova_ctx** out, int device)
     if (e != cudaSuccess || device < 0 || device >= count) return NOVA_ERR_CUDA;
     nova_ctx* ctx = new (std::nothrow) nova_ctx();
     if (!ctx) return NOVA_ERR_INVALID_ARG;
-    memset(ctx, 0, sizeof(*ctx));
     ctx->device = device;
+    ctx->dev_status = nullptr;
+    ctx->workspace = nullptr;
+    ctx->workspace_bytes = 0;
+    ctx->encode_tiled = nullptr;
+    ctx->num_sms = 0;
+    ctx->attr_select = ctx->attr_gemm = ctx->attr_attn = false;
+    ctx->err[0] = 0;
+    ctx->launches = 0;
+    ctx->profiling = false;
+    ctx->events_used = 0;
     if (cudaSetDevice(device) != cudaSuccess ||
         cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
         cudaMemset(ctx->dev_status, 0, 256) != cudaSuccess) {
@@ -56,8 +65,47 @@ void nova_destroy(nova_ctx* ctx)
 {
     if (!ctx) return;
     cudaSetDevice(ctx->device);
+    for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
     cudaFree(ctx->dev_status);
     delete ctx;
+}
+
+unsigned long long nova_launch_count(const nova_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int nova_profile_categories(void) { return NOVA_K_COUNT; }
+
+const char* nova_profile_category_name(int cat)
+{
+    static const char* names[NOVA_K_COUNT] = {
+        "entropy_rows", "entropy_mean", "select_topk", "build_row_maps", "layernorm", "gemm_qkv",
+        "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "advance_kv_len", "restore"};
+    return (cat >= 0 && cat < NOVA_K_COUNT) ? names[cat] : "?";
+}
+
+nova_status nova_profile_begin(nova_ctx* ctx)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    ctx->prof_recs.clear();
+    ctx->events_used = 0;
+    ctx->profiling = true;
+    return NOVA_OK;
+}
+
+nova_status nova_profile_end(nova_ctx* ctx, double* ms, long long* launches, int n)
+{
+    if (!ctx || !ms || !launches || n < NOVA_K_COUNT) return NOVA_ERR_INVALID_ARG;
+    ctx->profiling = false;
+    for (int i = 0; i < n; ++i) { ms[i] = 0.0; launches[i] = 0; }
+    for (const nova_prof_rec& r : ctx->prof_recs) {
+        NOVA_CUDA_CHECK(ctx, cudaEventSynchronize(r.stop));
+        float t = 0.f;
+        NOVA_CUDA_CHECK(ctx, cudaEventElapsedTime(&t, r.start, r.stop));
+        ms[r.cat] += (double)t;
+        launches[r.cat] += 1;
+    }
+    ctx->prof_recs.clear();
+    ctx->events_used = 0;
+    return NOVA_OK;
 }
 
 const char* nova_last_error(const nova_ctx* ctx) { return ctx ? ctx->err : "null context"; }

@@ -313,13 +313,20 @@ nova_status launch(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st)
         !make_tmap_bf16(ctx, &tv, a.v_cache, 3, dk, sk, BKV))
         return nova_fail(ctx, NOVA_ERR_CUDA, "attention: cuTensorMapEncodeTiled failed");
     auto kern = attention_kernel<DH>;
-    NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+    if (!ctx->attr_attn) {   // both head sizes opt in once per context
+        NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::kTotal));
+        NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::kTotal));
+        ctx->attr_attn = true;
+    }
     AttnParams p;
     p.cu_keep = a.cu_keep; p.kv_len = a.kv_len; p.o = a.o; p.B = a.B; p.C = a.C; p.Lmax = a.Lmax;
     p.scale_log2e = (float)((1.0 / sqrt((double)DH)) * 1.4426950408889634);
     p.status = ctx->dev_status;
     dim3 grid((a.M + BQ - 1) / BQ + a.B, a.n_heads);
-    kern<<<grid, kThreads, L::kTotal, st>>>(tq, tk, tv, p);
+    {
+        nova_launch_scope scope(ctx, NOVA_K_ATTENTION, st);
+        kern<<<grid, kThreads, L::kTotal, st>>>(tq, tk, tv, p);
+    }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }

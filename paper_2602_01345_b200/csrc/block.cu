@@ -156,6 +156,7 @@ nova_status nova_launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const int32_t*
     const int vec = C / 8;
     const int per_lane = (vec + 31) / 32;
     const dim3 grid((M + kLnWarps - 1) / kLnWarps), block(kLnWarps * 32);
+    nova_launch_scope scope(ctx, NOVA_K_LAYERNORM, st);
 #define NOVA_LN_CASE(V) layernorm_rows<V><<<grid, block, 0, st>>>((const uint4*)x, src_row, (const uint4*)g, (const uint4*)b, eps, M, vec, (uint4*)out)
     if (per_lane <= 2) NOVA_LN_CASE(2);
     else if (per_lane <= 4) NOVA_LN_CASE(4);
@@ -203,8 +204,11 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     typedef const __nv_bfloat16* cbf;
     typedef __nv_bfloat16* bf;
 
-    build_row_maps<<<(M + 255) / 256, 256, 0, st>>>(keep_idx, cu_keep, kv_len, s->B, s->N, s->Lmax, M,
-                                                    ws.src_row, ws.kv_row, ctx->dev_status);
+    {
+        nova_launch_scope scope(ctx, NOVA_K_ROW_MAPS, st);
+        build_row_maps<<<(M + 255) / 256, 256, 0, st>>>(keep_idx, cu_keep, kv_len, s->B, s->N, s->Lmax, M,
+                                                        ws.src_row, ws.kv_row, ctx->dev_status);
+    }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
 
     nova_status rc;
@@ -215,7 +219,7 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     nova_gemm_args g;
     memset(&g, 0, sizeof(g));
     g.A = ws.h; g.W = (cbf)w->w_qkv; g.bias = (cbf)w->b_qkv; g.M = M; g.N = 3 * C; g.K = C;
-    g.epilogue = NOVA_EPI_QKV; g.out = ws.q; g.C = C; g.k_cache = (bf)k_cache; g.v_cache = (bf)v_cache; g.kv_row = ws.kv_row;
+    g.epilogue = NOVA_EPI_QKV; g.cat = NOVA_K_GEMM_QKV; g.out = ws.q; g.C = C; g.k_cache = (bf)k_cache; g.v_cache = (bf)v_cache; g.kv_row = ws.kv_row;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     // o = softmax(q K^T / sqrt(dh)) V
@@ -227,7 +231,7 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     // x1 = Xc + o W_o^T + b_o
     memset(&g, 0, sizeof(g));
     g.A = ws.o; g.W = (cbf)w->w_o; g.bias = (cbf)w->b_o; g.M = M; g.N = C; g.K = C;
-    g.epilogue = NOVA_EPI_BIAS_RES; g.out = ws.x1; g.res = (cbf)x_in; g.res_row = ws.src_row;
+    g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_PROJ; g.out = ws.x1; g.res = (cbf)x_in; g.res_row = ws.src_row;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     // h = LN2(x1)
@@ -236,16 +240,17 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     // f = GELU(h W_fc1^T + b_fc1)
     memset(&g, 0, sizeof(g));
     g.A = ws.h; g.W = (cbf)w->w_fc1; g.bias = (cbf)w->b_fc1; g.M = M; g.N = F; g.K = C;
-    g.epilogue = NOVA_EPI_BIAS_GELU; g.out = ws.f;
+    g.epilogue = NOVA_EPI_BIAS_GELU; g.cat = NOVA_K_GEMM_FC1; g.out = ws.f;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     // y = x1 + f W_fc2^T + b_fc2
     memset(&g, 0, sizeof(g));
     g.A = ws.f; g.W = (cbf)w->w_fc2; g.bias = (cbf)w->b_fc2; g.M = M; g.N = C; g.K = F;
-    g.epilogue = NOVA_EPI_BIAS_RES; g.out = (bf)y_kept; g.res = ws.x1; g.res_row = nullptr;
+    g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_FC2; g.out = (bf)y_kept; g.res = ws.x1; g.res_row = nullptr;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     if (append_kv) {
+        nova_launch_scope scope(ctx, NOVA_K_KV_ADVANCE, st);
         advance_kv_len<<<(s->B + 127) / 128, 128, 0, st>>>(cu_keep, kv_len, s->B, s->Lmax);
         NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     }

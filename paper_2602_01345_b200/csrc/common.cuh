@@ -7,6 +7,7 @@
 #include <stdint.h>
 #include <stdio.h>
 #include <string.h>
+#include <vector>
 
 #include "../../include/nova.h"
 
@@ -14,6 +15,18 @@
 #define NOVA_DEV_NONFINITE 1u
 #define NOVA_DEV_TIMEOUT   2u
 #define NOVA_DEV_SHAPE     4u
+
+// Kernel categories for the launch counter and the optional per-kernel event timing.
+enum nova_kernel_cat {
+    NOVA_K_ENTROPY = 0, NOVA_K_ENTROPY_MEAN, NOVA_K_SELECT, NOVA_K_ROW_MAPS, NOVA_K_LAYERNORM,
+    NOVA_K_GEMM_QKV, NOVA_K_ATTENTION, NOVA_K_GEMM_PROJ, NOVA_K_GEMM_FC1, NOVA_K_GEMM_FC2,
+    NOVA_K_KV_ADVANCE, NOVA_K_RESTORE, NOVA_K_COUNT
+};
+
+struct nova_prof_rec {
+    int cat;
+    cudaEvent_t start, stop;
+};
 
 struct nova_ctx {
     int device;
@@ -24,6 +37,41 @@ struct nova_ctx {
     int num_sms;
     bool attr_select, attr_gemm, attr_attn;   // dynamic shared memory opt-in done on this device
     char err[256];
+    // measurement: launches since creation, and event pairs around each launch while profiling
+    unsigned long long launches;
+    bool profiling;
+    std::vector<nova_prof_rec> prof_recs;     // records of the current profiling window
+    std::vector<cudaEvent_t> event_pool;      // events created so far (reused across windows)
+    size_t events_used;
+};
+
+// Brackets one kernel launch: counts it and, while profiling, records events around it on the
+// launching stream.
+struct nova_launch_scope {
+    nova_ctx* ctx;
+    cudaStream_t st;
+    cudaEvent_t stop;
+    nova_launch_scope(nova_ctx* c, int cat, cudaStream_t s) : ctx(c), st(s), stop(nullptr)
+    {
+        ctx->launches++;
+        if (!ctx->profiling) return;
+        while (ctx->event_pool.size() < ctx->events_used + 2) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return;
+            ctx->event_pool.push_back(e);
+        }
+        nova_prof_rec r;
+        r.cat = cat;
+        r.start = ctx->event_pool[ctx->events_used++];
+        r.stop = ctx->event_pool[ctx->events_used++];
+        cudaEventRecord(r.start, st);
+        ctx->prof_recs.push_back(r);
+        stop = r.stop;
+    }
+    ~nova_launch_scope()
+    {
+        if (stop) cudaEventRecord(stop, st);
+    }
 };
 
 static inline nova_status nova_fail(nova_ctx* ctx, nova_status s, const char* msg)
@@ -66,6 +114,7 @@ struct nova_gemm_args {
     const __nv_bfloat16* bias;  // [N]
     int M, N, K;
     int epilogue;
+    int cat;                    // nova_kernel_cat of this launch
     __nv_bfloat16* out;         // [M, N] (QKV: q buffer [M, C])
     // residual epilogue
     const __nv_bfloat16* res;   // residual rows of width N

@@ -222,9 +222,15 @@ extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nov
     if (row_stride < V || (row_stride % per) != 0 || !nova_aligned16(logits))
         return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_scale_entropy: logits rows must start on 16-byte boundaries");
     cudaStream_t st = (cudaStream_t)stream;
-    if (dt == NOVA_BF16) launch_rows<true>(logits, rows, V, row_stride, ent, ctx->dev_status, st);
-    else launch_rows<false>(logits, rows, V, row_stride, ent, ctx->dev_status, st);
-    if (mean) entropy_mean<<<S, 1024, 0, st>>>(ent, N, mean);
+    {
+        nova_launch_scope scope(ctx, NOVA_K_ENTROPY, st);
+        if (dt == NOVA_BF16) launch_rows<true>(logits, rows, V, row_stride, ent, ctx->dev_status, st);
+        else launch_rows<false>(logits, rows, V, row_stride, ent, ctx->dev_status, st);
+    }
+    if (mean) {
+        nova_launch_scope scope(ctx, NOVA_K_ENTROPY_MEAN, st);
+        entropy_mean<<<S, 1024, 0, st>>>(ent, N, mean);
+    }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }

@@ -225,7 +225,10 @@ nova_status launch(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
     p.res = a.res; p.res_row = a.res_row; p.C = a.C; p.k_cache = a.k_cache; p.v_cache = a.v_cache;
     p.kv_row = a.kv_row; p.status = ctx->dev_status;
     dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM);
-    kern<<<grid, kThreads, L::kTotal, st>>>(ta, tw, p);
+    {
+        nova_launch_scope scope(ctx, a.cat, st);
+        kern<<<grid, kThreads, L::kTotal, st>>>(ta, tw, p);
+    }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }

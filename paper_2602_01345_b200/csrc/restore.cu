@@ -148,6 +148,7 @@ extern "C" nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, 
         !nova_aligned16(cache_prev) || !nova_aligned16(cache_out))
         return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_restore_from_cache: tensors must be 16-byte aligned");
     const unsigned blocks = (unsigned)((total + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    nova_launch_scope scope(ctx, NOVA_K_RESTORE, (cudaStream_t)stream);
     restore_kernel<<<blocks, kWarpsPerBlock * 32, 0, (cudaStream_t)stream>>>(
         (const uint4*)x_in, (const uint4*)y_kept, keep_idx, prune_idx, cu_keep, (const uint4*)cache_prev,
         hp, wp, h, w, C / 8, B, M, (uint4*)x_out, (uint4*)cache_out);

@@ -179,7 +179,10 @@ extern "C" nova_status nova_select_topk(nova_ctx* ctx, const float* ent, int S, 
         SegParams sp;
         memset(&sp, 0, sizeof(sp));
         for (int s = 0; s < n; ++s) sp.k[s] = k[s0 + s];
-        select_topk_kernel<<<n, kThreads, (size_t)N * 4, st>>>(ent, N, s0, cu, sp, keep_idx, prune_idx, cu_keep, pos);
+        {
+            nova_launch_scope scope(ctx, NOVA_K_SELECT, st);
+            select_topk_kernel<<<n, kThreads, (size_t)N * 4, st>>>(ent, N, s0, cu, sp, keep_idx, prune_idx, cu_keep, pos);
+        }
         for (int s = 0; s < n; ++s) cu += k[s0 + s];
     }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());

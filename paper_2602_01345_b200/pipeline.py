@@ -1,0 +1,112 @@
+"""One accelerated scale through all layers: the call sequence a user of the library makes.
+
+For every layer j of the scale: entropy of the layer's logits -> (means to the host) ->
+keep counts from the trigger/ratio functions -> top-k selection -> block on the kept rows
+-> restore of the pruned rows from the residual cache. This module only owns buffers and
+issues the five C-ABI calls in order; it computes nothing itself.
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import torch
+
+from . import binding as nv
+
+
+class PrunedScaleRunner:
+    """Buffers and launch sequence for one pruned scale of an L-layer model.
+
+    weights:     list of L dicts of bf16 device tensors (see BlockWeights)
+    k_caches / v_caches: lists of L tensors [B, Lmax, C]; kv_len: int32 tensor [L, B]
+    cache_prev:  list of L tensors [B, hp, wp, C] (previous scale's residual cache per layer)
+    """
+
+    def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, h: int, w: int, Lmax: int,
+                 k_caches, v_caches, kv_len, cache_prev, eps: float = 1e-6, keep_cache_out: bool = True):
+        self.ctx = ctx
+        self.L = len(weights)
+        self.B, self.h, self.w, self.N = B, h, w, h * w
+        self.C = weights[0]["w_o"].shape[0]
+        self.F = weights[0]["w_fc1"].shape[0]
+        self.n_heads, self.Lmax = n_heads, Lmax
+        self.weights = [nv.BlockWeights(wt, eps) for wt in weights]
+        self.k_caches, self.v_caches, self.kv_len = k_caches, v_caches, kv_len
+        self.cache_prev = cache_prev
+        dev = weights[0]["w_o"].device
+        self.dev = dev
+        N, Cc = self.N, self.C
+        self.ent = torch.empty((B, N), dtype=torch.float32, device=dev)
+        self.mean = torch.empty((B,), dtype=torch.float32, device=dev)
+        self.mean_host = torch.empty((B,), dtype=torch.float32).pin_memory()
+        self.keep_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
+        self.prune_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
+        self.cu_keep = torch.empty((B + 1,), dtype=torch.int32, device=dev)
+        self.y_kept = torch.empty((B * N, Cc), dtype=torch.bfloat16, device=dev)
+        self.x_buf = [torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        self.cache_out = ([torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev) for _ in range(self.L)]
+                          if keep_cache_out else None)
+        ctx.ensure_workspace(nv.BlockShape(B, N, Cc, n_heads, self.F, Lmax, B * N))
+        self.last_keep = None
+
+    def run_scale(self, x_in, layer_logits, sched: nv.SchedParams, t: int, hbar_scale, append_kv: bool = True,
+                  stream=None, logits_ready=None):
+        """x_in [B, N, C] bf16; layer_logits: sequence of L tensors [B, N, V]; hbar_scale: CPU
+        float32 [B, t] with the mean entropies of scales 1..t. Returns (x_out, keeps) where keeps
+        is the list of per-layer keep-count tensors. `logits_ready`, if given, is a list of
+        torch.cuda.Event to wait for before layer j's logits are read (upload overlap).
+        """
+        ctx, B, N = self.ctx, self.B, self.N
+        st = stream if stream is not None else torch.cuda.current_stream()
+        hbar_layer = torch.empty((B, self.L), dtype=torch.float32)
+        keeps = []
+        x = x_in
+        for j in range(self.L):
+            if logits_ready is not None:
+                st.wait_event(logits_ready[j])
+            nv.nova_scale_entropy(ctx, layer_logits[j], self.ent, self.mean, stream=st)
+            self.mean_host.copy_(self.mean, non_blocking=True)
+            st.synchronize()                                    # the keep count is decided on the host
+            hbar_layer[:, j] = self.mean_host
+            r = nv.nova_keep_ratios(sched, t, j + 1, N, hbar_scale, hbar_layer[:, : j + 1].contiguous())
+            keep = r["keep"]
+            M = int(keep.sum())
+            keeps.append(keep)
+            nv.nova_select_topk(ctx, self.ent, keep, self.keep_idx[:M], self.prune_idx[: B * N - M], self.cu_keep,
+                                None, stream=st)
+            shape = nv.BlockShape(B, N, self.C, self.n_heads, self.F, self.Lmax, M)
+            nv.nova_pruned_block_forward(ctx, self.weights[j], shape, x, self.keep_idx[:M], self.cu_keep,
+                                         self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
+                                         self.y_kept[:M], stream=st)
+            x_out = self.x_buf[j & 1] if x is not self.x_buf[j & 1] else self.x_buf[(j + 1) & 1]
+            nv.nova_restore_from_cache(ctx, x, self.y_kept[:M], self.keep_idx[:M], self.prune_idx[: B * N - M],
+                                       self.cu_keep, self.cache_prev[j], self.h, self.w, x_out,
+                                       self.cache_out[j] if self.cache_out is not None else None, stream=st)
+            x = x_out
+        self.last_keep = keeps
+        return x, keeps
+
+
+def launch_count(ctx: nv.Context) -> int:
+    nv._lib.nova_launch_count.restype = C.c_ulonglong
+    nv._lib.nova_launch_count.argtypes = [C.c_void_p]
+    return int(nv._lib.nova_launch_count(ctx.handle))
+
+
+def profile_begin(ctx: nv.Context):
+    nv._lib.nova_profile_begin.argtypes = [C.c_void_p]
+    ctx.check(nv._lib.nova_profile_begin(ctx.handle))
+
+
+def profile_end(ctx: nv.Context) -> dict:
+    """Returns {kernel category: (summed device ms, launches)} for the profiling window."""
+    lib = nv._lib
+    lib.nova_profile_categories.restype = C.c_int
+    lib.nova_profile_category_name.restype = C.c_char_p
+    lib.nova_profile_category_name.argtypes = [C.c_int]
+    lib.nova_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.c_int]
+    n = lib.nova_profile_categories()
+    ms = (C.c_double * n)()
+    cnt = (C.c_longlong * n)()
+    ctx.check(lib.nova_profile_end(ctx.handle, ms, cnt, n))
+    return {lib.nova_profile_category_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n)}
