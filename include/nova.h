@@ -196,6 +196,37 @@ nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block_weights* w
                                       void* k_cache, void* v_cache, int32_t* kv_len,
                                       int append_kv, void* y_kept, void* stream);
 
+/* ---- the same block for callers that cannot allocate device memory ------------------ */
+/*
+ * (The paper has no counterpart to this call; it exists for deployment.)
+ * nova_pruned_block_forward needs a scratch buffer that the caller allocates and hands over
+ * with nova_set_workspace. Some callers cannot do that: a plug-in that runs inside a host
+ * program which has already given all device memory to its own pool and forbids cudaMalloc, or
+ * a latency-critical serving loop where cudaMalloc/cudaFree would synchronise the whole device.
+ * For them this entry point computes exactly what nova_pruned_block_forward computes, with the
+ * scratch taken from a fixed array built into the library (nova_static_scratch_bytes() bytes,
+ * currently 6 MiB, held by every GPU that loads the library until the process exits).
+ * Arguments, layouts, results and error behaviour are those of nova_pruned_block_forward, except:
+ *  - no workspace is needed or used; the context's own workspace setting is left untouched;
+ *  - a shape whose nova_block_workspace_bytes() exceeds nova_static_scratch_bytes() is rejected
+ *    with NOVA_ERR_WORKSPACE (nova_last_error() states both sizes). Width 1024 / MLP 4096 fits
+ *    up to 256 kept rows;
+ *  - the context's device must be the current CUDA device (else NOVA_ERR_INVALID_ARG);
+ *  - it is refused (NOVA_ERR_INVALID_ARG) between nova_profile_begin and nova_profile_end.
+ * It calls no cudaMalloc, cudaFree or other allocating routine. The first call on each device
+ * looks up the array's device address (a one-time set-up); make that first call before any
+ * stream capture begins. The array is shared by every call and every context in the process and
+ * keeps whatever the last call left in it; the kernels never read a scratch element before
+ * writing it, so nothing has to be cleared, but two calls that overlap on the GPU (different
+ * streams or contexts) race on it and give undefined results: serialise them.
+ */
+size_t      nova_static_scratch_bytes(void);
+nova_status nova_pruned_block_forward_static(nova_ctx* ctx, const nova_block_weights* w,
+                                             const nova_block_shape* s, const void* x_in,
+                                             const int32_t* keep_idx, const int32_t* cu_keep,
+                                             void* k_cache, void* v_cache, int32_t* kv_len,
+                                             int append_kv, void* y_kept, void* stream);
+
 /* ---- Eq. 15-16: residual cache reuse -------------------------------------------- */
 /*
  * x_in:       device bf16 [B, h*w, C]   layer input

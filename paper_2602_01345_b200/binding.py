@@ -245,3 +245,29 @@ def nova_restore_from_cache(ctx: Context, x_in, y_kept, keep_idx, prune_idx, cu_
     ctx.check(_lib.nova_restore_from_cache(ctx.handle, _ptr(x_in), _ptr(y_kept), _ptr(keep_idx), _ptr(prune_idx),
                                            _ptr(cu_keep), _ptr(cache_prev), hp, wp, h, w, Cc, B, M,
                                            _ptr(x_out), _ptr(cache_out), _stream(stream)))
+
+
+_lib.nova_static_scratch_bytes.argtypes = []
+_lib.nova_static_scratch_bytes.restype = C.c_size_t
+_lib.nova_pruned_block_forward_static.argtypes = _lib.nova_pruned_block_forward.argtypes
+_lib.nova_pruned_block_forward_static.restype = _i
+
+
+def nova_static_scratch_bytes() -> int:
+    """Size of the scratch array built into the library for nova_pruned_block_forward_static."""
+    return int(_lib.nova_static_scratch_bytes())
+
+
+def nova_pruned_block_forward_static(ctx: Context, w: BlockWeights, shape: BlockShape, x_in, keep_idx, cu_keep,
+                                     k_cache, v_cache, kv_len, append_kv, y_kept, stream=None):
+    """nova_pruned_block_forward for callers that may not allocate device memory (a plug-in inside
+    a host program that owns all device memory, a serving loop that cannot afford cudaMalloc's
+    device-wide synchronisation): same arguments and results, but the scratch comes from a fixed
+    array inside the library instead of a workspace tensor. Shapes that need more than
+    nova_static_scratch_bytes() are refused; calls that overlap on the GPU race on the array.
+    """
+    c = shape._c()
+    with torch.cuda.device(ctx.device):
+        ctx.check(_lib.nova_pruned_block_forward_static(
+            ctx.handle, C.byref(w.c), C.byref(c), _ptr(x_in), _ptr(keep_idx), _ptr(cu_keep), _ptr(k_cache),
+            _ptr(v_cache), _ptr(kv_len), int(bool(append_kv)), _ptr(y_kept), _stream(stream)))

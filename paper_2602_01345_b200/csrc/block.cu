@@ -256,3 +256,58 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     }
     return NOVA_OK;
 }
+
+// ---- block forward for callers that cannot allocate device memory --------------------------
+// The scratch that nova_pruned_block_forward normally takes from the caller's workspace lives
+// here, in a fixed array that is part of the library image: every GPU that loads the library
+// holds these bytes until the process exits.
+#define NOVA_STATIC_SCRATCH_BYTES (6u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[NOVA_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch per CUDA device ordinal. In host code the array's name is
+// only a handle for the runtime, not an address a kernel can use; the real address is looked up
+// once per device with that device current.
+static void* g_static_scratch_addr[64];
+
+extern "C" size_t nova_static_scratch_bytes(void) { return NOVA_STATIC_SCRATCH_BYTES; }
+
+extern "C" nova_status nova_pruned_block_forward_static(nova_ctx* ctx, const nova_block_weights* w,
+                                                        const nova_block_shape* s, const void* x_in,
+                                                        const int32_t* keep_idx, const int32_t* cu_keep,
+                                                        void* k_cache, void* v_cache, int32_t* kv_len,
+                                                        int append_kv, void* y_kept, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if (!s) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward_static: null shape");
+    if (ctx->profiling)
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG,
+                         "nova_pruned_block_forward_static: not available inside a profiling window (event creation may allocate)");
+    const size_t need = nova_block_workspace_bytes(s);
+    if (need == 0) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_pruned_block_forward_static: unsupported shape");
+    if (need > NOVA_STATIC_SCRATCH_BYTES) {
+        snprintf(ctx->err, sizeof(ctx->err),
+                 "nova_pruned_block_forward_static: shape needs %zu bytes of scratch, the built-in array holds %u",
+                 need, (unsigned)NOVA_STATIC_SCRATCH_BYTES);
+        return NOVA_ERR_WORKSPACE;
+    }
+    int cur = -1;
+    NOVA_CUDA_CHECK(ctx, cudaGetDevice(&cur));
+    if (cur != ctx->device || cur < 0 || cur >= 64)
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG,
+                         "nova_pruned_block_forward_static: the context's device must be the current device");
+    if (!g_static_scratch_addr[cur]) {
+        void* addr = nullptr;
+        NOVA_CUDA_CHECK(ctx, cudaGetSymbolAddress(&addr, g_static_scratch));
+        g_static_scratch_addr[cur] = addr;
+    }
+    // Run the ordinary path with the built-in array standing in for the caller's workspace.
+    void* saved_ws = ctx->workspace;
+    const size_t saved_bytes = ctx->workspace_bytes;
+    ctx->workspace = g_static_scratch_addr[cur];
+    ctx->workspace_bytes = NOVA_STATIC_SCRATCH_BYTES;
+    const nova_status rc = nova_pruned_block_forward(ctx, w, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len,
+                                                     append_kv, y_kept, stream);
+    ctx->workspace = saved_ws;
+    ctx->workspace_bytes = saved_bytes;
+    return rc;
+}
