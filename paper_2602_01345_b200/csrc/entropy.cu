@@ -62,7 +62,46 @@ __device__ __forceinline__ void finish_row(float m, float s, float u, float* ent
     ent[row] = h;
 }
 
+__device__ __forceinline__ float fmax_nan(float a, float b)   // NaN if either input is NaN
+{
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
+
+// Per-lane running state of the streaming softmax-entropy: m = largest logit seen, s = sum of
+// e^{z-m}, u = sum of (z-m) e^{z-m} (u kept in the log2 domain; m2 = m * log2 e). Raising m to m'
+// multiplies both sums by f = e^{m-m'} and shifts u by (m-m') s:  u' = f (u + (m-m') s),  s' = f s.
+struct RowState {
+    float m, m2, s, u;
+    __device__ __forceinline__ void raise_to(float m_new)
+    {
+        if (m == -INFINITY) { s = 0.f; u = 0.f; }
+        else {
+            const float shift = (m - m_new) * kLog2e;
+            const float f = fast_exp2(shift);
+            u = (u + shift * s) * f;
+            s *= f;
+        }
+        m = m_new;
+        m2 = m_new * kLog2e;
+    }
+    // One multiply-add, one clamp, one ex2, one add, one multiply-add per logit. The clamp turns a
+    // -inf (or NaN) exponent into a huge negative finite one whose ex2 is exactly 0, so that it
+    // contributes 0 instead of -inf * 0; NaN logits are caught by the NaN-propagating maximum.
+    __device__ __forceinline__ void add(float z)
+    {
+        const float d = fmaxf(fmaf(z, kLog2e, -m2), -16000.f);
+        const float e = fast_exp2(d);
+        s += e;
+        u = fmaf(d, e, u);
+    }
+};
+
 // VEC = number of 16-byte vectors each lane holds. BF16: 8 values per vector; F32: 4.
+// All loads of the row are issued before the first use (VEC * 16 bytes in flight per lane); the
+// values stay packed in registers and are consumed once, vector by vector, by the streaming
+// update above, so the register footprint is the packed row plus a handful of scalars.
 template <int VEC, bool BF16>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 entropy_rows_reg(const void* __restrict__ logits, long rows, int V, long row_stride,
@@ -93,47 +132,59 @@ entropy_rows_reg(const void* __restrict__ logits, long rows, int V, long row_str
         }
     }
 
-    float m = tail;
+    RowState st;
+    st.m = -INFINITY; st.m2 = -INFINITY; st.s = 0.f; st.u = 0.f;
+    bool saw_nan = false;
 #pragma unroll
     for (int i = 0; i < VEC; ++i) {
         const uint32_t w[4] = {reg[i].x, reg[i].y, reg[i].z, reg[i].w};
+        float cm;
+        if (BF16) {
+            // packed maximum: two logits per instruction
+            __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&w[0]);
+            __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&w[1]);
+            __nv_bfloat162 c = *reinterpret_cast<const __nv_bfloat162*>(&w[2]);
+            __nv_bfloat162 d = *reinterpret_cast<const __nv_bfloat162*>(&w[3]);
+            const __nv_bfloat162 mx = __hmax2_nan(__hmax2_nan(a, b), __hmax2_nan(c, d));
+            const uint32_t mw = *reinterpret_cast<const uint32_t*>(&mx);
+            float lo, hi;
+            unpack_bf16x2(mw, lo, hi);
+            cm = fmax_nan(lo, hi);
+        } else {
+            cm = fmax_nan(fmax_nan(__uint_as_float(w[0]), __uint_as_float(w[1])),
+                          fmax_nan(__uint_as_float(w[2]), __uint_as_float(w[3])));
+        }
+        saw_nan |= (cm != cm);
+        if (cm > st.m) st.raise_to(cm);             // rare after the first few vectors
+        if (st.m != -INFINITY) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            if (BF16) {
-                float a, b;
-                unpack_bf16x2(w[q], a, b);
-                m = fmaxf(m, fmaxf(a, b));
-            } else {
-                m = fmaxf(m, __uint_as_float(w[q]));
+            for (int q = 0; q < 4; ++q) {
+                if (BF16) {
+                    float lo, hi;
+                    unpack_bf16x2(w[q], lo, hi);
+                    st.add(lo);
+                    st.add(hi);
+                } else {
+                    st.add(__uint_as_float(w[q]));
+                }
             }
         }
     }
-    m = warp_max(m);
-    // fmaxf drops NaNs; catch them through the sum below (NaN - m = NaN propagates into s)
+    saw_nan |= (tail != tail);
+    if (tail > st.m) st.raise_to(tail);
+    if (st.m != -INFINITY) st.add(tail);
 
+    // merge the 32 lanes: common maximum, then rescaled sums
+    const float m = warp_max(st.m);
     float s = 0.f, u = 0.f;
-    auto acc = [&](float z) {
-        const float d = (z - m) * kLog2e;           // <= 0, and exactly 0 at the maximum
-        const float e = fast_exp2(d);
-        s += e;
-        u = fmaf(d == -INFINITY ? 0.f : d, e, u);  // -inf logit contributes 0, not -inf * 0
-    };
-#pragma unroll
-    for (int i = 0; i < VEC; ++i) {
-        const uint32_t w[4] = {reg[i].x, reg[i].y, reg[i].z, reg[i].w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            if (BF16) {
-                float a, b;
-                unpack_bf16x2(w[q], a, b);
-                acc(a);
-                acc(b);
-            } else {
-                acc(__uint_as_float(w[q]));
-            }
-        }
+    if (st.m != -INFINITY) {
+        const float shift = (st.m - m) * kLog2e;
+        const float f = fast_exp2(shift);
+        s = st.s * f;
+        u = (st.u + shift * st.s) * f;
+        if (shift == -INFINITY) { s = 0.f; u = 0.f; }   // m = +inf: flagged below through m
     }
-    acc(tail);
+    if (saw_nan) s = __int_as_float(0x7fc00000);
     s = warp_sum(s);
     u = warp_sum(u);
     if (lane == 0) finish_row(m, s, u, ent, row, status);

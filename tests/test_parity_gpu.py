@@ -96,7 +96,7 @@ def test_entropy_closed_forms_on_gpu(ctx):
     ent, _ = gpu_entropy(ctx, z)
     e = ent.cpu().numpy()[0]
     assert abs(e[0] - math.log(V)) <= ENT_TOL
-    assert e[1] == 0.0
+    assert 0.0 <= e[1] < 1e-6                           # exact in the oracle; fp32 rounding of ln s here
     Z = 7 * math.exp(3.0) + (V - 7)
     assert abs(e[2] - (math.log(Z) - 7 * 3.0 * math.exp(3.0) / Z)) <= ENT_TOL
     assert abs(e[3] - math.log(2048)) <= ENT_TOL
