@@ -1,15 +1,23 @@
 // Attention of the kept queries over [prior-scale K/V cache ++ kept tokens' own K/V]
 // (no mask), on the sm_100a tensor cores.
 //
-// One CTA = 128 query rows of one image and one head. Streaming (flash-style) softmax:
-//   warp 0      TMA producer: Q once, then a 2-stage ring of {K tile, V tile} (128 keys each)
-//   warp 1      tcgen05.mma issuer:  S = Q K^T  (fp32 in TMEM, double buffered)
-//                                    O_tile = P V (fp32 in TMEM)
-//   warps 2-5   one query row per thread: read S from TMEM, running max / sum, write
-//               P = exp2(...) as bf16 into shared memory in the swizzled K-major layout the
-//               tensor core reads, then fold O_tile into the fp32 output registers.
-// K tiles are K-major operands; V tiles are used as the MN-major B operand of P V, so V is
-// consumed exactly as it lies in the cache ([keys, dh] row-major).
+// One CTA = 256 query rows (two 128-row tiles A and B) of one image and one head, streaming
+// over 128-key tiles of K and V:
+//   warp 0        TMA producer: Q tiles once, then a ring of {K tile, V tile} stages
+//   warp 1        tcgen05.mma issuer. Per key tile j:  O_A += P_A V_j ; S_A = Q_A K_{j+1}^T ;
+//                 O_B += P_B V_j ; S_B = Q_B K_{j+1}^T.  S and O are fp32 in tensor memory and
+//                 O accumulates there across all key tiles.
+//   warps 2-5     softmax of tile A, one query row per thread: read the row of S from tensor
+//   warps 6-9     memory once, probabilities P = 2^((s - m) * scale) packed to bf16 and stored
+//   (tile B)      back into tensor memory over the S columns, from where the next MMA takes them
+//                 as its A operand. While one tile's softmax runs, the tensor core works on the
+//                 other tile.
+// The running maximum m is only raised (and O, l rescaled, in tensor memory) when the row maximum
+// grows by more than 2^8 in the exponent; until then probabilities are taken against the stale
+// maximum, which cancels in the final division by l. K tiles are K-major operands; V tiles are
+// the MN-major B operand, i.e. V is consumed exactly as it lies in the cache ([keys, dh]).
+// MMAs issued by one thread execute in issue order, which orders "P_A read by O_A += P_A V" before
+// "S_A overwritten by the next Q_A K^T" and "O complete" before the next S of the same tile.
 // Every mbarrier wait is bounded.
 #include "tc_common.cuh"
 
@@ -17,25 +25,22 @@ namespace {
 
 using namespace tc;
 
-constexpr int BQ = 128;        // query rows per CTA
+constexpr int BQ = 128;        // query rows per tile (two tiles per CTA)
 constexpr int BKV = 128;       // keys per tile
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr int kSlabBytes = 128 * 128;   // [128 rows][64 bf16]
-constexpr int kKvStages = 2;
+constexpr float kRescaleThreshold = 8.f;   // in log2 units
 
 template <int DH>
 struct AttnSmem {
+    static constexpr int kStages = (DH == 64) ? 4 : 2;
     static constexpr int kSlabs = DH / 64;
-    static constexpr int kQBytes = kSlabs * kSlabBytes;
-    static constexpr int kKBytes = kSlabs * kSlabBytes;
-    static constexpr int kVBytes = kSlabs * kSlabBytes;
-    static constexpr int kPBytes = 2 * kSlabBytes;
+    static constexpr int kTileBytes = kSlabs * kSlabBytes;      // one 128-row Q, K or V tile
     static constexpr int kQOff = 0;
-    static constexpr int kKOff = kQBytes;
-    static constexpr int kVOff = kKOff + kKvStages * kKBytes;
-    static constexpr int kPOff = kVOff + kKvStages * kVBytes;
-    static constexpr int kBarOff = kPOff + kPBytes;
-    static constexpr int kTotal = kBarOff + 256 + 1024;
+    static constexpr int kKOff = 2 * kTileBytes;
+    static constexpr int kVOff = kKOff + kStages * kTileBytes;
+    static constexpr int kBarOff = kVOff + kStages * kTileBytes;
+    static constexpr int kTotal = kBarOff + 512 + 1024;
 };
 
 struct AttnParams {
@@ -60,27 +65,30 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 }
 
 template <int DH>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                  const __grid_constant__ CUtensorMap tmap_v, const AttnParams p)
 {
     using L = AttnSmem<DH>;
     constexpr int kSlabs = L::kSlabs;
+    constexpr int kStages = L::kStages;
     constexpr uint32_t kTmemCols = 512;
-    constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
+    // S tile t (fp32) sits at column 128*t; its first 64 columns are reused for P (bf16 pairs).
+    // O tile t (fp32, DH columns) sits at column 256 + 128*t.
 
-    // ---- which (image, query tile) is this CTA? ------------------------------------
+    // ---- which (image, 256-row query block) is this CTA? -----------------------------
     int slot = blockIdx.x, b = 0, k_b = 0, q_begin = 0;
     bool found = false;
     for (b = 0; b < p.B; ++b) {
         const int c0 = p.cu_keep[b];
         k_b = p.cu_keep[b + 1] - c0;
-        const int tiles = (k_b + BQ - 1) / BQ;
-        if (slot < tiles) { q_begin = c0 + slot * BQ; found = true; break; }
-        slot -= tiles;
+        const int blocks = (k_b + 2 * BQ - 1) / (2 * BQ);
+        if (slot < blocks) { q_begin = c0 + slot * 2 * BQ; found = true; break; }
+        slot -= blocks;
     }
     if (!found) return;
-    const int rows_valid = min(BQ, k_b - slot * BQ);
+    const int rows_valid = min(2 * BQ, k_b - slot * 2 * BQ);
+    const bool tile_b_active = rows_valid > BQ;
     const int head = blockIdx.y;
     const int n_keys = min(p.kv_len[b] + k_b, p.Lmax);
     const int n_tiles = (n_keys + BKV - 1) / BKV;
@@ -88,14 +96,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = (uint64_t*)(smem + L::kBarOff);
-    uint64_t* q_full = bars;            // 1
-    uint64_t* k_full = bars + 1;        // 2
-    uint64_t* v_full = bars + 3;        // 2
-    uint64_t* kv_empty = bars + 5;      // 2
-    uint64_t* s_full = bars + 7;        // 2
-    uint64_t* p_full = bars + 9;        // 1 (128 arrivals)
-    uint64_t* o_full = bars + 10;       // 1
-    uint32_t* tmem_slot = (uint32_t*)(bars + 11);
+    uint64_t* q_full = bars;                          // 1
+    uint64_t* k_full = bars + 1;                      // kStages
+    uint64_t* v_full = k_full + kStages;              // kStages
+    uint64_t* kv_empty = v_full + kStages;            // kStages
+    uint64_t* s_full = kv_empty + kStages;            // 2 (tile A, tile B)
+    uint64_t* p_full = s_full + 2;                    // 2, 128 arrivals each
+    uint64_t* o_done = p_full + 2;                    // 1
+    uint32_t* tmem_slot = (uint32_t*)(o_done + 1);
     __shared__ int abort_flag_s;
     volatile int* abort_flag = &abort_flag_s;
 
@@ -104,14 +112,16 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         mbar_init(q_full, 1);
-        for (int s = 0; s < kKvStages; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             mbar_init(&k_full[s], 1);
             mbar_init(&v_full[s], 1);
             mbar_init(&kv_empty[s], 1);
-            mbar_init(&s_full[s], 1);
         }
-        mbar_init(p_full, 128);
-        mbar_init(o_full, 1);
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&s_full[t], 1);
+            mbar_init(&p_full[t], 128);
+        }
+        mbar_init(o_done, 1);
         fence_barrier_init();
         prefetch_tmap(&tmap_q);
         prefetch_tmap(&tmap_k);
@@ -124,32 +134,34 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
 
     uint8_t* q_smem = smem + L::kQOff;
-    uint8_t* p_smem = smem + L::kPOff;
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_arrive_expect_tx(q_full, L::kQBytes);
-            for (int sl = 0; sl < kSlabs; ++sl)
-                tma_load_2d(q_smem + sl * kSlabBytes, &tmap_q, q_full, head * DH + sl * 64, q_begin);
+            const int q_tiles = tile_b_active ? 2 : 1;
+            mbar_arrive_expect_tx(q_full, q_tiles * L::kTileBytes);
+            for (int t = 0; t < q_tiles; ++t)
+                for (int sl = 0; sl < kSlabs; ++sl)
+                    tma_load_2d(q_smem + t * L::kTileBytes + sl * kSlabBytes, &tmap_q, q_full,
+                                head * DH + sl * 64, q_begin + t * BQ);
             int issued = 0;
             for (int j = 0; j < n_tiles; ++j) {
-                const int s = j % kKvStages;
-                if (j >= kKvStages && !mbar_wait(&kv_empty[s], ((j / kKvStages) - 1) & 1, abort_flag, p.status)) break;
-                uint8_t* k_dst = smem + L::kKOff + s * L::kKBytes;
-                uint8_t* v_dst = smem + L::kVOff + s * L::kVBytes;
-                mbar_arrive_expect_tx(&k_full[s], L::kKBytes);
+                const int s = j % kStages;
+                if (j >= kStages && !mbar_wait(&kv_empty[s], ((j / kStages) - 1) & 1, abort_flag, p.status)) break;
+                uint8_t* k_dst = smem + L::kKOff + s * L::kTileBytes;
+                uint8_t* v_dst = smem + L::kVOff + s * L::kTileBytes;
+                mbar_arrive_expect_tx(&k_full[s], L::kTileBytes);
                 for (int sl = 0; sl < kSlabs; ++sl)
                     tma_load_3d(k_dst + sl * kSlabBytes, &tmap_k, &k_full[s], head * DH + sl * 64, j * BKV, b);
-                mbar_arrive_expect_tx(&v_full[s], L::kVBytes);
+                mbar_arrive_expect_tx(&v_full[s], L::kTileBytes);
                 for (int sl = 0; sl < kSlabs; ++sl)
                     tma_load_3d(v_dst + sl * kSlabBytes, &tmap_v, &v_full[s], head * DH + sl * 64, j * BKV, b);
                 issued = j + 1;
             }
             if (*abort_flag) {
                 mbar_drain(q_full, 0);
-                for (int j = max(0, issued - kKvStages); j < issued; ++j) {
-                    mbar_drain(&k_full[j % kKvStages], (j / kKvStages) & 1);
-                    mbar_drain(&v_full[j % kKvStages], (j / kKvStages) & 1);
+                for (int j = max(0, issued - kStages); j < issued; ++j) {
+                    mbar_drain(&k_full[j % kStages], (j / kStages) & 1);
+                    mbar_drain(&v_full[j % kStages], (j / kStages) & 1);
                 }
             }
         }
@@ -157,140 +169,167 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         if (lane == 0) {
             constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
             constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
-            const uint32_t q_addr = smem_u32(q_smem), p_addr = smem_u32(p_smem);
+            const uint32_t q_addr = smem_u32(q_smem);
+            const int n_q = tile_b_active ? 2 : 1;
             bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
-            auto issue_s = [&](int j) -> bool {
-                const int s = j % kKvStages;
-                if (!mbar_wait(&k_full[s], (j / kKvStages) & 1, abort_flag, p.status)) return false;
-                tc_fence_after();
-                const uint32_t k_addr = smem_u32(smem + L::kKOff + s * L::kKBytes);
-                const uint32_t d = tmem_base + ((j & 1) ? kColS1 : kColS0);
+            // S_t = Q_t K_j^T
+            auto issue_s = [&](int t, int j) {
+                const uint32_t k_addr = smem_u32(smem + L::kKOff + (j % kStages) * L::kTileBytes);
+                const uint32_t qa = q_addr + t * L::kTileBytes;
 #pragma unroll
                 for (int kk = 0; kk < DH / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * kSlabBytes + (kk & 3) * 32;
-                    mma_bf16_ss(d, smem_desc_sw128(q_addr + off, 16, 1024), smem_desc_sw128(k_addr + off, 16, 1024),
-                                idesc_s, kk ? 1u : 0u);
+                    mma_bf16_ss(tmem_base + 128u * t, smem_desc_sw128(qa + off, 16, 1024),
+                                smem_desc_sw128(k_addr + off, 16, 1024), idesc_s, kk ? 1u : 0u);
                 }
-                mma_commit(&s_full[j & 1]);
-                return true;
+                mma_commit(&s_full[t]);
             };
-            if (ok) ok = issue_s(0);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int s = j % kKvStages;
-                if (j + 1 < n_tiles) { ok = issue_s(j + 1); if (!ok) break; }
-                ok = mbar_wait(p_full, j & 1, abort_flag, p.status) &&
-                     mbar_wait(&v_full[s], (j / kKvStages) & 1, abort_flag, p.status);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t v_addr = smem_u32(smem + L::kVOff + s * L::kVBytes);
+            // O_t (+)= P_t V_j ; P_t sits in the first 64 columns of S_t, two keys per column
+            auto issue_pv = [&](int t, int j) {
+                const uint32_t v_addr = smem_u32(smem + L::kVOff + (j % kStages) * L::kTileBytes);
 #pragma unroll
                 for (int kk = 0; kk < BKV / 16; ++kk) {
-                    // A = P: K-major, 16 keys = 32 bytes inside a 64-key slab
-                    const uint64_t adesc = smem_desc_sw128(p_addr + (kk >> 2) * kSlabBytes + (kk & 3) * 32, 16, 1024);
-                    // B = V: MN-major (dh contiguous); 16 keys = 16 rows of 128 bytes; the next
-                    // 64 dh columns live one slab further (leading byte offset)
                     const uint64_t bdesc = smem_desc_sw128(v_addr + kk * 2048, kSlabBytes, 1024);
-                    mma_bf16_ss(tmem_base + kColO, adesc, bdesc, idesc_o, kk ? 1u : 0u);
+                    mma_bf16_ts(tmem_base + 256u + 128u * t, tmem_base + 128u * t + kk * 8, bdesc, idesc_o,
+                                (j | kk) ? 1u : 0u);
                 }
-                mma_commit(o_full);
-                mma_commit(&kv_empty[s]);
+            };
+            if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag, p.status);
+            if (ok) {
+                tc_fence_after();
+                for (int t = 0; t < n_q; ++t) issue_s(t, 0);
             }
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int s = j % kStages;
+                const bool more = j + 1 < n_tiles;
+                ok = mbar_wait(&v_full[s], (j / kStages) & 1, abort_flag, p.status);
+                if (ok && more) ok = mbar_wait(&k_full[(j + 1) % kStages], ((j + 1) / kStages) & 1, abort_flag, p.status);
+                for (int t = 0; t < n_q && ok; ++t) {
+                    ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(t, j);
+                    if (t == n_q - 1) mma_commit(&kv_empty[s]);   // K_j and V_j have no reader left
+                    if (more) issue_s(t, j + 1);
+                }
+            }
+            if (ok) mma_commit(o_done);
         }
     } else {
-        const int q = warp & 3;
-        const int row = q * 32 + lane;
-        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-        float o_acc[DH];
-#pragma unroll
-        for (int i = 0; i < DH; ++i) o_acc[i] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f;
-        bool ok = true;
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            ok = mbar_wait_warp(&s_full[j & 1], (j >> 1) & 1, abort_flag, p.status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t s_addr = tmem_base + lane_off + ((j & 1) ? kColS1 : kColS0);
-            const int cols_valid = min(BKV, n_keys - j * BKV);
-            // pass 1: row maximum over the valid keys
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < BKV / 32; ++c) {
-                uint32_t sv[32];
-                tmem_ld32(s_addr + c * 32, sv);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c * 32 + i < cols_valid) mx = fmaxf(mx, __uint_as_float(sv[i]));
-            }
-            const float m_new = fmaxf(m_run, mx);
-            const float alpha = ex2((m_run - m_new) * p.scale_log2e);
-            const float m_scaled = m_new * p.scale_log2e;
-            // pass 2: probabilities -> bf16 -> shared memory (row `row`, 128-byte swizzle)
-            float lsum = 0.f;
-            uint8_t* p_row = p_smem + (row >> 3) * 1024 + (row & 7) * 128;
-#pragma unroll 1
-            for (int c = 0; c < BKV / 32; ++c) {
-                uint32_t sv[32];
-                tmem_ld32(s_addr + c * 32, sv);
-                tmem_ld_wait();
-                float pv[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float e = ex2(fmaf(__uint_as_float(sv[i]), p.scale_log2e, -m_scaled));
-                    pv[i] = (c * 32 + i < cols_valid) ? e : 0.f;
-                    lsum += pv[i];
-                }
-                uint8_t* slab = p_row + (c >> 1) * kSlabBytes;
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const int chunk16 = (c & 1) * 4 + g;
-                    uint4 val = make_uint4(pack_bf16(pv[g * 8], pv[g * 8 + 1]), pack_bf16(pv[g * 8 + 2], pv[g * 8 + 3]),
-                                           pack_bf16(pv[g * 8 + 4], pv[g * 8 + 5]), pack_bf16(pv[g * 8 + 6], pv[g * 8 + 7]));
-                    *(uint4*)(slab + ((chunk16 ^ (row & 7)) << 4)) = val;
-                }
-            }
-            l_run = l_run * alpha + lsum;
-            m_run = m_new;
-            if (cols_valid < BKV) {
-                // ragged last tile: rows of V past the last key may hold anything (even NaN);
-                // zero them so that 0 * garbage cannot poison the accumulator
-                const int s = j % kKvStages;
-                ok = mbar_wait_warp(&v_full[s], (j / kKvStages) & 1, abort_flag, p.status);
+        const int t = (warp >= 6) ? 1 : 0;            // which query tile this warpgroup owns
+        if (t == 0 || tile_b_active) {
+            const int q = warp & 3;
+            const int row = q * 32 + lane;               // row within the tile = TMEM lane
+            const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+            const uint32_t s_addr = tmem_base + lane_off + 128u * t;
+            const uint32_t o_addr = tmem_base + lane_off + 256u + 128u * t;
+            const float c = p.scale_log2e;
+            float m_ref = -INFINITY, l_run = 0.f;
+            bool ok = true;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                ok = mbar_wait_warp(&s_full[t], j & 1, abort_flag, p.status);
                 if (!ok) break;
-                if (row >= cols_valid) {
-                    uint8_t* v_row = smem + L::kVOff + s * L::kVBytes + row * 128;
+                tc_fence_after();
+                uint32_t sv[128];
 #pragma unroll
-                    for (int sl = 0; sl < kSlabs; ++sl)
+                for (int cch = 0; cch < 4; ++cch) {
+                    uint32_t tmp[32];
+                    tmem_ld32(s_addr + cch * 32, tmp);
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) *(uint4*)(v_row + sl * kSlabBytes + g * 16) = make_uint4(0, 0, 0, 0);
+                    for (int i = 0; i < 32; ++i) sv[cch * 32 + i] = tmp[i];
+                }
+                tmem_ld_wait();
+                const int cols_valid = n_keys - j * BKV;      // >= 1
+                if (cols_valid < BKV) {
+#pragma unroll
+                    for (int i = 0; i < 128; ++i)
+                        if (i >= cols_valid) sv[i] = 0xff800000u;   // -inf: key past the end
+                }
+                float mx = __uint_as_float(sv[0]);
+#pragma unroll
+                for (int i = 1; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(sv[i]));
+                // raise the reference maximum only when it would change the exponent by > 2^8
+                const bool need = (mx - m_ref) * c > kRescaleThreshold;     // true on the first tile
+                if (__any_sync(0xffffffffu, need)) {
+                    const float m_new = fmaxf(m_ref, mx);
+                    const float alpha = ex2((m_ref - m_new) * c);             // 0 on the first tile
+                    if (j > 0) {
+#pragma unroll
+                        for (int cch = 0; cch < DH / 32; ++cch) {
+                            uint32_t ov[32];
+                            tmem_ld32(o_addr + cch * 32, ov);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                            tmem_st32(o_addr + cch * 32, ov);
+                        }
+                    }
+                    l_run *= alpha;
+                    m_ref = m_new;
+                }
+                const float m_scaled = m_ref * c;
+                float lsum0 = 0.f, lsum1 = 0.f;
+                uint32_t pk[64];
+#pragma unroll
+                for (int i = 0; i < 64; ++i) {
+                    const float p0 = ex2(fmaf(__uint_as_float(sv[2 * i]), c, -m_scaled));
+                    const float p1 = ex2(fmaf(__uint_as_float(sv[2 * i + 1]), c, -m_scaled));
+                    lsum0 += p0;
+                    lsum1 += p1;
+                    pk[i] = pack_bf16(p0, p1);
+                }
+                l_run += lsum0 + lsum1;
+                {
+                    uint32_t half[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) half[i] = pk[i];
+                    tmem_st32(s_addr, half);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) half[i] = pk[32 + i];
+                    tmem_st32(s_addr + 32, half);
+                }
+                tmem_st_wait();
+                if (t == 0 && cols_valid < BKV) {
+                    // ragged last tile: rows of V past the last key may hold anything (even NaN);
+                    // zero them so that 0 * garbage cannot poison the accumulator
+                    const int s = j % kStages;
+                    ok = mbar_wait_warp(&v_full[s], (j / kStages) & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    if (row >= cols_valid) {
+                        uint8_t* v_row = smem + L::kVOff + s * L::kTileBytes + row * 128;
+#pragma unroll
+                        for (int sl = 0; sl < kSlabs; ++sl)
+#pragma unroll
+                            for (int g = 0; g < 8; ++g) *(uint4*)(v_row + sl * kSlabBytes + g * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async_smem();
+                }
+                tc_fence_before();
+                mbar_arrive(&p_full[t]);
+            }
+            if (ok) ok = mbar_wait_warp(o_done, 0, abort_flag, p.status);
+            if (ok) {
+                tc_fence_after();
+                const float inv = 1.f / l_run;
+                const int grow = t * BQ + row;
+                __nv_bfloat16* dst_row = p.o + (long)(q_begin + grow) * p.C + head * DH;
+#pragma unroll
+                for (int cch = 0; cch < DH / 32; ++cch) {
+                    uint32_t ov[32];
+                    tmem_ld32(o_addr + cch * 32, ov);
+                    tmem_ld_wait();
+                    if (grow < rows_valid) {
+                        uint4* dst = (uint4*)(dst_row + cch * 32);
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)
+                            dst[g] = make_uint4(
+                                pack_bf16(__uint_as_float(ov[g * 8]) * inv, __uint_as_float(ov[g * 8 + 1]) * inv),
+                                pack_bf16(__uint_as_float(ov[g * 8 + 2]) * inv, __uint_as_float(ov[g * 8 + 3]) * inv),
+                                pack_bf16(__uint_as_float(ov[g * 8 + 4]) * inv, __uint_as_float(ov[g * 8 + 5]) * inv),
+                                pack_bf16(__uint_as_float(ov[g * 8 + 6]) * inv, __uint_as_float(ov[g * 8 + 7]) * inv));
+                    }
                 }
             }
-            fence_proxy_async_smem();
-            tc_fence_before();
-            mbar_arrive(p_full);
-            // fold this tile's P V into the running output
-            ok = mbar_wait_warp(o_full, j & 1, abort_flag, p.status);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < DH / 32; ++c) {
-                uint32_t ov[32];
-                tmem_ld32(tmem_base + lane_off + kColO + c * 32, ov);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) o_acc[c * 32 + i] = fmaf(o_acc[c * 32 + i], alpha, __uint_as_float(ov[i]));
-            }
-            tc_fence_before();
-        }
-        if (ok && row < rows_valid) {
-            const float inv = 1.f / l_run;
-            uint4* dst = (uint4*)(p.o + (long)(q_begin + row) * p.C + head * DH);
-#pragma unroll
-            for (int g = 0; g < DH / 8; ++g)
-                dst[g] = make_uint4(pack_bf16(o_acc[g * 8] * inv, o_acc[g * 8 + 1] * inv),
-                                    pack_bf16(o_acc[g * 8 + 2] * inv, o_acc[g * 8 + 3] * inv),
-                                    pack_bf16(o_acc[g * 8 + 4] * inv, o_acc[g * 8 + 5] * inv),
-                                    pack_bf16(o_acc[g * 8 + 6] * inv, o_acc[g * 8 + 7] * inv));
         }
     }
     tc_fence_before();
@@ -322,7 +361,7 @@ nova_status launch(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st)
     p.cu_keep = a.cu_keep; p.kv_len = a.kv_len; p.o = a.o; p.B = a.B; p.C = a.C; p.Lmax = a.Lmax;
     p.scale_log2e = (float)((1.0 / sqrt((double)DH)) * 1.4426950408889634);
     p.status = ctx->dev_status;
-    dim3 grid((a.M + BQ - 1) / BQ + a.B, a.n_heads);
+    dim3 grid((a.M + 2 * BQ - 1) / (2 * BQ) + a.B, a.n_heads);
     {
         nova_launch_scope scope(ctx, NOVA_K_ATTENTION, st);
         kern<<<grid, kThreads, L::kTotal, st>>>(tq, tk, tv, p);
