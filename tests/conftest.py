@@ -8,6 +8,20 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def _ensure_built():
+    """Compile libnova.so if it is missing or older than its sources (nvcc cross-compiles without a
+    GPU). The build script is loaded by path because the package refuses to import without the library."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location(
+        "_nova_build", os.path.join(ROOT, "paper_2602_01345_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.build()
+
+
+_ensure_built()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: test needs a CUDA device (B200)")
 
