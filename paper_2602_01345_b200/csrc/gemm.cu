@@ -6,6 +6,11 @@
 //   warp 1      allocates TMEM, issues tcgen05.mma (one elected thread), commits to mbarriers
 //   warps 2-5   epilogue: tcgen05.ld the fp32 accumulator (one row per thread), add bias,
 //               apply GELU / residual / QKV routing, store bf16
+// Large problems run on a second kernel, gemm_bf16_tn_pair: a persistent grid of CTA pairs
+// (clusters of two, tcgen05 cta_group::2), each pair computing 256 x BN tiles. Per tensor-core
+// instruction each CTA supplies only its 128 rows of A and BN/2 rows of W, which halves the
+// shared-memory and L2 traffic per flop of the single-CTA tile; the fp32 accumulator is double
+// buffered in tensor memory so that the epilogue of tile i overlaps the main loop of tile i+1.
 // Every mbarrier wait is bounded; on expiry the CTA records a timeout and tears down.
 #include "tc_common.cuh"
 
@@ -54,6 +59,58 @@ struct GemmParams {
     const int32_t* kv_row;
     unsigned int* status;
 };
+
+
+// Epilogue of 32 consecutive accumulator columns [col0, col0 + 32) of output row `row`:
+// + bias, then GELU / residual / QKV routing, rounded to bf16 and stored with 128-bit stores.
+__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int row, int col0, const uint32_t (&acc)[32],
+                                               long res_base, long kv_base)
+{
+    float v[32];
+    const uint4* bias4 = (const uint4*)(p.bias + col0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 b = bias4[i];
+        const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            v[i * 8 + j * 2] = __uint_as_float(acc[i * 8 + j * 2]) + __uint_as_float(bw[j] << 16);
+            v[i * 8 + j * 2 + 1] = __uint_as_float(acc[i * 8 + j * 2 + 1]) + __uint_as_float(bw[j] & 0xffff0000u);
+        }
+    }
+    __nv_bfloat16* dst;
+    if (p.epilogue == NOVA_EPI_BIAS_GELU) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = gelu_tanh(v[i]);
+        dst = p.out + (long)row * p.N + col0;
+    } else if (p.epilogue == NOVA_EPI_BIAS_RES) {
+        const uint4* r4 = (const uint4*)(p.res + res_base + col0);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint4 r = r4[i];
+            const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                v[i * 8 + j * 2] += __uint_as_float(rw[j] << 16);
+                v[i * 8 + j * 2 + 1] += __uint_as_float(rw[j] & 0xffff0000u);
+            }
+        }
+        dst = p.out + (long)row * p.N + col0;
+    } else {
+        // QKV routing: this 32-column chunk lies entirely in q, k or v (C % 32 == 0)
+        const int which = col0 / p.C, cc = col0 - which * p.C;
+        if (which == 0) dst = p.out + (long)row * p.C + cc;
+        else {
+            if (kv_base < 0) return;   // cache overflow: flagged when the row map was built
+            dst = (which == 1 ? p.k_cache : p.v_cache) + kv_base * p.C + cc;
+        }
+    }
+    uint4* d4 = (uint4*)dst;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        d4[i] = make_uint4(pack_bf16(v[i * 8], v[i * 8 + 1]), pack_bf16(v[i * 8 + 2], v[i * 8 + 3]),
+                           pack_bf16(v[i * 8 + 4], v[i * 8 + 5]), pack_bf16(v[i * 8 + 6], v[i * 8 + 7]));
+}
 
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(kThreads)
@@ -151,50 +208,7 @@ gemm_bf16_tn(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
                 tmem_ld32(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), acc);
                 tmem_ld_wait();
                 if (!row_ok || col0 >= p.N) continue;
-                float v[32];
-                const uint4* bias4 = (const uint4*)(p.bias + col0);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint4 b = bias4[i];
-                    const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        v[i * 8 + j * 2] = __uint_as_float(acc[i * 8 + j * 2]) + __uint_as_float(bw[j] << 16);
-                        v[i * 8 + j * 2 + 1] = __uint_as_float(acc[i * 8 + j * 2 + 1]) + __uint_as_float(bw[j] & 0xffff0000u);
-                    }
-                }
-                __nv_bfloat16* dst;
-                if (p.epilogue == NOVA_EPI_BIAS_GELU) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = gelu_tanh(v[i]);
-                    dst = p.out + (long)row * p.N + col0;
-                } else if (p.epilogue == NOVA_EPI_BIAS_RES) {
-                    const uint4* r4 = (const uint4*)(p.res + res_base + col0);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint4 r = r4[i];
-                        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            v[i * 8 + j * 2] += __uint_as_float(rw[j] << 16);
-                            v[i * 8 + j * 2 + 1] += __uint_as_float(rw[j] & 0xffff0000u);
-                        }
-                    }
-                    dst = p.out + (long)row * p.N + col0;
-                } else {
-                    // QKV routing: this 32-column chunk lies entirely in q, k or v (C % 32 == 0)
-                    const int which = col0 / p.C, cc = col0 - which * p.C;
-                    if (which == 0) dst = p.out + (long)row * p.C + cc;
-                    else {
-                        if (kv_base < 0) continue;   // cache overflow: flagged when the row map was built
-                        dst = (which == 1 ? p.k_cache : p.v_cache) + kv_base * p.C + cc;
-                    }
-                }
-                uint4* d4 = (uint4*)dst;
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    d4[i] = make_uint4(pack_bf16(v[i * 8], v[i * 8 + 1]), pack_bf16(v[i * 8 + 2], v[i * 8 + 3]),
-                                       pack_bf16(v[i * 8 + 4], v[i * 8 + 5]), pack_bf16(v[i * 8 + 6], v[i * 8 + 7]));
+                epilogue_chunk(p, row, col0, acc, res_base, kv_base);
             }
         }
     }
@@ -204,6 +218,205 @@ gemm_bf16_tn(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
         tc_fence_after();
         tmem_dealloc(tmem_acc, BN);
     }
+}
+
+GemmParams make_params(nova_ctx* ctx, const nova_gemm_args& a)
+{
+    GemmParams p;
+    p.bias = a.bias; p.M = a.M; p.N = a.N; p.K = a.K; p.epilogue = a.epilogue; p.out = a.out;
+    p.res = a.res; p.res_row = a.res_row; p.C = a.C; p.k_cache = a.k_cache; p.v_cache = a.v_cache;
+    p.kv_row = a.kv_row; p.status = ctx->dev_status;
+    return p;
+}
+
+// ---- CTA-pair kernel ------------------------------------------------------------------------
+constexpr int kPairBM = 256;           // rows of one pair tile (128 per CTA)
+
+template <int BN, int STAGES>
+struct PairSmem {
+    static constexpr int kABytes = 128 * BK * 2;           // this CTA's 128 rows of A
+    static constexpr int kBBytes = (BN / 2) * BK * 2;      // this CTA's half of the W rows
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kTotal = STAGES * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+// Role layout as in gemm_bf16_tn. Barriers (all in each CTA's shared memory at equal offsets):
+//   full[s]       leader's copy is used: one arrival (its own expect_tx) + the bytes of both CTAs
+//   empty[s]      each CTA's copy, signalled in both CTAs by the leader's tcgen05.commit
+//   acc_full[a]   each CTA's copy, same; a = accumulator buffer of tile parity
+//   acc_empty[a]  leader's copy: one arrival per epilogue warp of both CTAs (8)
+template <int BN, int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                  const GemmParams p, const int tiles_m, const int tiles_n)
+{
+    using L = PairSmem<BN, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* full_bar = (uint64_t*)(smem + STAGES * L::kStageBytes);
+    uint64_t* empty_bar = full_bar + STAGES;
+    uint64_t* acc_full = empty_bar + STAGES;     // 2
+    uint64_t* acc_empty = acc_full + 2;          // 2
+    uint32_t* tmem_slot = (uint32_t*)(acc_empty + 2);
+    __shared__ int abort_flag_s;
+    volatile int* abort_flag = &abort_flag_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();     // 0 = leader
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_tiles = tiles_m * tiles_n;
+    const int num_kb = p.K / BK;
+    constexpr uint32_t kTmemCols = 2 * BN;       // two accumulator buffers
+
+    if (threadIdx.x == 0) {
+        abort_flag_s = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&acc_full[a], 1);
+            mbar_init(&acc_empty[a], 8);
+        }
+        fence_barrier_init();
+        prefetch_tmap(&tmap_a);
+        prefetch_tmap(&tmap_w);
+    }
+    if (warp == 1) tmem_alloc_pair(tmem_slot, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                          // both CTAs' barriers exist before either signals the other
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            long it = 0;                         // k-blocks issued so far over all tiles of this pair
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+                const int m0 = (tile % tiles_m) * kPairBM + (int)rank * 128;
+                const int n0 = (tile / tiles_m) * BN + (int)rank * (BN / 2);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = (int)(it % STAGES);
+                    if (it >= STAGES && !mbar_wait(&empty_bar[s], (uint32_t)((it / STAGES) - 1) & 1, abort_flag, p.status)) {
+                        ok = false;
+                        break;
+                    }
+                    uint8_t* a_dst = smem + s * L::kStageBytes;
+                    uint8_t* b_dst = a_dst + L::kABytes;
+                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * L::kStageBytes);
+                    const uint32_t bar = map_to_cta(smem_u32(&full_bar[s]), 0);
+                    tma_load_2d_pair(a_dst, &tmap_a, bar, kb * BK, m0);
+                    tma_load_2d_pair(b_dst, &tmap_w, bar, kb * BK, n0);
+                }
+            }
+            if (*abort_flag && rank == 0) {
+                // let the copies already issued land before shared memory is released
+                for (long k2 = (it > STAGES ? it - STAGES : 0); k2 < it; ++k2)
+                    mbar_drain(&full_bar[k2 % STAGES], (uint32_t)(k2 / STAGES) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(kPairBM, BN, 0);
+            long it = 0;
+            int local = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++local) {
+                const int a = local & 1;
+                if (local >= 2) {
+                    ok = mbar_wait(&acc_empty[a], (uint32_t)((local >> 1) - 1) & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * BN);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = (int)(it % STAGES);
+                    ok = mbar_wait(&full_bar[s], (uint32_t)(it / STAGES) & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + s * L::kStageBytes);
+                    const uint32_t b_addr = a_addr + L::kABytes;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk) {
+                        const uint64_t adesc = smem_desc_sw128(a_addr + kk * 32, 16, 1024);
+                        const uint64_t bdesc = smem_desc_sw128(b_addr + kk * 32, 16, 1024);
+                        mma_bf16_ss_pair(d_tmem, adesc, bdesc, idesc, (kb | kk) ? 1u : 0u);
+                    }
+                    mma_commit_pair(&empty_bar[s], 3);      // frees the stage in both CTAs
+                }
+                if (ok) mma_commit_pair(&acc_full[a], 3);    // accumulator complete in both CTAs
+            }
+        }
+    } else {
+        // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31 of this CTA's half of the tile
+        const int q = warp & 3;
+        const uint32_t acc_empty_leader = map_to_cta(smem_u32(&acc_empty[0]), 0);
+        int local = 0;
+        bool ok = true;
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++local) {
+            const int a = local & 1;
+            const int row = (tile % tiles_m) * kPairBM + (int)rank * 128 + q * 32 + lane;
+            const int n0 = (tile / tiles_m) * BN;
+            ok = mbar_wait_warp(&acc_full[a], (uint32_t)(local >> 1) & 1, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const bool row_ok = row < p.M;
+            long res_base = 0;
+            long kv_base = -1;
+            if (row_ok) {
+                if (p.epilogue == NOVA_EPI_BIAS_RES) res_base = (long)(p.res_row ? p.res_row[row] : row) * p.N;
+                if (p.epilogue == NOVA_EPI_QKV) kv_base = (long)p.kv_row[row];
+            }
+            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * BN);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col0 = n0 + c * 32;
+                uint32_t acc[32];
+                tmem_ld32(t_addr + (uint32_t)(c * 32), acc);
+                tmem_ld_wait();
+                if (!row_ok || col0 >= p.N) continue;
+                epilogue_chunk(p, row, col0, acc, res_base, kv_base);
+            }
+            // this warp has read its part of the buffer: tell the leader's MMA thread
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty_leader + (uint32_t)(a * 8));
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();     // the peer may still read this CTA's shared memory or signal its barriers
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+template <int BN, int STAGES>
+nova_status launch_pair(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
+{
+    using L = PairSmem<BN, STAGES>;
+    CUtensorMap ta, tw;
+    const uint64_t da[2] = {(uint64_t)a.K, (uint64_t)a.M}, sa[1] = {(uint64_t)a.K * 2};
+    const uint64_t dw[2] = {(uint64_t)a.K, (uint64_t)a.N}, sw[1] = {(uint64_t)a.K * 2};
+    if (!make_tmap_bf16(ctx, &ta, a.A, 2, da, sa, 128) || !make_tmap_bf16(ctx, &tw, a.W, 2, dw, sw, BN / 2))
+        return nova_fail(ctx, NOVA_ERR_CUDA, "gemm: cuTensorMapEncodeTiled failed");
+    auto kern = gemm_bf16_tn_pair<BN, STAGES>;
+    static bool attr_done[64];
+    if (ctx->device < 64 && !attr_done[ctx->device]) {
+        NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
+        attr_done[ctx->device] = true;
+    }
+    GemmParams p = make_params(ctx, a);
+    const int tiles_m = (a.M + kPairBM - 1) / kPairBM, tiles_n = (a.N + BN - 1) / BN;
+    const int pairs = min(tiles_m * tiles_n, ctx->num_sms / 2);
+    {
+        nova_launch_scope scope(ctx, a.cat, st);
+        kern<<<dim3(2 * pairs), kThreads, L::kTotal, st>>>(ta, tw, p, tiles_m, tiles_n);
+    }
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    return NOVA_OK;
 }
 
 template <int BN, int STAGES>
@@ -220,10 +433,7 @@ nova_status launch(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
         NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal));
         ctx->attr_gemm = true;
     }
-    GemmParams p;
-    p.bias = a.bias; p.M = a.M; p.N = a.N; p.K = a.K; p.epilogue = a.epilogue; p.out = a.out;
-    p.res = a.res; p.res_row = a.res_row; p.C = a.C; p.k_cache = a.k_cache; p.v_cache = a.v_cache;
-    p.kv_row = a.kv_row; p.status = ctx->dev_status;
+    GemmParams p = make_params(ctx, a);
     dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM);
     {
         nova_launch_scope scope(ctx, a.cat, st);
@@ -239,5 +449,9 @@ nova_status nova_launch_gemm(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_
 {
     if (a.M <= 0) return NOVA_OK;
     if (a.K % BK || a.N % 32 || a.K < BK) return nova_fail(ctx, NOVA_ERR_SHAPE, "gemm: K must be a multiple of 64 and N of 32");
+    // CTA pairs with 256 x 256 tiles once there is at least one tile per pair of SMs; below that the
+    // single-CTA 128 x 128 tiles spread a small problem over more SMs.
+    const long tiles_pair = (long)((a.M + 255) / 256) * ((a.N + 255) / 256);
+    if (tiles_pair >= ctx->num_sms / 2 && ctx->num_sms >= 2) return launch_pair<256, 6>(ctx, a, st);
     return launch<128, 3>(ctx, a, st);
 }

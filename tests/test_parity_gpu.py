@@ -309,6 +309,18 @@ def test_block_keep_all_equals_dense(ctx):
     _block_case(ctx, B=1, N=256, C=128, heads=2, F=256, Lmax=512, ks=[256], kv_lens=[100], seed=7)
 
 
+def test_block_full_size_1024_shape_sampled_rows(ctx):
+    """The 1024x1024 large-model shape in the configuration the benchmark times (batch 4, 4096
+    tokens per image, about half kept, 6425 prior tokens, width 2048, 16 heads x 128, MLP 8192),
+    with ragged keep counts so the last row tile is partial. The appended K/V rows are compared
+    for every kept token; the block output on sampled rows (tile corners, the ragged tail)."""
+    ks = [2048, 1901, 2048, 2100]
+    M = sum(ks)
+    rows = [0, 127, 128, 2047, 2048, 2048 + 1900, M - 2100, M - 130, M - 1]
+    _block_case(ctx, B=4, N=4096, C=2048, heads=16, F=8192, Lmax=10521, ks=ks, kv_lens=[6425] * 4, seed=11,
+                rows=np.array(rows, np.int32))
+
+
 def test_block_without_append_leaves_kv_len(ctx):
     B, N, C, heads, F, Lmax = 1, 64, 128, 2, 256, 256
     wt = synth.block_weights(C, F, 1, DEV)
