@@ -240,6 +240,36 @@ struct PairSmem {
     static constexpr int kTotal = STAGES * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
+// Work list of one launch: entries [0, tiles_full) are whole 256 x BN tiles in column-major tile
+// order; the tiles after those, which would otherwise leave most pairs idle in a last partial wave,
+// are each split into two 256 x BN/2 halves (entries tiles_full, tiles_full + 1, ...).
+struct PairTile {
+    int m0;     // first row of the pair tile
+    int n0;     // first column
+    int bn;     // columns: BN or BN / 2
+};
+// `span` > 0: tile index = m_tile + tiles_m * n_tile with span = tiles_m (tiles that run at the same
+// time share few W rows and sweep all of A); span < 0: index = n_tile + tiles_n * m_tile with
+// -span = tiles_n (they sweep all of W and share few A rows). The launcher picks the order whose
+// swept operand is the smaller one, so that the larger one is fetched from HBM only once.
+template <int BN>
+__device__ __forceinline__ PairTile decode_tile(int entry, int span, int tiles_full)
+{
+    PairTile t;
+    int whole = entry, half = -1;
+    if (entry >= tiles_full) {
+        const int h = entry - tiles_full;
+        whole = tiles_full + (h >> 1);
+        half = h & 1;
+    }
+    const int mt = span > 0 ? whole % span : whole / (-span);
+    const int nt = span > 0 ? whole / span : whole % (-span);
+    t.m0 = mt * kPairBM;
+    t.n0 = nt * BN + (half > 0 ? BN / 2 : 0);
+    t.bn = half >= 0 ? BN / 2 : BN;
+    return t;
+}
+
 // Role layout as in gemm_bf16_tn. Barriers (all in each CTA's shared memory at equal offsets):
 //   full[s]       leader's copy is used: one arrival (its own expect_tx) + the bytes of both CTAs
 //   empty[s]      each CTA's copy, signalled in both CTAs by the leader's tcgen05.commit
@@ -248,7 +278,8 @@ struct PairSmem {
 template <int BN, int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-                  const GemmParams p, const int tiles_m, const int tiles_n)
+                  const __grid_constant__ CUtensorMap tmap_w_half, const GemmParams p, const int span,
+                  const int tiles_full, const int num_tiles)
 {
     using L = PairSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
@@ -264,7 +295,6 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();     // 0 = leader
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int num_tiles = tiles_m * tiles_n;
     const int num_kb = p.K / BK;
     constexpr uint32_t kTmemCols = 2 * BN;       // two accumulator buffers
 
@@ -281,6 +311,7 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         fence_barrier_init();
         prefetch_tmap(&tmap_a);
         prefetch_tmap(&tmap_w);
+        prefetch_tmap(&tmap_w_half);
     }
     if (warp == 1) tmem_alloc_pair(tmem_slot, kTmemCols);
     tc_fence_before();
@@ -294,8 +325,11 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             long it = 0;                         // k-blocks issued so far over all tiles of this pair
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
-                const int m0 = (tile % tiles_m) * kPairBM + (int)rank * 128;
-                const int n0 = (tile / tiles_m) * BN + (int)rank * (BN / 2);
+                const PairTile t = decode_tile<BN>(tile, span, tiles_full);
+                const int m0 = t.m0 + (int)rank * 128;
+                const int n0 = t.n0 + (int)rank * (t.bn / 2);
+                const CUtensorMap* wmap = (t.bn == BN) ? &tmap_w : &tmap_w_half;
+                const uint32_t stage_tx = 2u * (uint32_t)(L::kABytes + (t.bn / 2) * BK * 2);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = (int)(it % STAGES);
                     if (it >= STAGES && !mbar_wait(&empty_bar[s], (uint32_t)((it / STAGES) - 1) & 1, abort_flag, p.status)) {
@@ -304,10 +338,10 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                     uint8_t* a_dst = smem + s * L::kStageBytes;
                     uint8_t* b_dst = a_dst + L::kABytes;
-                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * L::kStageBytes);
+                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], stage_tx);
                     const uint32_t bar = map_to_cta(smem_u32(&full_bar[s]), 0);
                     tma_load_2d_pair(a_dst, &tmap_a, bar, kb * BK, m0);
-                    tma_load_2d_pair(b_dst, &tmap_w, bar, kb * BK, n0);
+                    tma_load_2d_pair(b_dst, wmap, bar, kb * BK, n0);
                 }
             }
             if (*abort_flag && rank == 0) {
@@ -318,7 +352,8 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = idesc_bf16_f32(kPairBM, BN, 0);
+            constexpr uint32_t idesc_whole = idesc_bf16_f32(kPairBM, BN, 0);
+            constexpr uint32_t idesc_half = idesc_bf16_f32(kPairBM, BN / 2, 0);
             long it = 0;
             int local = 0;
             bool ok = true;
@@ -330,6 +365,7 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     tc_fence_after();
                 }
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * BN);
+                const uint32_t idesc = (tile < tiles_full) ? idesc_whole : idesc_half;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = (int)(it % STAGES);
                     ok = mbar_wait(&full_bar[s], (uint32_t)(it / STAGES) & 1, abort_flag, p.status);
@@ -356,8 +392,9 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         bool ok = true;
         for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++local) {
             const int a = local & 1;
-            const int row = (tile % tiles_m) * kPairBM + (int)rank * 128 + q * 32 + lane;
-            const int n0 = (tile / tiles_m) * BN;
+            const PairTile t = decode_tile<BN>(tile, span, tiles_full);
+            const int row = t.m0 + (int)rank * 128 + q * 32 + lane;
+            const int n0 = t.n0, n_chunks = t.bn / 32;
             ok = mbar_wait_warp(&acc_full[a], (uint32_t)(local >> 1) & 1, abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
@@ -370,7 +407,7 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * BN);
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = 0; c < n_chunks; ++c) {
                 const int col0 = n0 + c * 32;
                 uint32_t acc[32];
                 tmem_ld32(t_addr + (uint32_t)(c * 32), acc);
@@ -400,7 +437,9 @@ nova_status launch_pair(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
     CUtensorMap ta, tw;
     const uint64_t da[2] = {(uint64_t)a.K, (uint64_t)a.M}, sa[1] = {(uint64_t)a.K * 2};
     const uint64_t dw[2] = {(uint64_t)a.K, (uint64_t)a.N}, sw[1] = {(uint64_t)a.K * 2};
-    if (!make_tmap_bf16(ctx, &ta, a.A, 2, da, sa, 128) || !make_tmap_bf16(ctx, &tw, a.W, 2, dw, sw, BN / 2))
+    CUtensorMap tw_half;
+    if (!make_tmap_bf16(ctx, &ta, a.A, 2, da, sa, 128) || !make_tmap_bf16(ctx, &tw, a.W, 2, dw, sw, BN / 2) ||
+        !make_tmap_bf16(ctx, &tw_half, a.W, 2, dw, sw, BN / 4))
         return nova_fail(ctx, NOVA_ERR_CUDA, "gemm: cuTensorMapEncodeTiled failed");
     auto kern = gemm_bf16_tn_pair<BN, STAGES>;
     static bool attr_done[64];
@@ -410,10 +449,16 @@ nova_status launch_pair(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
     }
     GemmParams p = make_params(ctx, a);
     const int tiles_m = (a.M + kPairBM - 1) / kPairBM, tiles_n = (a.N + BN - 1) / BN;
-    const int pairs = min(tiles_m * tiles_n, ctx->num_sms / 2);
+    const int tiles = tiles_m * tiles_n;
+    const int pairs = min(tiles, ctx->num_sms / 2);
+    // a last partial wave that would occupy at most half of the pairs runs as half-width tiles
+    const int rem = tiles % pairs;
+    const int tiles_full = (rem > 0 && 2 * rem <= pairs) ? tiles - rem : tiles;
+    const int entries = tiles_full + 2 * (tiles - tiles_full);
     {
         nova_launch_scope scope(ctx, a.cat, st);
-        kern<<<dim3(2 * pairs), kThreads, L::kTotal, st>>>(ta, tw, p, tiles_m, tiles_n);
+        const int span = ((long)a.M >= (long)a.N) ? -tiles_n : tiles_m;   // sweep the smaller operand
+        kern<<<dim3(2 * pairs), kThreads, L::kTotal, st>>>(ta, tw, tw_half, p, span, tiles_full, entries);
     }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
