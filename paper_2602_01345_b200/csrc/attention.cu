@@ -33,13 +33,17 @@ constexpr float kRescaleThreshold = 8.f;   // in log2 units
 
 template <int DH>
 struct AttnSmem {
-    static constexpr int kStages = (DH == 64) ? 4 : 2;
+    // K tiles are released right after the last S = Q K^T that reads them, V tiles only after
+    // O += P V one softmax later, so the two rings run separately; head size 128 fills the
+    // 227 KB with two Q tiles, three K stages and two V stages.
+    static constexpr int kKStages = (DH == 64) ? 4 : 3;
+    static constexpr int kVStages = (DH == 64) ? 4 : 2;
     static constexpr int kSlabs = DH / 64;
     static constexpr int kTileBytes = kSlabs * kSlabBytes;      // one 128-row Q, K or V tile
     static constexpr int kQOff = 0;
     static constexpr int kKOff = 2 * kTileBytes;
-    static constexpr int kVOff = kKOff + kStages * kTileBytes;
-    static constexpr int kBarOff = kVOff + kStages * kTileBytes;
+    static constexpr int kVOff = kKOff + kKStages * kTileBytes;
+    static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
     static constexpr int kTotal = kBarOff + 512 + 1024;
 };
 
@@ -64,6 +68,73 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// ---- two fp32 values per 64-bit register: one instruction does both lanes' arithmetic ----------
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_rm_f32x2(uint64_t a, uint64_t b)   // rounds toward -inf
+{
+    uint64_t r;
+    asm("add.rm.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t sub_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// 2^x for two values without the special-function unit, which the softmax would otherwise
+// saturate (it evaluates 16 exponentials per clock per SM against 128 multiply-adds). With
+// t = x + 1.5 * 2^23 rounded toward -inf, the low bits of t hold j = floor(x) and f = x - j lies in
+// [0, 1); 2^f comes from a cubic fitted to 9.2e-5 relative error (far below the bf16 rounding the
+// probabilities get next) and j is added to the exponent field as an integer. x is clamped at
+// -126 so that the exponent cannot wrap; a masked (-inf) score therefore yields 2^-126, not 0.
+__device__ __forceinline__ void exp2_poly_x2(uint64_t x2, float& p0, float& p1)
+{
+    float x0, x1;
+    unpack_f32x2(x2, x0, x1);
+    const uint64_t xc = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const uint64_t magic = pack_f32x2(12582912.f, 12582912.f);
+    const uint64_t t = add_rm_f32x2(xc, magic);
+    const uint64_t f = sub_f32x2(xc, sub_f32x2(t, magic));
+    uint64_t q = fma_f32x2(f, pack_f32x2(0.07711965590715408f, 0.07711965590715408f),
+                           pack_f32x2(0.2276432067155838f, 0.2276432067155838f));
+    q = fma_f32x2(q, f, pack_f32x2(0.6950892806053162f, 0.6950892806053162f));
+    q = fma_f32x2(q, f, pack_f32x2(1.f, 1.f));
+    float q0, q1, t0, t1;
+    unpack_f32x2(q, q0, q1);
+    unpack_f32x2(t, t0, t1);
+    p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+    p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -71,7 +142,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 {
     using L = AttnSmem<DH>;
     constexpr int kSlabs = L::kSlabs;
-    constexpr int kStages = L::kStages;
+    constexpr int kKStages = L::kKStages, kVStages = L::kVStages;
     constexpr uint32_t kTmemCols = 512;
     // S tile t (fp32) sits at column 128*t; its first 64 columns are reused for P (bf16 pairs).
     // O tile t (fp32, DH columns) sits at column 256 + 128*t.
@@ -97,10 +168,11 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = (uint64_t*)(smem + L::kBarOff);
     uint64_t* q_full = bars;                          // 1
-    uint64_t* k_full = bars + 1;                      // kStages
-    uint64_t* v_full = k_full + kStages;              // kStages
-    uint64_t* kv_empty = v_full + kStages;            // kStages
-    uint64_t* s_full = kv_empty + kStages;            // 2 (tile A, tile B)
+    uint64_t* k_full = bars + 1;                      // kKStages
+    uint64_t* k_empty = k_full + kKStages;            // kKStages
+    uint64_t* v_full = k_empty + kKStages;            // kVStages
+    uint64_t* v_empty = v_full + kVStages;            // kVStages
+    uint64_t* s_full = v_empty + kVStages;            // 2 (tile A, tile B)
     uint64_t* p_full = s_full + 2;                    // 2, 128 arrivals each
     uint64_t* o_done = p_full + 2;                    // 1
     uint32_t* tmem_slot = (uint32_t*)(o_done + 1);
@@ -112,10 +184,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         mbar_init(q_full, 1);
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kKStages; ++s) {
             mbar_init(&k_full[s], 1);
+            mbar_init(&k_empty[s], 1);
+        }
+        for (int s = 0; s < kVStages; ++s) {
             mbar_init(&v_full[s], 1);
-            mbar_init(&kv_empty[s], 1);
+            mbar_init(&v_empty[s], 1);
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&s_full[t], 1);
@@ -143,74 +218,84 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 for (int sl = 0; sl < kSlabs; ++sl)
                     tma_load_2d(q_smem + t * L::kTileBytes + sl * kSlabBytes, &tmap_q, q_full,
                                 head * DH + sl * 64, q_begin + t * BQ);
-            int issued = 0;
+            // order of issue = order in which the slots come free: K_j, V_j, K_{j+1}, ...
+            int k_issued = 0, v_issued = 0;
             for (int j = 0; j < n_tiles; ++j) {
-                const int s = j % kStages;
-                if (j >= kStages && !mbar_wait(&kv_empty[s], ((j / kStages) - 1) & 1, abort_flag, p.status)) break;
-                uint8_t* k_dst = smem + L::kKOff + s * L::kTileBytes;
-                uint8_t* v_dst = smem + L::kVOff + s * L::kTileBytes;
-                mbar_arrive_expect_tx(&k_full[s], L::kTileBytes);
+                const int ks = j % kKStages, vs = j % kVStages;
+                if (j >= kKStages && !mbar_wait(&k_empty[ks], ((j / kKStages) - 1) & 1, abort_flag, p.status)) break;
+                uint8_t* k_dst = smem + L::kKOff + ks * L::kTileBytes;
+                mbar_arrive_expect_tx(&k_full[ks], L::kTileBytes);
                 for (int sl = 0; sl < kSlabs; ++sl)
-                    tma_load_3d(k_dst + sl * kSlabBytes, &tmap_k, &k_full[s], head * DH + sl * 64, j * BKV, b);
-                mbar_arrive_expect_tx(&v_full[s], L::kTileBytes);
+                    tma_load_3d(k_dst + sl * kSlabBytes, &tmap_k, &k_full[ks], head * DH + sl * 64, j * BKV, b);
+                k_issued = j + 1;
+                if (j >= kVStages && !mbar_wait(&v_empty[vs], ((j / kVStages) - 1) & 1, abort_flag, p.status)) break;
+                uint8_t* v_dst = smem + L::kVOff + vs * L::kTileBytes;
+                mbar_arrive_expect_tx(&v_full[vs], L::kTileBytes);
                 for (int sl = 0; sl < kSlabs; ++sl)
-                    tma_load_3d(v_dst + sl * kSlabBytes, &tmap_v, &v_full[s], head * DH + sl * 64, j * BKV, b);
-                issued = j + 1;
+                    tma_load_3d(v_dst + sl * kSlabBytes, &tmap_v, &v_full[vs], head * DH + sl * 64, j * BKV, b);
+                v_issued = j + 1;
             }
             if (*abort_flag) {
                 mbar_drain(q_full, 0);
-                for (int j = max(0, issued - kStages); j < issued; ++j) {
-                    mbar_drain(&k_full[j % kStages], (j / kStages) & 1);
-                    mbar_drain(&v_full[j % kStages], (j / kStages) & 1);
-                }
+                for (int j = max(0, k_issued - kKStages); j < k_issued; ++j) mbar_drain(&k_full[j % kKStages], (j / kKStages) & 1);
+                for (int j = max(0, v_issued - kVStages); j < v_issued; ++j) mbar_drain(&v_full[j % kVStages], (j / kVStages) & 1);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
             constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
-            const uint32_t q_addr = smem_u32(q_smem);
             const int n_q = tile_b_active ? 2 : 1;
+            // Shared-memory descriptors are split into a constant high word and a low word that
+            // holds (address >> 4) in its low 14 bits, so stepping through a tile is one integer
+            // add per operand: the issuing thread has about 64 clocks per instruction to stay
+            // ahead of the tensor core.
+            const uint64_t q_desc = smem_desc_sw128(smem_u32(q_smem), 16, 1024);
+            const uint64_t k_desc = smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024);
+            const uint64_t v_desc = smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024);
+            constexpr uint32_t kTileStep = L::kTileBytes >> 4;
             bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
             // S_t = Q_t K_j^T
             auto issue_s = [&](int t, int j) {
-                const uint32_t k_addr = smem_u32(smem + L::kKOff + (j % kStages) * L::kTileBytes);
-                const uint32_t qa = q_addr + t * L::kTileBytes;
+                const uint64_t qd = q_desc + (uint32_t)t * kTileStep;
+                const uint64_t kd = k_desc + (uint32_t)(j % kKStages) * kTileStep;
 #pragma unroll
                 for (int kk = 0; kk < DH / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * kSlabBytes + (kk & 3) * 32;
-                    mma_bf16_ss(tmem_base + 128u * t, smem_desc_sw128(qa + off, 16, 1024),
-                                smem_desc_sw128(k_addr + off, 16, 1024), idesc_s, kk ? 1u : 0u);
+                    constexpr uint32_t kSlabStep = kSlabBytes >> 4;
+                    const uint32_t off = (kk >> 2) * kSlabStep + (kk & 3) * 2;    // 32 bytes per 16 k
+                    mma_bf16_ss(tmem_base + 128u * t, qd + off, kd + off, idesc_s, kk ? 1u : 0u);
                 }
                 mma_commit(&s_full[t]);
             };
             // O_t (+)= P_t V_j ; P_t sits in the first 64 columns of S_t, two keys per column
             auto issue_pv = [&](int t, int j) {
-                const uint32_t v_addr = smem_u32(smem + L::kVOff + (j % kStages) * L::kTileBytes);
+                const uint64_t vd = v_desc + (uint32_t)(j % kVStages) * kTileStep;
 #pragma unroll
-                for (int kk = 0; kk < BKV / 16; ++kk) {
-                    const uint64_t bdesc = smem_desc_sw128(v_addr + kk * 2048, kSlabBytes, 1024);
-                    mma_bf16_ts(tmem_base + 256u + 128u * t, tmem_base + 128u * t + kk * 8, bdesc, idesc_o,
-                                (j | kk) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < BKV / 16; ++kk)
+                    mma_bf16_ts(tmem_base + 256u + 128u * t, tmem_base + 128u * t + kk * 8, vd + (uint32_t)(kk * 128),
+                                idesc_o, (j | kk) ? 1u : 0u);
             };
             if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag, p.status);
             if (ok) {
                 tc_fence_after();
                 for (int t = 0; t < n_q; ++t) issue_s(t, 0);
+                mma_commit(&k_empty[0]);
             }
             for (int j = 0; j < n_tiles && ok; ++j) {
-                const int s = j % kStages;
+                const int vs = j % kVStages;
                 const bool more = j + 1 < n_tiles;
-                ok = mbar_wait(&v_full[s], (j / kStages) & 1, abort_flag, p.status);
-                if (ok && more) ok = mbar_wait(&k_full[(j + 1) % kStages], ((j + 1) / kStages) & 1, abort_flag, p.status);
+                ok = mbar_wait(&v_full[vs], (j / kVStages) & 1, abort_flag, p.status);
+                if (ok && more) ok = mbar_wait(&k_full[(j + 1) % kKStages], ((j + 1) / kKStages) & 1, abort_flag, p.status);
                 for (int t = 0; t < n_q && ok; ++t) {
                     ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(t, j);
-                    if (t == n_q - 1) mma_commit(&kv_empty[s]);   // K_j and V_j have no reader left
-                    if (more) issue_s(t, j + 1);
+                    if (t == n_q - 1) mma_commit(&v_empty[vs]);                        // V_j has no reader left
+                    if (more) {
+                        issue_s(t, j + 1);
+                        if (t == n_q - 1) mma_commit(&k_empty[(j + 1) % kKStages]);    // nor has K_{j+1}
+                    }
                 }
             }
             if (ok) mma_commit(o_done);
@@ -230,24 +315,28 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 ok = mbar_wait_warp(&s_full[t], j & 1, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
-                uint32_t sv[128];
+                const int cols_valid = n_keys - j * BKV;      // >= 1; < BKV only on a ragged last tile
+                // pass 1: row maximum, 32 columns at a time (the row is read again in pass 2 instead
+                // of being held in 128 registers)
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                 for (int cch = 0; cch < 4; ++cch) {
-                    uint32_t tmp[32];
-                    tmem_ld32(s_addr + cch * 32, tmp);
+                    uint32_t sv[32];
+                    tmem_ld32(s_addr + cch * 32, sv);
+                    tmem_ld_wait();
+                    if (cols_valid < BKV) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) sv[cch * 32 + i] = tmp[i];
+                        for (int i = 0; i < 32; ++i)
+                            if (cch * 32 + i >= cols_valid) sv[i] = 0xff800000u;   // -inf: key past the end
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+#pragma unroll
+                        for (int a = 0; a < 4; ++a)
+                            mx4[a] = fmax3(mx4[a], __uint_as_float(sv[i + 2 * a]), __uint_as_float(sv[i + 2 * a + 1]));
+                    }
                 }
-                tmem_ld_wait();
-                const int cols_valid = n_keys - j * BKV;      // >= 1
-                if (cols_valid < BKV) {
-#pragma unroll
-                    for (int i = 0; i < 128; ++i)
-                        if (i >= cols_valid) sv[i] = 0xff800000u;   // -inf: key past the end
-                }
-                float mx = __uint_as_float(sv[0]);
-#pragma unroll
-                for (int i = 1; i < 128; ++i) mx = fmaxf(mx, __uint_as_float(sv[i]));
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // raise the reference maximum only when it would change the exponent by > 2^8
                 const bool need = (mx - m_ref) * c > kRescaleThreshold;     // true on the first tile
                 if (__any_sync(0xffffffffu, need)) {
@@ -267,33 +356,55 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     l_run *= alpha;
                     m_ref = m_new;
                 }
-                const float m_scaled = m_ref * c;
-                float lsum0 = 0.f, lsum1 = 0.f;
-                uint32_t pk[64];
+                // pass 2: p = 2^(s*c - m*c). Of every four scores, two go through the special-function
+                // unit and two through the polynomial, which balances the two pipes. Each 32 scores
+                // become 16 registers of bf16 pairs, written over the first columns of S.
+                const uint64_t c2 = pack_f32x2(c, c);
+                const uint64_t nm2 = pack_f32x2(-m_ref * c, -m_ref * c);
+                uint64_t lsum_a = pack_f32x2(0.f, 0.f), lsum_b = lsum_a;
+                uint32_t sv[2][32];
+                tmem_ld32(s_addr, sv[0]);
 #pragma unroll
-                for (int i = 0; i < 64; ++i) {
-                    const float p0 = ex2(fmaf(__uint_as_float(sv[2 * i]), c, -m_scaled));
-                    const float p1 = ex2(fmaf(__uint_as_float(sv[2 * i + 1]), c, -m_scaled));
-                    lsum0 += p0;
-                    lsum1 += p1;
-                    pk[i] = pack_bf16(p0, p1);
+                for (int cch = 0; cch < 4; ++cch) {
+                    tmem_ld_wait();
+                    if (cch + 1 < 4) tmem_ld32(s_addr + (cch + 1) * 32, sv[(cch + 1) & 1]);   // in flight during the math
+                    uint32_t(&cur)[32] = sv[cch & 1];
+                    if (cols_valid < BKV) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (cch * 32 + i >= cols_valid) cur[i] = 0xff800000u;
+                    }
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        const uint64_t ya = fma_f32x2(pack_f32x2(__uint_as_float(cur[4 * g]), __uint_as_float(cur[4 * g + 1])), c2, nm2);
+                        const uint64_t yb = fma_f32x2(pack_f32x2(__uint_as_float(cur[4 * g + 2]), __uint_as_float(cur[4 * g + 3])), c2, nm2);
+                        float ya0, ya1, p0, p1, p2, p3;
+                        unpack_f32x2(ya, ya0, ya1);
+                        p0 = ex2(ya0);
+                        p1 = ex2(ya1);
+                        exp2_poly_x2(yb, p2, p3);
+                        lsum_a = add_f32x2(lsum_a, pack_f32x2(p0, p1));
+                        lsum_b = add_f32x2(lsum_b, pack_f32x2(p2, p3));
+                        pk[2 * g] = pack_bf16(p0, p1);
+                        pk[2 * g + 1] = pack_bf16(p2, p3);
+                    }
+                    // the S columns this overwrites (16*cch .. 16*cch+15) were read in an earlier
+                    // or the current chunk; the prefetched chunk starts at column 32*(cch+1)
+                    tmem_st16(s_addr + cch * 16, pk);
                 }
+                float lsum0, lsum1, lsum2, lsum3;
+                unpack_f32x2(lsum_a, lsum0, lsum1);
+                unpack_f32x2(lsum_b, lsum2, lsum3);
+                lsum0 += lsum2;
+                lsum1 += lsum3;
                 l_run += lsum0 + lsum1;
-                {
-                    uint32_t half[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) half[i] = pk[i];
-                    tmem_st32(s_addr, half);
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) half[i] = pk[32 + i];
-                    tmem_st32(s_addr + 32, half);
-                }
                 tmem_st_wait();
                 if (t == 0 && cols_valid < BKV) {
                     // ragged last tile: rows of V past the last key may hold anything (even NaN);
                     // zero them so that 0 * garbage cannot poison the accumulator
-                    const int s = j % kStages;
-                    ok = mbar_wait_warp(&v_full[s], (j / kStages) & 1, abort_flag, p.status);
+                    const int s = j % kVStages;
+                    ok = mbar_wait_warp(&v_full[s], (j / kVStages) & 1, abort_flag, p.status);
                     if (!ok) break;
                     if (row >= cols_valid) {
                         uint8_t* v_row = smem + L::kVOff + s * L::kTileBytes + row * 128;
