@@ -1,11 +1,12 @@
 // Eq. 4 / Eq. 7: per-token softmax entropy over the codebook logits and its per-image mean.
 //
-// One warp owns one row. The row is pulled from HBM exactly once with 128-bit loads and
-// held in registers; the warp takes the row maximum, then one pass of exp2 gives
-//   s = sum e^{z-m},  u = sum (z-m) e^{z-m},  H = ln s - u / s.
-// Rows too wide for the register file fall back to a two-read streaming kernel.
-// The mean is a second tiny kernel that sums in a fixed tree order (deterministic).
-#include "common.cuh"
+// One warp owns one row. The row is pulled from HBM exactly once and held packed in registers;
+// the warp takes the row maximum m, then one pass gives
+//   s = sum e^{z-m},  u = sum (z-m) e^{z-m},  H = ln s - u / s,
+// two logits per instruction (packed fp32). Rows of 2, 4 or 8 KiB (V = 4096 bf16 is 8 KiB) are
+// staged through a shared-memory ring by bulk copies in a persistent kernel that also takes the
+// per-image means; other shapes use one-warp-per-row kernels and a separate mean kernel.
+#include "tc_common.cuh"
 
 namespace {
 
@@ -47,7 +48,7 @@ __device__ __forceinline__ void unpack_bf16x2(uint32_t w, float& lo, float& hi)
     hi = __uint_as_float(w & 0xffff0000u);
 }
 
-// finishing step shared by both kernels: lane 0 writes the row result
+// finishing step shared by all kernels: lane 0 writes the row result
 __device__ __forceinline__ void finish_row(float m, float s, float u, float* ent, long row,
                                            unsigned int* status)
 {
@@ -62,46 +63,149 @@ __device__ __forceinline__ void finish_row(float m, float s, float u, float* ent
     ent[row] = h;
 }
 
-__device__ __forceinline__ float fmax_nan(float a, float b)   // NaN if either input is NaN
+// ---- two fp32 values per 64-bit register: one instruction does both lanes' arithmetic ----------
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
 {
-    float r;
-    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
     return r;
 }
 
-// Per-lane running state of the streaming softmax-entropy: m = largest logit seen, s = sum of
-// e^{z-m}, u = sum of (z-m) e^{z-m} (u kept in the log2 domain; m2 = m * log2 e). Raising m to m'
-// multiplies both sums by f = e^{m-m'} and shifts u by (m-m') s:  u' = f (u + (m-m') s),  s' = f s.
-struct RowState {
-    float m, m2, s, u;
-    __device__ __forceinline__ void raise_to(float m_new)
-    {
-        if (m == -INFINITY) { s = 0.f; u = 0.f; }
-        else {
-            const float shift = (m - m_new) * kLog2e;
-            const float f = fast_exp2(shift);
-            u = (u + shift * s) * f;
-            s *= f;
-        }
-        m = m_new;
-        m2 = m_new * kLog2e;
+// Exact two-pass evaluation of one row straight from global memory (the row is in L2): used for
+// rows that do not fit the register kernels and for the rare rows whose fast result is not
+// finite. -inf logits contribute 0; NaN or +inf logits leave m or s non-finite, which finish_row
+// reports. All 32 lanes of the warp call it together; every lane gets the row's m, s, u.
+template <bool BF16>
+__device__ __forceinline__ void entropy_row_exact(const char* base, int V, int lane, float& m, float& s, float& u)
+{
+    auto at = [&](int e) -> float {
+        return BF16 ? __bfloat162float(((const __nv_bfloat16*)base)[e]) : ((const float*)base)[e];
+    };
+    float mm = -INFINITY;
+    bool nan = false;
+    for (int e = lane; e < V; e += 32) {
+        const float z = at(e);
+        nan |= (z != z);
+        mm = fmaxf(mm, z);
     }
-    // One multiply-add, one clamp, one ex2, one add, one multiply-add per logit. The clamp turns a
-    // -inf (or NaN) exponent into a huge negative finite one whose ex2 is exactly 0, so that it
-    // contributes 0 instead of -inf * 0; NaN logits are caught by the NaN-propagating maximum.
-    __device__ __forceinline__ void add(float z)
-    {
-        const float d = fmaxf(fmaf(z, kLog2e, -m2), -16000.f);
-        const float e = fast_exp2(d);
-        s += e;
-        u = fmaf(d, e, u);
+    mm = warp_max(mm);
+    float ss = 0.f, uu = 0.f;
+    for (int e = lane; e < V; e += 32) {
+        const float d = (at(e) - mm) * kLog2e;
+        const float ex = fast_exp2(d);
+        ss += ex;
+        uu = fmaf(d == -INFINITY ? 0.f : d, ex, uu);
     }
-};
+    if (nan) ss = __int_as_float(0x7fc00000);
+    m = mm;
+    s = warp_sum(ss);
+    u = warp_sum(uu);
+}
 
-// VEC = number of 16-byte vectors each lane holds. BF16: 8 values per vector; F32: 4.
-// All loads of the row are issued before the first use (VEC * 16 bytes in flight per lane); the
-// values stay packed in registers and are consumed once, vector by vector, by the streaming
-// update above, so the register footprint is the packed row plus a handful of scalars.
+// Entropy sums of one row held as VEC packed 16-byte vectors per lane (BF16: 8 logits per vector,
+// F32: 4). First the row maximum m (packed bf16 maxima, then one warp reduction), then one
+// branch-free pass with, per pair of logits, two unpacks, one packed multiply-add
+// d = z * log2(e) - m * log2(e), two ex2, one packed add into s and one packed multiply-add into u
+// (u in the log2 domain), spread over independent accumulators. This pass handles finite logits
+// only: a -inf logit gives -inf * 0 = NaN in u, a NaN or +inf logit poisons m or s; any row whose
+// result is not finite is recomputed by entropy_row_exact, which treats every special value as
+// documented. On return every lane holds the row's m, s, u.
+template <int VEC, bool BF16>
+__device__ __forceinline__ void entropy_row_from_regs(const uint4 (&reg)[VEC], const char* base, int V, int lane,
+                                                      float& m_out, float& s_out, float& u_out)
+{
+    float m;
+    if (BF16) {
+        __nv_bfloat162 mx[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) mx[q] = *reinterpret_cast<const __nv_bfloat162*>(&(&reg[0].x)[q]);
+#pragma unroll
+        for (int i = 1; i < VEC; ++i) {
+            const uint32_t w[4] = {reg[i].x, reg[i].y, reg[i].z, reg[i].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) mx[q] = __hmax2(mx[q], *reinterpret_cast<const __nv_bfloat162*>(&w[q]));
+        }
+        const __nv_bfloat162 t = __hmax2(__hmax2(mx[0], mx[1]), __hmax2(mx[2], mx[3]));
+        float lo, hi;
+        unpack_bf16x2(*reinterpret_cast<const uint32_t*>(&t), lo, hi);
+        m = fmaxf(lo, hi);
+    } else {
+        float mx[4] = {__uint_as_float(reg[0].x), __uint_as_float(reg[0].y), __uint_as_float(reg[0].z), __uint_as_float(reg[0].w)};
+#pragma unroll
+        for (int i = 1; i < VEC; ++i) {
+            mx[0] = fmaxf(mx[0], __uint_as_float(reg[i].x));
+            mx[1] = fmaxf(mx[1], __uint_as_float(reg[i].y));
+            mx[2] = fmaxf(mx[2], __uint_as_float(reg[i].z));
+            mx[3] = fmaxf(mx[3], __uint_as_float(reg[i].w));
+        }
+        m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+    }
+    m = warp_max(m);
+
+    const uint64_t log2e2 = pack_f32x2(kLog2e, kLog2e);
+    const uint64_t neg_m2 = pack_f32x2(-m * kLog2e, -m * kLog2e);
+    uint64_t s2[4], u2[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) s2[a] = u2[a] = pack_f32x2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) {
+        const uint32_t w[4] = {reg[i].x, reg[i].y, reg[i].z, reg[i].w};
+        if (BF16) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float lo, hi;
+                unpack_bf16x2(w[q], lo, hi);
+                const uint64_t d2 = fma_f32x2(pack_f32x2(lo, hi), log2e2, neg_m2);
+                float d0, d1;
+                unpack_f32x2(d2, d0, d1);
+                const uint64_t e2 = pack_f32x2(fast_exp2(d0), fast_exp2(d1));
+                s2[q] = add_f32x2(s2[q], e2);
+                u2[q] = fma_f32x2(d2, e2, u2[q]);
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                const uint64_t d2 = fma_f32x2(pack_f32x2(__uint_as_float(w[2 * q]), __uint_as_float(w[2 * q + 1])), log2e2, neg_m2);
+                float d0, d1;
+                unpack_f32x2(d2, d0, d1);
+                const uint64_t e2 = pack_f32x2(fast_exp2(d0), fast_exp2(d1));
+                s2[2 * (i & 1) + q] = add_f32x2(s2[2 * (i & 1) + q], e2);
+                u2[2 * (i & 1) + q] = fma_f32x2(d2, e2, u2[2 * (i & 1) + q]);
+            }
+        }
+    }
+    const uint64_t st = add_f32x2(add_f32x2(s2[0], s2[1]), add_f32x2(s2[2], s2[3]));
+    const uint64_t ut = add_f32x2(add_f32x2(u2[0], u2[1]), add_f32x2(u2[2], u2[3]));
+    float s_lo, s_hi, u_lo, u_hi;
+    unpack_f32x2(st, s_lo, s_hi);
+    unpack_f32x2(ut, u_lo, u_hi);
+    float s = warp_sum(s_lo + s_hi);
+    float u = warp_sum(u_lo + u_hi);
+    const float h = logf(s) - (u / s) * kLn2;
+    // Anything unusual (-inf, +inf or NaN logits) shows up as a non-finite result and takes the
+    // exact path; the decision is the same in every lane.
+    if (!(fabsf(h) < INFINITY)) entropy_row_exact<BF16>(base, V, lane, m, s, u);
+    m_out = m; s_out = s; u_out = u;
+}
+
+// One warp per row, the row loaded straight into registers: all loads of the row are issued before
+// the first use (VEC * 16 bytes in flight per lane).
 template <int VEC, bool BF16>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 entropy_rows_reg(const void* __restrict__ logits, long rows, int V, long row_stride,
@@ -111,83 +215,153 @@ entropy_rows_reg(const void* __restrict__ logits, long rows, int V, long row_str
     const int lane = threadIdx.x & 31;
     const long row = (long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (row >= rows) return;
-    const int n_vec = V / PER;           // full vectors in the row (V % PER handled below)
+    const int n_vec = V / PER;
     const char* base = (const char*)logits + row * row_stride * (BF16 ? 2 : 4);
     const uint4* src = (const uint4*)base;
 
-    uint4 reg[VEC];
+    float m, s, u;
+    if (n_vec * PER != V || n_vec != VEC * 32) {
+        // the row does not fill the register tile exactly (same for every row of the launch)
+        entropy_row_exact<BF16>(base, V, lane, m, s, u);
+    } else {
+        uint4 reg[VEC];
 #pragma unroll
-    for (int i = 0; i < VEC; ++i) {
-        const int v = i * 32 + lane;
-        if (v < n_vec) reg[i] = ld_stream(src + v);
-        else reg[i] = BF16 ? make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u)   // -inf
-                           : make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
+        for (int i = 0; i < VEC; ++i) reg[i] = ld_stream(src + i * 32 + lane);
+        entropy_row_from_regs<VEC, BF16>(reg, base, V, lane, m, s, u);
     }
-    // ragged tail (V not a multiple of the vector width): lane t takes element n_vec*PER + t
-    float tail = -INFINITY;
-    {
-        const int e = n_vec * PER + lane;
-        if (e < V) {
-            tail = BF16 ? __bfloat162float(((const __nv_bfloat16*)base)[e]) : ((const float*)base)[e];
-        }
-    }
-
-    RowState st;
-    st.m = -INFINITY; st.m2 = -INFINITY; st.s = 0.f; st.u = 0.f;
-    bool saw_nan = false;
-#pragma unroll
-    for (int i = 0; i < VEC; ++i) {
-        const uint32_t w[4] = {reg[i].x, reg[i].y, reg[i].z, reg[i].w};
-        float cm;
-        if (BF16) {
-            // packed maximum: two logits per instruction
-            __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&w[0]);
-            __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&w[1]);
-            __nv_bfloat162 c = *reinterpret_cast<const __nv_bfloat162*>(&w[2]);
-            __nv_bfloat162 d = *reinterpret_cast<const __nv_bfloat162*>(&w[3]);
-            const __nv_bfloat162 mx = __hmax2_nan(__hmax2_nan(a, b), __hmax2_nan(c, d));
-            const uint32_t mw = *reinterpret_cast<const uint32_t*>(&mx);
-            float lo, hi;
-            unpack_bf16x2(mw, lo, hi);
-            cm = fmax_nan(lo, hi);
-        } else {
-            cm = fmax_nan(fmax_nan(__uint_as_float(w[0]), __uint_as_float(w[1])),
-                          fmax_nan(__uint_as_float(w[2]), __uint_as_float(w[3])));
-        }
-        saw_nan |= (cm != cm);
-        if (cm > st.m) st.raise_to(cm);             // rare after the first few vectors
-        if (st.m != -INFINITY) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if (BF16) {
-                    float lo, hi;
-                    unpack_bf16x2(w[q], lo, hi);
-                    st.add(lo);
-                    st.add(hi);
-                } else {
-                    st.add(__uint_as_float(w[q]));
-                }
-            }
-        }
-    }
-    saw_nan |= (tail != tail);
-    if (tail > st.m) st.raise_to(tail);
-    if (st.m != -INFINITY) st.add(tail);
-
-    // merge the 32 lanes: common maximum, then rescaled sums
-    const float m = warp_max(st.m);
-    float s = 0.f, u = 0.f;
-    if (st.m != -INFINITY) {
-        const float shift = (st.m - m) * kLog2e;
-        const float f = fast_exp2(shift);
-        s = st.s * f;
-        u = (st.u + shift * st.s) * f;
-        if (shift == -INFINITY) { s = 0.f; u = 0.f; }   // m = +inf: flagged below through m
-    }
-    if (saw_nan) s = __int_as_float(0x7fc00000);
-    s = warp_sum(s);
-    u = warp_sum(u);
     if (lane == 0) finish_row(m, s, u, ent, row, status);
+}
+
+// ---- persistent kernel: rows staged through a shared-memory ring by bulk copies ----------------
+// One CTA per SM. A producer thread keeps the ring's slots (whole rows) in flight with
+// cp.async.bulk, one copy per row, completion counted on an mbarrier; sixteen consumer warps take
+// rows from the ring in turn, move the row into registers, hand the slot back at once and then do
+// the arithmetic. HBM sees one deep, steady stream per SM instead of waves of CTAs that load, then
+// compute. The per-segment means are taken by whichever CTA finishes last (a counter in global
+// memory), always with the same summation tree, so the result does not depend on which CTA it is.
+constexpr int kRingConsumers = 16;
+constexpr int kRingThreads = (kRingConsumers + 1) * 32;
+constexpr int kRingBytes = 192 * 1024;
+
+// Bulk copy global -> shared of `bytes` (multiple of 16, both addresses 16-byte aligned).
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(tc::smem_u32(dst)), "l"(src), "r"(bytes), "r"(tc::smem_u32(bar)) : "memory");
+}
+
+template <int VEC, bool BF16>
+__global__ void __launch_bounds__(kRingThreads, 1)
+entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_stride_bytes,
+                  float* __restrict__ ent, float* __restrict__ mean, int seg_rows, int n_seg,
+                  unsigned int* status, unsigned int* done_counter)
+{
+    using namespace tc;
+    constexpr int kRowBytes = VEC * 512;
+    constexpr int kSlots = kRingBytes / kRowBytes;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* ring = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    uint64_t* full_bar = (uint64_t*)(ring + kSlots * kRowBytes);
+    uint64_t* empty_bar = full_bar + kSlots;
+    __shared__ int abort_flag_s;
+    __shared__ int is_last_s;
+    __shared__ float part[8][kRingThreads / 32];
+    volatile int* abort_flag = &abort_flag_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long G = gridDim.x;
+    const long n_my = (rows > blockIdx.x) ? (rows - blockIdx.x + G - 1) / G : 0;   // rows b, b+G, ...
+
+    if (threadIdx.x == 0) {
+        abort_flag_s = 0;
+        for (int i = 0; i < kSlots; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], 1);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    if (warp == kRingConsumers) {
+        if (lane == 0) {
+            long issued = 0;
+            for (long i = 0; i < n_my; ++i) {
+                const int slot = (int)(i % kSlots);
+                if (i >= kSlots && !mbar_wait(&empty_bar[slot], (uint32_t)((i / kSlots) - 1) & 1, abort_flag, status)) break;
+                const long row = blockIdx.x + i * G;
+                mbar_arrive_expect_tx(&full_bar[slot], kRowBytes);
+                bulk_load(ring + slot * kRowBytes, logits + row * row_stride_bytes, kRowBytes, &full_bar[slot]);
+                issued = i + 1;
+            }
+            if (*abort_flag)
+                for (long i = (issued > kSlots ? issued - kSlots : 0); i < issued; ++i)
+                    mbar_drain(&full_bar[i % kSlots], (uint32_t)(i / kSlots) & 1);
+        }
+    } else {
+        for (long i = warp; i < n_my; i += kRingConsumers) {
+            const int slot = (int)(i % kSlots);
+            if (!mbar_wait_warp(&full_bar[slot], (uint32_t)(i / kSlots) & 1, abort_flag, status)) break;
+            const uint4* src = (const uint4*)(ring + slot * kRowBytes);
+            uint4 reg[VEC];
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) reg[v] = src[v * 32 + lane];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[slot]);       // the row now lives in registers
+            const long row = blockIdx.x + i * G;
+            float m, s_sum, u;
+            entropy_row_from_regs<VEC, BF16>(reg, logits + row * row_stride_bytes, V, lane, m, s_sum, u);
+            if (lane == 0) finish_row(m, s_sum, u, ent, row, status);
+        }
+    }
+    if (!mean) return;
+
+    // ---- last CTA to finish takes the means ----------------------------------------------------
+    // Writers publish their entropies (fence) before the CTA's ticket is drawn; the last CTA reads
+    // them with L2 loads (ld.cg), so it needs no fence of its own.
+    if (lane == 0 && warp < kRingConsumers) __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int ticket = atomicAdd(done_counter, 1u);
+        is_last_s = (ticket == gridDim.x - 1);
+        if (is_last_s) *done_counter = 0;      // ready for the next launch
+    }
+    __syncthreads();
+    if (!is_last_s) return;
+    // Eight segments at a time: every thread first issues all its loads (thread t takes elements
+    // t, t + 544, ... of each segment), so the whole read costs about one L2 round trip; then one
+    // shuffle tree per segment, one exchange through shared memory, and warp g finishes segment g.
+    constexpr int kGroup = 8;
+    constexpr int kWarps = kRingThreads / 32;
+    for (int sg0 = 0; sg0 < n_seg; sg0 += kGroup) {
+        float acc[kGroup];
+#pragma unroll
+        for (int g = 0; g < kGroup; ++g) acc[g] = 0.f;
+#pragma unroll 2
+        for (int i0 = threadIdx.x; i0 < seg_rows; i0 += 4 * kRingThreads) {
+            float v[kGroup][4];
+#pragma unroll
+            for (int g = 0; g < kGroup; ++g)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int i = i0 + r * kRingThreads;
+                    v[g][r] = (sg0 + g < n_seg && i < seg_rows) ? __ldcg(ent + (long)(sg0 + g) * seg_rows + i) : 0.f;
+                }
+#pragma unroll
+            for (int g = 0; g < kGroup; ++g) acc[g] += (v[g][0] + v[g][1]) + (v[g][2] + v[g][3]);
+        }
+#pragma unroll
+        for (int g = 0; g < kGroup; ++g) {
+            const float w = warp_sum(acc[g]);
+            if (lane == 0) part[g][warp] = w;
+        }
+        __syncthreads();
+        if (warp < kGroup && sg0 + warp < n_seg) {
+            float v = (lane < kWarps) ? part[warp][lane] : 0.f;
+            v = warp_sum(v);
+            if (lane == 0) mean[sg0 + warp] = v / (float)seg_rows;
+        }
+        __syncthreads();
+    }
 }
 
 // Any V: two reads of the row (the second one is served by L1/L2).
@@ -200,21 +374,8 @@ entropy_rows_stream(const void* __restrict__ logits, long rows, int V, long row_
     const long row = (long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (row >= rows) return;
     const char* base = (const char*)logits + row * row_stride * (BF16 ? 2 : 4);
-    auto at = [&](int e) -> float {
-        return BF16 ? __bfloat162float(((const __nv_bfloat16*)base)[e]) : ((const float*)base)[e];
-    };
-    float m = -INFINITY;
-    for (int e = lane; e < V; e += 32) m = fmaxf(m, at(e));
-    m = warp_max(m);
-    float s = 0.f, u = 0.f;
-    for (int e = lane; e < V; e += 32) {
-        const float d = (at(e) - m) * kLog2e;
-        const float ex = fast_exp2(d);
-        s += ex;
-        u = fmaf(d == -INFINITY ? 0.f : d, ex, u);
-    }
-    s = warp_sum(s);
-    u = warp_sum(u);
+    float m, s, u;
+    entropy_row_exact<BF16>(base, V, lane, m, s, u);
     if (lane == 0) finish_row(m, s, u, ent, row, status);
 }
 
@@ -257,6 +418,25 @@ void launch_rows(const void* logits, long rows, int V, long row_stride, float* e
 #undef NOVA_ENT_CASE
 }
 
+template <int VEC, bool BF16>
+nova_status launch_ring(nova_ctx* ctx, const void* logits, long rows, int V, long stride_bytes, float* ent,
+                        float* mean, int N, int S, cudaStream_t st)
+{
+    constexpr int kSlots = kRingBytes / (VEC * 512);
+    const size_t smem = kRingBytes + 128 + 2 * sizeof(uint64_t) * kSlots;
+    static bool attr_done[64];
+    if (ctx->device < 64 && !attr_done[ctx->device]) {
+        NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(entropy_rows_ring<VEC, BF16>,
+                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_done[ctx->device] = true;
+    }
+    const int grid = (int)(rows < ctx->num_sms ? rows : ctx->num_sms);
+    entropy_rows_ring<VEC, BF16><<<grid, kRingThreads, smem, st>>>(
+        (const char*)logits, rows, V, stride_bytes, ent, mean, N, S, ctx->dev_status, ctx->dev_status + 1);
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    return NOVA_OK;
+}
+
 }  // namespace
 
 extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nova_dtype dt,
@@ -273,6 +453,20 @@ extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nov
     if (row_stride < V || (row_stride % per) != 0 || !nova_aligned16(logits))
         return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_scale_entropy: logits rows must start on 16-byte boundaries");
     cudaStream_t st = (cudaStream_t)stream;
+    const int elt = (dt == NOVA_BF16) ? 2 : 4;
+    const long row_bytes = (long)V * elt;
+    if ((row_bytes == 2048 || row_bytes == 4096 || row_bytes == 8192) && rows >= 64) {
+        // persistent ring kernel; the second word of the status allocation is its completion counter
+        const long stride_bytes = (long)row_stride * elt;
+        nova_launch_scope scope(ctx, NOVA_K_ENTROPY, st);
+        const bool bf = (dt == NOVA_BF16);
+        if (row_bytes == 2048) return bf ? launch_ring<4, true>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st)
+                                         : launch_ring<4, false>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st);
+        if (row_bytes == 4096) return bf ? launch_ring<8, true>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st)
+                                         : launch_ring<8, false>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st);
+        return bf ? launch_ring<16, true>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st)
+                  : launch_ring<16, false>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st);
+    }
     {
         nova_launch_scope scope(ctx, NOVA_K_ENTROPY, st);
         if (dt == NOVA_BF16) launch_rows<true>(logits, rows, V, row_stride, ent, ctx->dev_status, st);

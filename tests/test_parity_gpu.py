@@ -74,6 +74,46 @@ def test_entropy_matches_oracle(ctx, S, N, V, dtype):
         assert want_ent.max() - want_ent.min() > 2.0   # the field really spans low and high entropy
 
 
+@pytest.mark.parametrize("S,N,V,dtype", [
+    (3, 1500, 4096, torch.bfloat16),    # 4500 rows: every ring slot of the persistent kernel is reused
+    (2, 700, 2048, torch.bfloat16),     # 4 KiB rows
+    (1, 333, 1024, torch.bfloat16),     # 2 KiB rows
+    (2, 200, 2048, torch.float32),      # 8 KiB rows of fp32
+    (4, 4096, 4096, torch.bfloat16),    # the benchmark's launch: batch 4 at 64 x 64 tokens
+])
+def test_entropy_persistent_kernel_matches_oracle(ctx, S, N, V, dtype):
+    a = synth.smooth_temperature_field(S, 1, N, seed=9, device=DEV)
+    logits = synth.logits_from_temperature(a, V, seed=13, dtype=dtype)
+    ent, mean = gpu_entropy(ctx, logits)
+    want_ent, want_mean = oracle.scale_entropy(f32(logits))
+    assert np.abs(ent.cpu().numpy() - want_ent).max() <= ENT_TOL
+    assert np.abs(mean.cpu().numpy() - want_mean).max() <= ENT_TOL
+    # same launch again: the means come from whichever CTA finishes last, in a fixed order
+    ent2, mean2 = gpu_entropy(ctx, logits)
+    assert torch.equal(ent, ent2) and torch.equal(mean, mean2)
+    assert ctx.device_status() == 0
+
+
+def test_entropy_persistent_kernel_special_values(ctx):
+    V, N = 4096, 300
+    z = synth.randn_bf16((1, N, V), 21, DEV, std=2.0)
+    z[0, 7, 2048:] = float("-inf")                      # exact path: the finite half only
+    z[0, 100] = 0.25                                    # uniform -> ln V
+    z[0, 150, 5] = float("nan")
+    z[0, 299, 4095] = float("inf")
+    ent = torch.empty((1, N), dtype=torch.float32, device=DEV)
+    nova.nova_scale_entropy(ctx, z, ent, None)
+    e = ent.cpu().numpy()[0]
+    zz_ok = np.delete(f32(z), [150, 299], axis=1)
+    want, _ = oracle.scale_entropy(zz_ok)
+    got = np.delete(e, [150, 299])
+    assert np.abs(got - want[0]).max() <= ENT_TOL
+    assert abs(e[100] - math.log(V)) <= ENT_TOL
+    assert np.isnan(e[150]) and np.isnan(e[299])
+    assert ctx.device_status() == 5
+    assert ctx.device_status() == 0
+
+
 def test_entropy_ragged_v_and_row_stride(ctx):
     V, stride = 1003, 1008
     buf = torch.zeros((2, 6, stride), dtype=torch.bfloat16, device=DEV)
