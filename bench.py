@@ -197,7 +197,8 @@ def run_ours(args):
     for _ in range(args.warmup):
         one_step()
     barrier()
-    assert ctx.device_status() == 0, "device status after warm-up"
+    status = ctx.device_status()
+    assert status == 0, f"device status after warm-up: {nova.STATUS_NAMES.get(status, status)}"
 
     clocks = ClockSampler(local)
     launches0 = pipeline.launch_count(ctx)
@@ -219,7 +220,8 @@ def run_ours(args):
         total_ms = float(tt.item())
     ms_per_step = total_ms / args.steps
     value = world * B / (ms_per_step / 1e3)
-    assert ctx.device_status() == 0, "device status after the timed region"
+    status = ctx.device_status()
+    assert status == 0, f"device status after the timed region: {nova.STATUS_NAMES.get(status, status)}"
 
     # ---- rooflines from the events recorded around every launch inside the timed region. The two
     # contractions (the attention kernel and the GEMM kernel, four launches per layer) take about

@@ -233,15 +233,20 @@ entropy_rows_reg(const void* __restrict__ logits, long rows, int V, long row_str
 }
 
 // ---- persistent kernel: rows staged through a shared-memory ring by bulk copies ----------------
-// One CTA per SM. A producer thread keeps the ring's slots (whole rows) in flight with
+// One CTA per SM. A producer thread keeps the ring's slots (whole rows, 128 KB) in flight with
 // cp.async.bulk, one copy per row, completion counted on an mbarrier; sixteen consumer warps take
 // rows from the ring in turn, move the row into registers, hand the slot back at once and then do
 // the arithmetic. HBM sees one deep, steady stream per SM instead of waves of CTAs that load, then
 // compute. The per-segment means are taken by whichever CTA finishes last (a counter in global
 // memory), always with the same summation tree, so the result does not depend on which CTA it is.
+// Row i of a CTA goes to slot i % kSlots and to consumer warp i % 16; kSlots is a multiple of 16, so
+// every use of a slot is consumed by the same warp, in order. That matters: a parity wait for use
+// n of a slot succeeds at once while use n-1 has not completed yet, and bulk copies may land out of
+// order (a copy that misses the TLB can trail later ones by microseconds), so a warp must never
+// poll a slot whose previous use some other warp has yet to see.
 constexpr int kRingConsumers = 16;
 constexpr int kRingThreads = (kRingConsumers + 1) * 32;
-constexpr int kRingBytes = 192 * 1024;
+constexpr int kRingBytes = 128 * 1024;
 
 // Bulk copy global -> shared of `bytes` (multiple of 16, both addresses 16-byte aligned).
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
@@ -259,6 +264,7 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
     using namespace tc;
     constexpr int kRowBytes = VEC * 512;
     constexpr int kSlots = kRingBytes / kRowBytes;
+    static_assert(kSlots % kRingConsumers == 0, "each slot must belong to one consumer warp");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* ring = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     uint64_t* full_bar = (uint64_t*)(ring + kSlots * kRowBytes);
