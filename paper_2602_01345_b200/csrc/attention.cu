@@ -51,7 +51,7 @@ struct AttnParams {
     const int32_t* cu_keep;
     const int32_t* kv_len;
     __nv_bfloat16* o;
-    int B, C, Lmax;
+    int B, C, Lmax, n_heads, num_sms;
     float scale_log2e;     // (1 / sqrt(dh)) * log2(e)
     unsigned int* status;
 };
@@ -147,20 +147,40 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     // S tile t (fp32) sits at column 128*t; its first 64 columns are reused for P (bf16 pairs).
     // O tile t (fp32, DH columns) sits at column 256 + 128*t.
 
-    // ---- which (image, 256-row query block) is this CTA? -----------------------------
-    int slot = blockIdx.x, b = 0, k_b = 0, q_begin = 0;
-    bool found = false;
+    // ---- which (image, 256-row query block, head) is this CTA? ----------------------------
+    // Work items are (head, query block), blocks fastest so that CTAs running together share K/V
+    // in L2. All items cost the same, so a grid of T items runs in ceil(T / SMs) waves and the last
+    // wave may be nearly empty: when it would fill at most half of the SMs, its items are split
+    // into their two 128-row tiles, each run by a CTA of its own (one tile, no ping-pong), which
+    // cuts the last wave to roughly 60 % of a full one.
+    int units = 0;
+    for (int i = 0; i < p.B; ++i) units += (p.cu_keep[i + 1] - p.cu_keep[i] + 2 * BQ - 1) / (2 * BQ);
+    const int items = units * p.n_heads;
+    const int rem = items % p.num_sms;
+    const int whole_items = (rem > 0 && 2 * rem <= p.num_sms) ? items - rem : items;
+    int item = blockIdx.x, half = -1;
+    if (item >= whole_items) {
+        const int h = item - whole_items;
+        item = whole_items + (h >> 1);
+        half = h & 1;
+    }
+    if (item >= items) return;
+    const int head = item / units;
+    int slot = item - head * units, b = 0, k_b = 0, q_begin = 0;
     for (b = 0; b < p.B; ++b) {
         const int c0 = p.cu_keep[b];
         k_b = p.cu_keep[b + 1] - c0;
         const int blocks = (k_b + 2 * BQ - 1) / (2 * BQ);
-        if (slot < blocks) { q_begin = c0 + slot * 2 * BQ; found = true; break; }
+        if (slot < blocks) { q_begin = c0 + slot * 2 * BQ; break; }
         slot -= blocks;
     }
-    if (!found) return;
-    const int rows_valid = min(2 * BQ, k_b - slot * 2 * BQ);
+    int rows_valid = min(2 * BQ, k_b - slot * 2 * BQ);
+    if (half >= 0) {
+        q_begin += half * BQ;
+        rows_valid = min(BQ, rows_valid - half * BQ);
+        if (rows_valid <= 0) return;
+    }
     const bool tile_b_active = rows_valid > BQ;
-    const int head = blockIdx.y;
     const int n_keys = min(p.kv_len[b] + k_b, p.Lmax);
     const int n_tiles = (n_keys + BKV - 1) / BKV;
 
@@ -242,23 +262,27 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
-            constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
-            const int n_q = tile_b_active ? 2 : 1;
-            // Shared-memory descriptors are split into a constant high word and a low word that
-            // holds (address >> 4) in its low 14 bits, so stepping through a tile is one integer
-            // add per operand: the issuing thread has about 64 clocks per instruction to stay
-            // ahead of the tensor core.
-            const uint64_t q_desc = smem_desc_sw128(smem_u32(q_smem), 16, 1024);
-            const uint64_t k_desc = smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024);
-            const uint64_t v_desc = smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024);
-            constexpr uint32_t kTileStep = L::kTileBytes >> 4;
-            bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
-            // S_t = Q_t K_j^T
-            auto issue_s = [&](int t, int j) {
-                const uint64_t qd = q_desc + (uint32_t)t * kTileStep;
-                const uint64_t kd = k_desc + (uint32_t)(j % kKStages) * kTileStep;
+        // The whole warp runs this loop in lockstep and one lane issues. Control flow, stage
+        // counters and descriptors are then warp-uniform by construction, which lets the compiler
+        // keep the operands of tcgen05.mma where the instruction takes them from (uniform
+        // registers) instead of moving them there before every issue from a diverged thread; the
+        // tensor core executes an instruction every 64 clocks and accepts them hardly faster, so
+        // every clock of issue overhead is a clock of tensor-core idle time.
+        constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
+        constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
+        const int n_q = tile_b_active ? 2 : 1;
+        // Shared-memory descriptors: (address >> 4) sits in the low 14 bits, so stepping through
+        // a tile or to another stage is an integer add.
+        constexpr uint32_t kTileStep = L::kTileBytes >> 4;
+        const uint64_t q_desc = smem_desc_sw128(smem_u32(q_smem), 16, 1024);
+        const uint64_t k_desc = smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024);
+        const uint64_t v_desc = smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024);
+        const bool issuer = (lane == 0);
+        // S_t = Q_t K^T with K in stage ks
+        auto issue_s = [&](int t, int ks) {
+            const uint64_t qd = q_desc + (uint32_t)t * kTileStep;
+            const uint64_t kd = k_desc + (uint32_t)ks * kTileStep;
+            if (issuer) {
 #pragma unroll
                 for (int kk = 0; kk < DH / 16; ++kk) {
                     constexpr uint32_t kSlabStep = kSlabBytes >> 4;
@@ -266,40 +290,57 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     mma_bf16_ss(tmem_base + 128u * t, qd + off, kd + off, idesc_s, kk ? 1u : 0u);
                 }
                 mma_commit(&s_full[t]);
-            };
-            // O_t (+)= P_t V_j ; P_t sits in the first 64 columns of S_t, two keys per column
-            auto issue_pv = [&](int t, int j) {
-                const uint64_t vd = v_desc + (uint32_t)(j % kVStages) * kTileStep;
+            }
+            __syncwarp();
+        };
+        // O_t (+)= P_t V with V in stage vs; P_t sits in the first 64 columns of S_t, two keys per column
+        auto issue_pv = [&](int t, int vs, bool first) {
+            const uint64_t vd = v_desc + (uint32_t)vs * kTileStep;
+            if (issuer) {
 #pragma unroll
                 for (int kk = 0; kk < BKV / 16; ++kk)
                     mma_bf16_ts(tmem_base + 256u + 128u * t, tmem_base + 128u * t + kk * 8, vd + (uint32_t)(kk * 128),
-                                idesc_o, (j | kk) ? 1u : 0u);
-            };
-            if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag, p.status);
-            if (ok) {
-                tc_fence_after();
-                for (int t = 0; t < n_q; ++t) issue_s(t, 0);
-                mma_commit(&k_empty[0]);
+                                idesc_o, (first && kk == 0) ? 0u : 1u);
             }
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int vs = j % kVStages;
-                const bool more = j + 1 < n_tiles;
-                ok = mbar_wait(&v_full[vs], (j / kVStages) & 1, abort_flag, p.status);
-                if (ok && more) ok = mbar_wait(&k_full[(j + 1) % kKStages], ((j + 1) / kKStages) & 1, abort_flag, p.status);
-                for (int t = 0; t < n_q && ok; ++t) {
-                    ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(t, j);
-                    if (t == n_q - 1) mma_commit(&v_empty[vs]);                        // V_j has no reader left
-                    if (more) {
-                        issue_s(t, j + 1);
-                        if (t == n_q - 1) mma_commit(&k_empty[(j + 1) % kKStages]);    // nor has K_{j+1}
+            __syncwarp();
+        };
+        bool ok = mbar_wait_warp(q_full, 0, abort_flag, p.status);
+        if (ok) ok = mbar_wait_warp(&k_full[0], 0, abort_flag, p.status);
+        if (ok) {
+            tc_fence_after();
+            for (int t = 0; t < n_q; ++t) issue_s(t, 0);
+            if (issuer) mma_commit(&k_empty[0]);
+            __syncwarp();
+        }
+        // ring positions and phase parities, stepped without divisions
+        int vs = 0, ks_next = (kKStages > 1) ? 1 : 0;
+        uint32_t v_par = 0, k_par_next = (kKStages > 1) ? 0u : 1u;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const bool more = j + 1 < n_tiles;
+            ok = mbar_wait_warp(&v_full[vs], v_par, abort_flag, p.status);
+            if (ok && more) ok = mbar_wait_warp(&k_full[ks_next], k_par_next, abort_flag, p.status);
+            for (int t = 0; t < n_q && ok; ++t) {
+                ok = mbar_wait_warp(&p_full[t], j & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                issue_pv(t, vs, j == 0);
+                if (t == n_q - 1) {
+                    if (issuer) mma_commit(&v_empty[vs]);                 // V_j has no reader left
+                    __syncwarp();
+                }
+                if (more) {
+                    issue_s(t, ks_next);
+                    if (t == n_q - 1) {
+                        if (issuer) mma_commit(&k_empty[ks_next]);        // nor has K_{j+1}
+                        __syncwarp();
                     }
                 }
             }
-            if (ok) mma_commit(o_done);
+            if (++vs == kVStages) { vs = 0; v_par ^= 1u; }
+            if (++ks_next == kKStages) { ks_next = 0; k_par_next ^= 1u; }
         }
+        if (ok && issuer) mma_commit(o_done);
+        __syncwarp();
     } else {
         const int t = (warp >= 6) ? 1 : 0;            // which query tile this warpgroup owns
         if (t == 0 || tile_b_active) {
@@ -472,7 +513,10 @@ nova_status launch(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st)
     p.cu_keep = a.cu_keep; p.kv_len = a.kv_len; p.o = a.o; p.B = a.B; p.C = a.C; p.Lmax = a.Lmax;
     p.scale_log2e = (float)((1.0 / sqrt((double)DH)) * 1.4426950408889634);
     p.status = ctx->dev_status;
-    dim3 grid((a.M + 2 * BQ - 1) / (2 * BQ) + a.B, a.n_heads);
+    p.n_heads = a.n_heads; p.num_sms = ctx->num_sms;
+    // upper bound of the work items (the kept counts per image live on the device) plus the CTAs a
+    // split last wave adds; CTAs past the end return at once
+    dim3 grid(((a.M + 2 * BQ - 1) / (2 * BQ) + a.B) * a.n_heads + ctx->num_sms / 2);
     {
         nova_launch_scope scope(ctx, NOVA_K_ATTENTION, st);
         kern<<<grid, kThreads, L::kTotal, st>>>(tq, tk, tv, p);

@@ -361,6 +361,19 @@ def test_block_full_size_1024_shape_sampled_rows(ctx):
                 rows=np.array(rows, np.int32))
 
 
+def test_block_attention_ragged_mid_size(ctx):
+    """Thousands of kept rows per image at head size 128, with keep counts and cache lengths that
+    leave partial 256-row query blocks, blocks with only one of the two query tiles in use, and
+    ragged last key tiles. K/V appends are compared for every row, the block output on sampled
+    rows around the tile and block boundaries."""
+    ks = [7000, 6013, 6100 + 260]
+    M = sum(ks)
+    rows = [0, 127, 128, 255, 256, 511, 512, 6999, 7000, 7000 + 6012, 7000 + 6013, 7000 + 6013 + 6143,
+            7000 + 6013 + 6144, M - 1]
+    _block_case(ctx, B=3, N=8192, C=256, heads=2, F=512, Lmax=9000, ks=ks, kv_lens=[300, 5, 129], seed=17,
+                rows=np.array(rows, np.int32))
+
+
 def test_block_without_append_leaves_kv_len(ctx):
     B, N, C, heads, F, Lmax = 1, 64, 128, 2, 256, 256
     wt = synth.block_weights(C, F, 1, DEV)
