@@ -7,8 +7,8 @@
 //   warp 1        tcgen05.mma issuer. Per key tile j:  O_A += P_A V_j ; S_A = Q_A K_{j+1}^T ;
 //                 O_B += P_B V_j ; S_B = Q_B K_{j+1}^T.  S and O are fp32 in tensor memory and
 //                 O accumulates there across all key tiles.
-//   warps 2-5     softmax of tile A, one query row per thread: read the row of S from tensor
-//   warps 6-9     memory once, probabilities P = 2^((s - m) * scale) packed to bf16 and stored
+//   warps 4-7     softmax of tile A, one query row per thread: read the row of S from tensor
+//   warps 8-11    memory once, probabilities P = 2^((s - m) * scale) packed to bf16 and stored
 //   (tile B)      back into tensor memory over the S columns, from where the next MMA takes them
 //                 as its A operand. While one tile's softmax runs, the tensor core works on the
 //                 other tile.
@@ -27,7 +27,8 @@ using namespace tc;
 
 constexpr int BQ = 128;        // query rows per tile (two tiles per CTA)
 constexpr int BKV = 128;       // keys per tile
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;     // warpgroup 0: producer + MMA issuer (+2 idle warps); 1, 2: softmax of tile A, B
+constexpr int kRegsLow = 56, kRegsHigh = 216;   // 128 * 56 + 256 * 216 <= 64 K registers
 constexpr int kSlabBytes = 128 * 128;   // [128 rows][64 bf16]
 constexpr float kRescaleThreshold = 8.f;   // in log2 units
 
@@ -230,6 +231,11 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
     uint8_t* q_smem = smem + L::kQOff;
 
+    // The softmax warps hold a whole 128-column row of S in registers; the producer and the MMA
+    // issuer need few. Each warpgroup resizes its share of the register file accordingly (the
+    // resize must dominate all of the role's code, hence the nesting).
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLow));
     if (warp == 0) {
         if (lane == 0) {
             const int q_tiles = tile_b_active ? 2 : 1;
@@ -341,8 +347,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         }
         if (ok && issuer) mma_commit(o_done);
         __syncwarp();
+    }
     } else {
-        const int t = (warp >= 6) ? 1 : 0;            // which query tile this warpgroup owns
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsHigh));
+        const int t = (warp >= 8) ? 1 : 0;            // which query tile this warpgroup owns
         if (t == 0 || tile_b_active) {
             const int q = warp & 3;
             const int row = q * 32 + lane;               // row within the tile = TMEM lane
@@ -357,25 +365,23 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
                 const int cols_valid = n_keys - j * BKV;      // >= 1; < BKV only on a ragged last tile
-                // pass 1: row maximum, 32 columns at a time (the row is read again in pass 2 instead
-                // of being held in 128 registers)
+                // the whole row of S (128 scores) into registers with one round trip to tensor memory
+                uint32_t sv[128];
+#pragma unroll
+                for (int cch = 0; cch < 4; ++cch)
+                    tmem_ld32(s_addr + cch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[cch * 32]));
+                tmem_ld_wait();
+                if (cols_valid < BKV) {
+#pragma unroll
+                    for (int i = 0; i < 128; ++i)
+                        if (i >= cols_valid) sv[i] = 0xff800000u;   // -inf: key past the end
+                }
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int cch = 0; cch < 4; ++cch) {
-                    uint32_t sv[32];
-                    tmem_ld32(s_addr + cch * 32, sv);
-                    tmem_ld_wait();
-                    if (cols_valid < BKV) {
+                for (int i = 0; i < 128; i += 8) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (cch * 32 + i >= cols_valid) sv[i] = 0xff800000u;   // -inf: key past the end
-                    }
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-#pragma unroll
-                        for (int a = 0; a < 4; ++a)
-                            mx4[a] = fmax3(mx4[a], __uint_as_float(sv[i + 2 * a]), __uint_as_float(sv[i + 2 * a + 1]));
-                    }
+                    for (int a = 0; a < 4; ++a)
+                        mx4[a] = fmax3(mx4[a], __uint_as_float(sv[i + 2 * a]), __uint_as_float(sv[i + 2 * a + 1]));
                 }
                 const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // raise the reference maximum only when it would change the exponent by > 2^8
@@ -397,29 +403,20 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     l_run *= alpha;
                     m_ref = m_new;
                 }
-                // pass 2: p = 2^(s*c - m*c). Of every four scores, two go through the special-function
-                // unit and two through the polynomial, which balances the two pipes. Each 32 scores
+                // p = 2^(s*c - m*c). Of every four scores, two go through the special-function unit
+                // and two through the polynomial, which balances the two pipes. Each 32 scores
                 // become 16 registers of bf16 pairs, written over the first columns of S.
                 const uint64_t c2 = pack_f32x2(c, c);
                 const uint64_t nm2 = pack_f32x2(-m_ref * c, -m_ref * c);
                 uint64_t lsum_a = pack_f32x2(0.f, 0.f), lsum_b = lsum_a;
-                uint32_t sv[2][32];
-                tmem_ld32(s_addr, sv[0]);
 #pragma unroll
                 for (int cch = 0; cch < 4; ++cch) {
-                    tmem_ld_wait();
-                    if (cch + 1 < 4) tmem_ld32(s_addr + (cch + 1) * 32, sv[(cch + 1) & 1]);   // in flight during the math
-                    uint32_t(&cur)[32] = sv[cch & 1];
-                    if (cols_valid < BKV) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (cch * 32 + i >= cols_valid) cur[i] = 0xff800000u;
-                    }
                     uint32_t pk[16];
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
-                        const uint64_t ya = fma_f32x2(pack_f32x2(__uint_as_float(cur[4 * g]), __uint_as_float(cur[4 * g + 1])), c2, nm2);
-                        const uint64_t yb = fma_f32x2(pack_f32x2(__uint_as_float(cur[4 * g + 2]), __uint_as_float(cur[4 * g + 3])), c2, nm2);
+                        const int i = cch * 32 + 4 * g;
+                        const uint64_t ya = fma_f32x2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2, nm2);
+                        const uint64_t yb = fma_f32x2(pack_f32x2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), c2, nm2);
                         float ya0, ya1, p0, p1, p2, p3;
                         unpack_f32x2(ya, ya0, ya1);
                         p0 = ex2(ya0);
@@ -430,8 +427,6 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         pk[2 * g] = pack_bf16(p0, p1);
                         pk[2 * g + 1] = pack_bf16(p2, p3);
                     }
-                    // the S columns this overwrites (16*cch .. 16*cch+15) were read in an earlier
-                    // or the current chunk; the prefetched chunk starts at column 32*(cch+1)
                     tmem_st16(s_addr + cch * 16, pk);
                 }
                 float lsum0, lsum1, lsum2, lsum3;
