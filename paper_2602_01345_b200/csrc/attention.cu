@@ -28,7 +28,7 @@ using namespace tc;
 constexpr int BQ = 128;        // query rows per tile (two tiles per CTA)
 constexpr int BKV = 128;       // keys per tile
 constexpr int kThreads = 384;     // warpgroup 0: producer + MMA issuer (+2 idle warps); 1, 2: softmax of tile A, B
-constexpr int kRegsLow = 56, kRegsHigh = 216;   // 128 * 56 + 256 * 216 <= 64 K registers
+constexpr int kRegsLow = 64, kRegsHigh = 216;   // 128 * 64 + 256 * 216 <= 64 K registers
 constexpr int kSlabBytes = 128 * 128;   // [128 rows][64 bf16]
 constexpr float kRescaleThreshold = 8.f;   // in log2 units
 
@@ -276,13 +276,23 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         // every clock of issue overhead is a clock of tensor-core idle time.
         constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
         constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
-        const int n_q = tile_b_active ? 2 : 1;
         // Shared-memory descriptors: (address >> 4) sits in the low 14 bits, so stepping through
         // a tile or to another stage is an integer add.
+        // tcgen05.mma takes its descriptors and addresses from uniform registers. Everything
+        // they are built from is broadcast from lane 0 once, which tells the compiler that the
+        // values are warp-uniform, so the per-instruction address arithmetic stays in the uniform
+        // datapath instead of being moved there from a lane's registers before every issue.
         constexpr uint32_t kTileStep = L::kTileBytes >> 4;
-        const uint64_t q_desc = smem_desc_sw128(smem_u32(q_smem), 16, 1024);
-        const uint64_t k_desc = smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024);
-        const uint64_t v_desc = smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024);
+        auto uniform32 = [](uint32_t v) { return __shfl_sync(0xffffffffu, v, 0); };
+        auto uniform64 = [&](uint64_t v) {
+            return ((uint64_t)uniform32((uint32_t)(v >> 32)) << 32) | uniform32((uint32_t)v);
+        };
+        const uint64_t q_desc = uniform64(smem_desc_sw128(smem_u32(q_smem), 16, 1024));
+        const uint64_t k_desc = uniform64(smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024));
+        const uint64_t v_desc = uniform64(smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024));
+        const uint32_t tmem_u = uniform32(tmem_base);
+        const int n_tiles_u = (int)uniform32((uint32_t)n_tiles);     // loop bounds too: uniform control flow
+        const int n_q = (int)uniform32(tile_b_active ? 2u : 1u);
         const bool issuer = (lane == 0);
         // S_t = Q_t K^T with K in stage ks
         auto issue_s = [&](int t, int ks) {
@@ -293,7 +303,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 for (int kk = 0; kk < DH / 16; ++kk) {
                     constexpr uint32_t kSlabStep = kSlabBytes >> 4;
                     const uint32_t off = (kk >> 2) * kSlabStep + (kk & 3) * 2;    // 32 bytes per 16 k
-                    mma_bf16_ss(tmem_base + 128u * t, qd + off, kd + off, idesc_s, kk ? 1u : 0u);
+                    mma_bf16_ss(tmem_u + 128u * t, qd + off, kd + off, idesc_s, kk ? 1u : 0u);
                 }
                 mma_commit(&s_full[t]);
             }
@@ -305,7 +315,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             if (issuer) {
 #pragma unroll
                 for (int kk = 0; kk < BKV / 16; ++kk)
-                    mma_bf16_ts(tmem_base + 256u + 128u * t, tmem_base + 128u * t + kk * 8, vd + (uint32_t)(kk * 128),
+                    mma_bf16_ts(tmem_u + 256u + 128u * t, tmem_u + 128u * t + kk * 8, vd + (uint32_t)(kk * 128),
                                 idesc_o, (first && kk == 0) ? 0u : 1u);
             }
             __syncwarp();
@@ -321,8 +331,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         // ring positions and phase parities, stepped without divisions
         int vs = 0, ks_next = (kKStages > 1) ? 1 : 0;
         uint32_t v_par = 0, k_par_next = (kKStages > 1) ? 0u : 1u;
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            const bool more = j + 1 < n_tiles;
+        for (int j = 0; j < n_tiles_u && ok; ++j) {
+            const bool more = j + 1 < n_tiles_u;
             ok = mbar_wait_warp(&v_full[vs], v_par, abort_flag, p.status);
             if (ok && more) ok = mbar_wait_warp(&k_full[ks_next], k_par_next, abort_flag, p.status);
             for (int t = 0; t < n_q && ok; ++t) {
