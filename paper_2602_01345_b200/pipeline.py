@@ -1,6 +1,6 @@
 """One accelerated scale through all layers: the call sequence a user of the library makes.
 
-For every layer j of the scale: entropy of the layer's logits -> (means to the host) ->
+Entropy of every layer's logits -> (all means to the host in one copy) -> then for every layer j:
 keep counts from the trigger/ratio functions -> top-k selection -> block on the kept rows
 -> restore of the pruned rows from the residual cache. This module only owns buffers and
 issues the five C-ABI calls in order; it computes nothing itself.
@@ -36,9 +36,9 @@ class PrunedScaleRunner:
         dev = weights[0]["w_o"].device
         self.dev = dev
         N, Cc = self.N, self.C
-        self.ent = torch.empty((B, N), dtype=torch.float32, device=dev)
-        self.mean = torch.empty((B,), dtype=torch.float32, device=dev)
-        self.mean_host = torch.empty((B,), dtype=torch.float32).pin_memory()
+        self.ent = torch.empty((self.L, B, N), dtype=torch.float32, device=dev)
+        self.mean = torch.empty((self.L, B), dtype=torch.float32, device=dev)
+        self.mean_host = torch.empty((self.L, B), dtype=torch.float32).pin_memory()
         self.keep_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
         self.prune_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
         self.cu_keep = torch.empty((B + 1,), dtype=torch.int32, device=dev)
@@ -58,31 +58,40 @@ class PrunedScaleRunner:
         """
         ctx, B, N = self.ctx, self.B, self.N
         st = stream if stream is not None else torch.cuda.current_stream()
+        # The layers' logits are inputs of the scale, not results of its layers, so the entropy maps
+        # of a whole group of layers are taken first and their means cross to the host in one copy:
+        # one synchronisation per group decides the keep counts of all its layers. With resident
+        # logits the group is the whole scale; while logits are still being uploaded a small group
+        # lets the blocks of the first layers run under the uploads of the later ones.
+        group = self.L if logits_ready is None else min(self.L, 4)
         hbar_layer = torch.empty((B, self.L), dtype=torch.float32)
         keeps = []
         x = x_in
-        for j in range(self.L):
-            if logits_ready is not None:
-                st.wait_event(logits_ready[j])
-            nv.nova_scale_entropy(ctx, layer_logits[j], self.ent, self.mean, stream=st)
-            self.mean_host.copy_(self.mean, non_blocking=True)
-            st.synchronize()                                    # the keep count is decided on the host
-            hbar_layer[:, j] = self.mean_host
-            r = nv.nova_keep_ratios(sched, t, j + 1, N, hbar_scale, hbar_layer[:, : j + 1].contiguous())
-            keep = r["keep"]
-            M = int(keep.sum())
-            keeps.append(keep)
-            nv.nova_select_topk(ctx, self.ent, keep, self.keep_idx[:M], self.prune_idx[: B * N - M], self.cu_keep,
-                                None, stream=st)
-            shape = nv.BlockShape(B, N, self.C, self.n_heads, self.F, self.Lmax, M)
-            nv.nova_pruned_block_forward(ctx, self.weights[j], shape, x, self.keep_idx[:M], self.cu_keep,
-                                         self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
-                                         self.y_kept[:M], stream=st)
-            x_out = self.x_buf[j & 1] if x is not self.x_buf[j & 1] else self.x_buf[(j + 1) & 1]
-            nv.nova_restore_from_cache(ctx, x, self.y_kept[:M], self.keep_idx[:M], self.prune_idx[: B * N - M],
-                                       self.cu_keep, self.cache_prev[j], self.h, self.w, x_out,
-                                       self.cache_out[j] if self.cache_out is not None else None, stream=st)
-            x = x_out
+        for g0 in range(0, self.L, group):
+            g1 = min(self.L, g0 + group)
+            for j in range(g0, g1):
+                if logits_ready is not None:
+                    st.wait_event(logits_ready[j])
+                nv.nova_scale_entropy(ctx, layer_logits[j], self.ent[j], self.mean[j], stream=st)
+            self.mean_host[g0:g1].copy_(self.mean[g0:g1], non_blocking=True)
+            st.synchronize()
+            hbar_layer[:, g0:g1] = self.mean_host[g0:g1].t()
+            for j in range(g0, g1):
+                r = nv.nova_keep_ratios(sched, t, j + 1, N, hbar_scale, hbar_layer[:, : j + 1].contiguous())
+                keep = r["keep"]
+                M = int(keep.sum())
+                keeps.append(keep)
+                nv.nova_select_topk(ctx, self.ent[j], keep, self.keep_idx[:M], self.prune_idx[: B * N - M],
+                                    self.cu_keep, None, stream=st)
+                shape = nv.BlockShape(B, N, self.C, self.n_heads, self.F, self.Lmax, M)
+                nv.nova_pruned_block_forward(ctx, self.weights[j], shape, x, self.keep_idx[:M], self.cu_keep,
+                                             self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
+                                             self.y_kept[:M], stream=st)
+                x_out = self.x_buf[j & 1] if x is not self.x_buf[j & 1] else self.x_buf[(j + 1) & 1]
+                nv.nova_restore_from_cache(ctx, x, self.y_kept[:M], self.keep_idx[:M], self.prune_idx[: B * N - M],
+                                           self.cu_keep, self.cache_prev[j], self.h, self.w, x_out,
+                                           self.cache_out[j] if self.cache_out is not None else None, stream=st)
+                x = x_out
         self.last_keep = keeps
         return x, keeps
 
