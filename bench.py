@@ -160,6 +160,24 @@ def peaks():
         return dict(hbm=6650.0, tensor=1400.0, source="fallback")
 
 
+# ------------------------------------------------------------------- replicas (N > 1)
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The job's time is the slowest rank's: all-reduce MAX of the per-rank device time. With
+    dist None (one process) the value passes through."""
+    if dist is None:
+        return float(ms)
+    tt = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def replica_throughput(world: int, units_per_rank: float, ms_per_step: float) -> float:
+    """Whole-job throughput of `world` independent replicas (images are independent: no data-path
+    collective; weak scaling): every rank processes units_per_rank per step, the step lasts as
+    long as the slowest rank."""
+    return world * units_per_rank / (ms_per_step / 1e3)
+
+
 # ------------------------------------------------------------------------------ ours
 def run_ours(args):
     import paper_2602_01345_b200 as nova
@@ -214,12 +232,9 @@ def run_ours(args):
     prof = pipeline.profile_end(ctx)
     launches = pipeline.launch_count(ctx) - launches0
     clk = clocks.stop()
-    if dist is not None:
-        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * B / (ms_per_step / 1e3)
+    value = replica_throughput(world, B, ms_per_step)
     status = ctx.device_status()
     assert status == 0, f"device status after the timed region: {nova.STATUS_NAMES.get(status, status)}"
 
@@ -349,10 +364,7 @@ def run_e2e(args, wd, st, runner, sched, hbar_scale, barrier, dist, dev, world):
     wall_ms = (time.perf_counter() - t0) * 1e3
     dev_ms = e0.elapsed_time(e1)
     t_ms = max(wall_ms, dev_ms)
-    if dist is not None:
-        tt = torch.tensor([t_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t_ms = float(tt.item())
+    t_ms = max_over_ranks(t_ms, dist, dev)
     per = t_ms / args.steps
     return {"value": round(world * B / (per / 1e3), 3), "unit": UNIT, "ms_per_step": round(per, 3),
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
