@@ -374,6 +374,27 @@ def test_block_attention_ragged_mid_size(ctx):
                 rows=np.array(rows, np.int32))
 
 
+def test_block_512_shape_sampled_rows(ctx):
+    """VAR-d30-shaped 512x512 block: width 1920, 30 heads x 64, MLP 7680, last scale 32x32 over 1216
+    prior tokens, batch 4, ragged keep counts. Widths that are not multiples of 256 (partial GEMM
+    tiles), head size 64, and a mix of the CTA-pair and single-CTA GEMM kernels."""
+    ks = [512, 300, 1024, 77]
+    M = sum(ks)
+    rows = [0, 255, 256, 511, 512, 811, 812, 1835, 1836, M - 1]
+    _block_case(ctx, B=4, N=1024, C=1920, heads=30, F=7680, Lmax=2240, ks=ks, kv_lens=[1216] * 4, seed=23,
+                rows=np.array(rows, np.int32))
+
+
+def test_block_2048_shape_sampled_rows(ctx):
+    """2048x2048 stress shape: one image, 16384 tokens of which 3277 kept (keep ratio 0.2), attending
+    to 26137 prior tokens; width 2048, 16 heads x 128, MLP 8192."""
+    k = 16384 - int(0.8 * 16384)
+    assert k == 3277
+    rows = [0, 127, 128, 255, 256, 3071, 3072, 3199, 3200, k - 1]
+    _block_case(ctx, B=1, N=16384, C=2048, heads=16, F=8192, Lmax=42521, ks=[k], kv_lens=[26137], seed=29,
+                rows=np.array(rows, np.int32))
+
+
 def test_block_without_append_leaves_kv_len(ctx):
     B, N, C, heads, F, Lmax = 1, 64, 128, 2, 256, 256
     wt = synth.block_weights(C, F, 1, DEV)
@@ -463,3 +484,59 @@ def test_whole_pruned_step_config1(ctx):
     fx, _ = oracle.restore_from_cache(f32(x), wy, w_keep, w_prune, w_cu, f32(cache_prev), h, w)
     assert _rel_err(f32(x_out), fx) <= BLOCK_TOL
     assert ctx.device_status() == 0
+
+
+def test_pipeline_literal_schedule_256_shape(ctx):
+    """VAR-d16-shaped layers through the pipeline runner with the paper's schedule taken literally
+    (no overrides): the scale history puts the inflection at scale 7, so scale 9 (13 x 13 tokens) is
+    pruned with Ratio_9 = sigmoid(1 / tau) - lambda tanh(g_9), modulated per layer by Eq. 12-13 on the
+    means the GPU measured. Keep counts, activation scale and index lists must equal the oracle's on
+    the GPU's own entropies; the final activations follow the oracle run layer by layer."""
+    from paper_2602_01345_b200 import pipeline
+    ms = synth.CONFIGS["c2_var_d16_256"]
+    B, L, t = 2, 3, 9
+    h = w = ms.scales[t - 1]
+    hp = wp = ms.scales[t - 2]
+    N, P, Lmax = h * w, ms.prior_tokens(t), ms.total_tokens
+    weights = [synth.block_weights(ms.C, ms.F, 40 + j, DEV) for j in range(L)]
+    caches = [synth.kv_cache(B, Lmax, P, ms.C, 50 + j, DEV) for j in range(L)]
+    k_caches, v_caches = [c[0] for c in caches], [c[1] for c in caches]
+    kv_len = torch.full((L, B), P, dtype=torch.int32, device=DEV)
+    cache_prev = [synth.residual_cache(B, hp, wp, ms.C, 60 + j, DEV) for j in range(L)]
+    a = synth.smooth_temperature_field(B, h, w, seed=5, device=DEV)
+    beta = synth.layer_inverse_temperatures(L, 5)
+    logits = [synth.logits_from_temperature(a * float(beta[j]), synth.V_CODEBOOK, 70 + j) for j in range(L)]
+    x_in = synth.activations(B, N, ms.C, 80, DEV)
+    k0 = [k.clone() for k in k_caches]
+    v0 = [v.clone() for v in v_caches]
+    # mean entropies of scales 1..8 rise by 1 per scale, then flatten: t* = 7, pruning from scale 8
+    hist = torch.tensor([[1, 2, 3, 4, 5, 6, 6, 6, 0]], dtype=torch.float32).repeat(B, 1)
+
+    runner = pipeline.PrunedScaleRunner(ctx, weights, ms.heads, B, h, w, Lmax, k_caches, v_caches, kv_len, cache_prev)
+    # scale 9's own mean entropy (layer 1's map) completes the history, as the caller would do
+    ent0, mean0 = gpu_entropy(ctx, logits[0])
+    hist[:, t - 1] = mean0.cpu()
+    sched = nova.SchedParams()
+    x_out, keeps = runner.run_scale(x_in, logits, sched, t, hist)
+    assert ctx.device_status() == 0
+
+    osched = oracle.SchedParams()
+    x_ref = f32(x_in)
+    hbar_layer = np.zeros((B, L), np.float32)
+    for j in range(L):
+        ent_gpu = runner.ent[j].cpu().numpy()
+        w_ent, _ = oracle.scale_entropy(f32(logits[j]))
+        assert np.abs(ent_gpu - w_ent).max() <= ENT_TOL
+        hbar_layer[:, j] = runner.mean[j].cpu().numpy()
+        wr = oracle.keep_ratios(osched, t, j + 1, N, hist.numpy(), hbar_layer[:, : j + 1].copy())
+        assert np.array_equal(keeps[j].numpy(), wr["keep"])
+        assert (wr["act_scale"] == 8).all() and (wr["t_star"] == 7).all()
+        assert (wr["keep"] < N).all() and (wr["keep"] >= 1).all()          # this scale really is pruned
+        w_keep, w_prune, w_cu, _ = oracle.select_topk(ent_gpu, wr["keep"])
+        wy, _, _ = oracle.pruned_block_forward({n: f32(v) for n, v in weights[j].items()}, 1e-6, ms.heads, x_ref,
+                                               w_keep, w_cu, f32(k0[j]), f32(v0[j]), np.full(B, P, np.int32))
+        x_ref, _ = oracle.restore_from_cache(x_ref, wy, w_keep, w_prune, w_cu, f32(cache_prev[j]), h, w)
+    assert keeps[1].tolist() != keeps[0].tolist() or keeps[2].tolist() != keeps[0].tolist()   # Eq. 13 moved them
+    # free-running over three layers: bf16 storage between stages on the GPU, fp32 in the oracle
+    assert _rel_err(f32(x_out), x_ref) <= BLOCK_TOL
+    assert kv_len.cpu().tolist() == [[P + int(k) for k in keeps[j].tolist()] for j in range(L)]
