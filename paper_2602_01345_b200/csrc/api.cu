@@ -77,8 +77,8 @@ int nova_profile_categories(void) { return NOVA_K_COUNT; }
 const char* nova_profile_category_name(int cat)
 {
     static const char* names[NOVA_K_COUNT] = {
-        "entropy_rows", "entropy_mean", "select_topk", "build_row_maps", "layernorm", "gemm_qkv",
-        "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "advance_kv_len", "restore"};
+        "entropy_rows", "entropy_mean", "select_topk", "layernorm", "gemm_qkv",
+        "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "restore"};
     return (cat >= 0 && cat < NOVA_K_COUNT) ? names[cat] : "?";
 }
 

@@ -10,36 +10,17 @@ namespace {
 // src_row[r] = b*N + keep_idx[r]            row of x_in feeding compacted row r
 // kv_row[r]  = b*Lmax + kv_len[b] + (r - cu_keep[b])   cache row receiving r's k and v
 //              (-1 and a SHAPE flag if the image's cache would overflow)
-__global__ void build_row_maps(const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ cu_keep,
-                               const int32_t* __restrict__ kv_len, int B, int N, int Lmax, int M,
-                               int32_t* __restrict__ src_row, int32_t* __restrict__ kv_row,
-                               unsigned int* status)
-{
-    const int r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r >= M) return;
-    int lo = 0, hi = B;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (cu_keep[mid] <= r) lo = mid; else hi = mid;
-    }
-    const int b = lo;
-    src_row[r] = b * N + keep_idx[r];
-    const int k_b = cu_keep[b + 1] - cu_keep[b];
-    if (kv_len[b] + k_b > Lmax) {
-        kv_row[r] = -1;
-        atomicOr(status, NOVA_DEV_SHAPE);
-    } else {
-        kv_row[r] = b * Lmax + kv_len[b] + (r - cu_keep[b]);
-    }
-}
-
-__global__ void advance_kv_len(const int32_t* __restrict__ cu_keep, int32_t* __restrict__ kv_len, int B, int Lmax)
-{
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= B) return;
-    const int k_b = cu_keep[b + 1] - cu_keep[b];
-    if (kv_len[b] + k_b <= Lmax) kv_len[b] += k_b;
-}
+// Both are produced by the first LayerNorm (one warp per compacted row) on its way: it needs
+// src_row to gather its input anyway.
+struct RowMapArgs {
+    const int32_t* keep_idx;
+    const int32_t* cu_keep;
+    const int32_t* kv_len;
+    int B, N, Lmax;
+    int32_t* src_row;
+    int32_t* kv_row;
+    unsigned int* status;
+};
 
 // ---- LayerNorm ----------------------------------------------------------------------------
 // One warp per row; the row (C <= 32*8*VEC bf16) stays in registers between the mean, the
@@ -53,15 +34,35 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-template <int VEC>
+template <int VEC, bool MAPS>
 __global__ void __launch_bounds__(kLnWarps * 32)
-layernorm_rows(const uint4* __restrict__ x, const int32_t* __restrict__ src_row, const uint4* __restrict__ gamma,
-               const uint4* __restrict__ beta, float eps, int M, int vec_per_row, uint4* __restrict__ out)
+layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
+               float eps, int M, int vec_per_row, uint4* __restrict__ out, const RowMapArgs maps)
 {
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
     if (r >= M) return;
-    const long src = src_row ? (long)src_row[r] : (long)r;
+    long src = r;
+    if (MAPS) {
+        // image of compacted row r: largest b with cu_keep[b] <= r
+        int lo = 0, hi = maps.B;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (maps.cu_keep[mid] <= r) lo = mid; else hi = mid;
+        }
+        const int b = lo, c0 = maps.cu_keep[b];
+        src = (long)b * maps.N + maps.keep_idx[r];
+        if (lane == 0) {
+            maps.src_row[r] = (int32_t)src;
+            const int k_b = maps.cu_keep[b + 1] - c0, len = maps.kv_len[b];
+            if (len + k_b > maps.Lmax) {
+                maps.kv_row[r] = -1;
+                atomicOr(maps.status, NOVA_DEV_SHAPE);
+            } else {
+                maps.kv_row[r] = b * maps.Lmax + len + (r - c0);
+            }
+        }
+    }
     const uint4* xr = x + src * vec_per_row;
     float v[VEC][8];
     float sum = 0.f;
@@ -148,16 +149,22 @@ bool shape_ok(const nova_block_shape* s)
 
 }  // namespace
 
-nova_status nova_launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const int32_t* src_row,
-                           const __nv_bfloat16* g, const __nv_bfloat16* b, float eps, int M, int C,
-                           __nv_bfloat16* out, cudaStream_t st)
+static nova_status launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const RowMapArgs* maps,
+                             const __nv_bfloat16* g, const __nv_bfloat16* b, float eps, int M, int C,
+                             __nv_bfloat16* out, cudaStream_t st)
 {
     if (M <= 0) return NOVA_OK;
     const int vec = C / 8;
     const int per_lane = (vec + 31) / 32;
     const dim3 grid((M + kLnWarps - 1) / kLnWarps), block(kLnWarps * 32);
+    RowMapArgs none;
+    memset(&none, 0, sizeof(none));
     nova_launch_scope scope(ctx, NOVA_K_LAYERNORM, st);
-#define NOVA_LN_CASE(V) layernorm_rows<V><<<grid, block, 0, st>>>((const uint4*)x, src_row, (const uint4*)g, (const uint4*)b, eps, M, vec, (uint4*)out)
+#define NOVA_LN_CASE(V)                                                                                          \
+    do {                                                                                                         \
+        if (maps) layernorm_rows<V, true><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, vec, (uint4*)out, *maps); \
+        else layernorm_rows<V, false><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, vec, (uint4*)out, none);      \
+    } while (0)
     if (per_lane <= 2) NOVA_LN_CASE(2);
     else if (per_lane <= 4) NOVA_LN_CASE(4);
     else if (per_lane <= 8) NOVA_LN_CASE(8);
@@ -204,16 +211,12 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     typedef const __nv_bfloat16* cbf;
     typedef __nv_bfloat16* bf;
 
-    {
-        nova_launch_scope scope(ctx, NOVA_K_ROW_MAPS, st);
-        build_row_maps<<<(M + 255) / 256, 256, 0, st>>>(keep_idx, cu_keep, kv_len, s->B, s->N, s->Lmax, M,
-                                                        ws.src_row, ws.kv_row, ctx->dev_status);
-    }
-    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
-
     nova_status rc;
-    // h = LN1(gathered rows)
-    rc = nova_launch_ln(ctx, (cbf)x_in, ws.src_row, (cbf)w->ln1_g, (cbf)w->ln1_b, w->eps, M, C, ws.h, st);
+    // h = LN1(gathered rows); the same kernel writes the row maps the GEMM epilogues use
+    RowMapArgs maps;
+    maps.keep_idx = keep_idx; maps.cu_keep = cu_keep; maps.kv_len = kv_len; maps.B = s->B; maps.N = s->N;
+    maps.Lmax = s->Lmax; maps.src_row = ws.src_row; maps.kv_row = ws.kv_row; maps.status = ctx->dev_status;
+    rc = launch_ln(ctx, (cbf)x_in, &maps, (cbf)w->ln1_g, (cbf)w->ln1_b, w->eps, M, C, ws.h, st);
     if (rc) return rc;
     // [q | k | v] = h W_qkv^T + b; k, v go straight to their cache rows
     nova_gemm_args g;
@@ -235,7 +238,7 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     // h = LN2(x1)
-    rc = nova_launch_ln(ctx, ws.x1, nullptr, (cbf)w->ln2_g, (cbf)w->ln2_b, w->eps, M, C, ws.h, st);
+    rc = launch_ln(ctx, ws.x1, nullptr, (cbf)w->ln2_g, (cbf)w->ln2_b, w->eps, M, C, ws.h, st);
     if (rc) return rc;
     // f = GELU(h W_fc1^T + b_fc1)
     memset(&g, 0, sizeof(g));
@@ -247,13 +250,13 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     memset(&g, 0, sizeof(g));
     g.A = ws.f; g.W = (cbf)w->w_fc2; g.bias = (cbf)w->b_fc2; g.M = M; g.N = C; g.K = F;
     g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_FC2; g.out = (bf)y_kept; g.res = ws.x1; g.res_row = nullptr;
+    if (append_kv) {
+        // the last kernel of the block also advances kv_len: every reader of the old lengths (row
+        // maps, attention) ran in an earlier kernel of this call
+        g.adv_cu_keep = cu_keep; g.adv_kv_len = kv_len; g.adv_B = s->B; g.adv_Lmax = s->Lmax;
+    }
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
-    if (append_kv) {
-        nova_launch_scope scope(ctx, NOVA_K_KV_ADVANCE, st);
-        advance_kv_len<<<(s->B + 127) / 128, 128, 0, st>>>(cu_keep, kv_len, s->B, s->Lmax);
-        NOVA_CUDA_CHECK(ctx, cudaGetLastError());
-    }
     return NOVA_OK;
 }
 

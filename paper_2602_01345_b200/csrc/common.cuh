@@ -18,9 +18,9 @@
 
 // Kernel categories for the launch counter and the optional per-kernel event timing.
 enum nova_kernel_cat {
-    NOVA_K_ENTROPY = 0, NOVA_K_ENTROPY_MEAN, NOVA_K_SELECT, NOVA_K_ROW_MAPS, NOVA_K_LAYERNORM,
+    NOVA_K_ENTROPY = 0, NOVA_K_ENTROPY_MEAN, NOVA_K_SELECT, NOVA_K_LAYERNORM,
     NOVA_K_GEMM_QKV, NOVA_K_ATTENTION, NOVA_K_GEMM_PROJ, NOVA_K_GEMM_FC1, NOVA_K_GEMM_FC2,
-    NOVA_K_KV_ADVANCE, NOVA_K_RESTORE, NOVA_K_COUNT
+    NOVA_K_RESTORE, NOVA_K_COUNT
 };
 
 struct nova_prof_rec {
@@ -98,9 +98,6 @@ static inline nova_status nova_cuda_fail(nova_ctx* ctx, cudaError_t e, const cha
 static inline bool nova_aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
 
 // Kernel launchers implemented in the other translation units.
-nova_status nova_launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const int32_t* src_row,
-                           const __nv_bfloat16* g, const __nv_bfloat16* b, float eps, int M, int C,
-                           __nv_bfloat16* out, cudaStream_t st);
 
 enum nova_epilogue {
     NOVA_EPI_QKV = 0,       // +bias; columns [0,C) -> q, [C,2C) -> k cache rows, [2C,3C) -> v cache rows
@@ -124,6 +121,10 @@ struct nova_gemm_args {
     __nv_bfloat16* k_cache;
     __nv_bfloat16* v_cache;
     const int32_t* kv_row;      // [M] destination cache row (b*Lmax + kv_len[b] + m), -1 = skip
+    // optional tail of the launch: kv_len[b] += cu_keep[b+1] - cu_keep[b] where it fits in Lmax
+    const int32_t* adv_cu_keep;
+    int32_t* adv_kv_len;
+    int adv_B, adv_Lmax;
 };
 
 nova_status nova_launch_gemm(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st);

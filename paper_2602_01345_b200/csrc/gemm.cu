@@ -58,7 +58,20 @@ struct GemmParams {
     __nv_bfloat16* v_cache;
     const int32_t* kv_row;
     unsigned int* status;
+    const int32_t* adv_cu_keep;
+    int32_t* adv_kv_len;
+    int adv_B, adv_Lmax;
 };
+
+// Advance of the K/V cache lengths, done by one warp-sized loop of the launch's first CTA.
+__device__ __forceinline__ void advance_kv_len(const GemmParams& p)
+{
+    if (!p.adv_kv_len) return;
+    for (int b = threadIdx.x; b < p.adv_B; b += blockDim.x) {
+        const int k_b = p.adv_cu_keep[b + 1] - p.adv_cu_keep[b];
+        if (p.adv_kv_len[b] + k_b <= p.adv_Lmax) p.adv_kv_len[b] += k_b;
+    }
+}
 
 
 // Epilogue of 32 consecutive accumulator columns [col0, col0 + 32) of output row `row`:
@@ -130,6 +143,7 @@ gemm_bf16_tn(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int num_kb = p.K / BK;
+    if (blockIdx.x == 0 && blockIdx.y == 0) advance_kv_len(p);
 
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
@@ -226,6 +240,7 @@ GemmParams make_params(nova_ctx* ctx, const nova_gemm_args& a)
     p.bias = a.bias; p.M = a.M; p.N = a.N; p.K = a.K; p.epilogue = a.epilogue; p.out = a.out;
     p.res = a.res; p.res_row = a.res_row; p.C = a.C; p.k_cache = a.k_cache; p.v_cache = a.v_cache;
     p.kv_row = a.kv_row; p.status = ctx->dev_status;
+    p.adv_cu_keep = a.adv_cu_keep; p.adv_kv_len = a.adv_kv_len; p.adv_B = a.adv_B; p.adv_Lmax = a.adv_Lmax;
     return p;
 }
 
@@ -295,6 +310,7 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();     // 0 = leader
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    if (blockIdx.x == 0) advance_kv_len(p);
     const int num_kb = p.K / BK;
     constexpr uint32_t kTmemCols = 2 * BN;       // two accumulator buffers
 
