@@ -27,6 +27,14 @@ struct RowMapArgs {
 // variance and the normalisation, so x is read once and out written once.
 constexpr int kLnWarps = 8;
 
+__device__ __forceinline__ uint4 ld_nc_stream(const uint4* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll
@@ -64,44 +72,56 @@ layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, con
         }
     }
     const uint4* xr = x + src * vec_per_row;
-    float v[VEC][8];
-    float sum = 0.f;
+    // The row is read once (streaming loads, all issued before the first use) and stays in
+    // registers for the three sweeps: sum, squared deviations, normalise.
+    uint4 raw[VEC];
 #pragma unroll
     for (int i = 0; i < VEC; ++i) {
         const int c = i * 32 + lane;
-        uint4 raw = make_uint4(0, 0, 0, 0);
-        if (c < vec_per_row) raw = xr[c];
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        raw[i] = (c < vec_per_row) ? ld_nc_stream(xr + c) : make_uint4(0, 0, 0, 0);
+    }
+    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) {
+        const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            v[i][2 * q] = __uint_as_float(w[q] << 16);
-            v[i][2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
-            sum += v[i][2 * q] + v[i][2 * q + 1];
+            sum0 += __uint_as_float(w[q] << 16);
+            sum1 += __uint_as_float(w[q] & 0xffff0000u);
         }
     }
     const float n = (float)(vec_per_row * 8);
-    const float mean = warp_sum(sum) / n;
-    float sq = 0.f;
+    const float mean = warp_sum(sum0 + sum1) / n;
+    float sq0 = 0.f, sq1 = 0.f;
 #pragma unroll
     for (int i = 0; i < VEC; ++i) {
         if (i * 32 + lane < vec_per_row) {
+            const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
 #pragma unroll
-            for (int q = 0; q < 8; ++q) { const float d = v[i][q] - mean; sq += d * d; }
+            for (int q = 0; q < 4; ++q) {
+                const float d0 = __uint_as_float(w[q] << 16) - mean, d1 = __uint_as_float(w[q] & 0xffff0000u) - mean;
+                sq0 = fmaf(d0, d0, sq0);
+                sq1 = fmaf(d1, d1, sq1);
+            }
         }
     }
-    const float rstd = rsqrtf(warp_sum(sq) / n + eps);
+    const float rstd = rsqrtf(warp_sum(sq0 + sq1) / n + eps);
+    const float shift = -mean * rstd;
 #pragma unroll
     for (int i = 0; i < VEC; ++i) {
         const int c = i * 32 + lane;
         if (c < vec_per_row) {
             const uint4 g = gamma[c], bt = beta[c];
+            const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
             const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, bw[4] = {bt.x, bt.y, bt.z, bt.w};
             uint32_t o[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const float y0 = (v[i][2 * q] - mean) * rstd * __uint_as_float(gw[q] << 16) + __uint_as_float(bw[q] << 16);
-                const float y1 = (v[i][2 * q + 1] - mean) * rstd * __uint_as_float(gw[q] & 0xffff0000u) +
-                                 __uint_as_float(bw[q] & 0xffff0000u);
+                // (x - mean) * rstd = x * rstd + shift
+                const float n0 = fmaf(__uint_as_float(w[q] << 16), rstd, shift);
+                const float n1 = fmaf(__uint_as_float(w[q] & 0xffff0000u), rstd, shift);
+                const float y0 = fmaf(n0, __uint_as_float(gw[q] << 16), __uint_as_float(bw[q] << 16));
+                const float y1 = fmaf(n1, __uint_as_float(gw[q] & 0xffff0000u), __uint_as_float(bw[q] & 0xffff0000u));
                 __nv_bfloat162 t = __floats2bfloat162_rn(y0, y1);
                 o[q] = *reinterpret_cast<uint32_t*>(&t);
             }
