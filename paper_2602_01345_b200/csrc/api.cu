@@ -42,8 +42,8 @@ nova_status nova_create(nova_ctx** out, int device)
     ctx->profiling = false;
     ctx->events_used = 0;
     if (cudaSetDevice(device) != cudaSuccess ||
-        cudaMalloc(&ctx->dev_status, 256) != cudaSuccess ||
-        cudaMemset(ctx->dev_status, 0, 256) != cudaSuccess) {
+        cudaMalloc(&ctx->dev_status, NOVA_STATUS_BYTES) != cudaSuccess ||
+        cudaMemset(ctx->dev_status, 0, NOVA_STATUS_BYTES) != cudaSuccess) {
         delete ctx;
         return NOVA_ERR_CUDA;
     }

@@ -16,6 +16,14 @@
 #define NOVA_DEV_TIMEOUT   2u
 #define NOVA_DEV_SHAPE     4u
 
+// Layout of the context's one device allocation: NOVA_STATUS_WORDS 32-bit words (word 0 = status
+// bits, word 1 = completion counter of the entropy kernel), then the per-CTA partial sums of the
+// entropy means, float[NOVA_MEAN_MAX_CTAS][NOVA_MEAN_MAX_SEGMENTS].
+#define NOVA_STATUS_WORDS 64
+#define NOVA_MEAN_MAX_CTAS 192
+#define NOVA_MEAN_MAX_SEGMENTS 256
+#define NOVA_STATUS_BYTES (NOVA_STATUS_WORDS * 4 + NOVA_MEAN_MAX_CTAS * NOVA_MEAN_MAX_SEGMENTS * 4)
+
 // Kernel categories for the launch counter and the optional per-kernel event timing.
 enum nova_kernel_cat {
     NOVA_K_ENTROPY = 0, NOVA_K_ENTROPY_MEAN, NOVA_K_SELECT, NOVA_K_LAYERNORM,

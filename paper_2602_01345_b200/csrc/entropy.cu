@@ -49,8 +49,8 @@ __device__ __forceinline__ void unpack_bf16x2(uint32_t w, float& lo, float& hi)
 }
 
 // finishing step shared by all kernels: lane 0 writes the row result
-__device__ __forceinline__ void finish_row(float m, float s, float u, float* ent, long row,
-                                           unsigned int* status)
+__device__ __forceinline__ float finish_row(float m, float s, float u, float* ent, long row,
+                                            unsigned int* status)
 {
     // H = ln s - u/s with u accumulated in the log2 domain: d2 = (z-m)*log2e, u2 = sum d2 * 2^d2
     float h = logf(s) - (u / s) * kLn2;   // precise log once per row: ln 1 must be exactly 0
@@ -61,6 +61,7 @@ __device__ __forceinline__ void finish_row(float m, float s, float u, float* ent
         h = 0.f;   // also turns -0 into +0; true entropy is never negative
     }
     ent[row] = h;
+    return h;
 }
 
 // ---- two fp32 values per 64-bit register: one instruction does both lanes' arithmetic ----------
@@ -246,6 +247,7 @@ entropy_rows_reg(const void* __restrict__ logits, long rows, int V, long row_str
 // poll a slot whose previous use some other warp has yet to see.
 constexpr int kRingConsumers = 16;
 constexpr int kRingThreads = (kRingConsumers + 1) * 32;
+constexpr int kMaxMeanSegments = NOVA_MEAN_MAX_SEGMENTS;
 constexpr int kRingBytes = 128 * 1024;
 
 // Bulk copy global -> shared of `bytes` (multiple of 16, both addresses 16-byte aligned).
@@ -259,7 +261,7 @@ template <int VEC, bool BF16>
 __global__ void __launch_bounds__(kRingThreads, 1)
 entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_stride_bytes,
                   float* __restrict__ ent, float* __restrict__ mean, int seg_rows, int n_seg,
-                  unsigned int* status, unsigned int* done_counter)
+                  unsigned int* status, unsigned int* done_counter, float* __restrict__ cta_part)
 {
     using namespace tc;
     constexpr int kRowBytes = VEC * 512;
@@ -269,9 +271,9 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
     uint8_t* ring = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     uint64_t* full_bar = (uint64_t*)(ring + kSlots * kRowBytes);
     uint64_t* empty_bar = full_bar + kSlots;
+    float* warp_part = (float*)(empty_bar + kSlots);       // [kRingConsumers][n_seg] partial sums per warp
     __shared__ int abort_flag_s;
     __shared__ int is_last_s;
-    __shared__ float part[8][kRingThreads / 32];
     volatile int* abort_flag = &abort_flag_s;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -286,6 +288,8 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
         }
         fence_barrier_init();
     }
+    if (mean)
+        for (int i = threadIdx.x; i < kRingConsumers * n_seg; i += kRingThreads) warp_part[i] = 0.f;
     __syncthreads();
 
     if (warp == kRingConsumers) {
@@ -304,6 +308,9 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
                     mbar_drain(&full_bar[i % kSlots], (uint32_t)(i / kSlots) & 1);
         }
     } else {
+        // running sum of this warp's entropies in the segment it is in (rows come in rising order)
+        int cur_seg = -1;
+        float seg_acc = 0.f;
         for (long i = warp; i < n_my; i += kRingConsumers) {
             const int slot = (int)(i % kSlots);
             if (!mbar_wait_warp(&full_bar[slot], (uint32_t)(i / kSlots) & 1, abort_flag, status)) break;
@@ -316,15 +323,33 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
             const long row = blockIdx.x + i * G;
             float m, s_sum, u;
             entropy_row_from_regs<VEC, BF16>(reg, logits + row * row_stride_bytes, V, lane, m, s_sum, u);
-            if (lane == 0) finish_row(m, s_sum, u, ent, row, status);
+            if (lane == 0) {
+                const float h = finish_row(m, s_sum, u, ent, row, status);
+                if (mean) {
+                    const int seg = (int)(row / seg_rows);
+                    if (seg != cur_seg) {
+                        if (cur_seg >= 0) warp_part[warp * n_seg + cur_seg] = seg_acc;
+                        cur_seg = seg;
+                        seg_acc = 0.f;
+                    }
+                    seg_acc += h;
+                }
+            }
         }
+        if (lane == 0 && mean && cur_seg >= 0) warp_part[warp * n_seg + cur_seg] = seg_acc;
     }
     if (!mean) return;
 
-    // ---- last CTA to finish takes the means ----------------------------------------------------
-    // Writers publish their entropies (fence) before the CTA's ticket is drawn; the last CTA reads
-    // them with L2 loads (ld.cg), so it needs no fence of its own.
-    if (lane == 0 && warp < kRingConsumers) __threadfence();
+    // ---- means: per-CTA partial sums, combined by the last CTA to finish ------------------------
+    // Every level adds in a fixed order (a warp's rows in row order, the 16 warps in warp order,
+    // the CTAs in CTA order with a fixed tree), so the means do not depend on which CTA is last.
+    __syncthreads();
+    for (int sg = threadIdx.x; sg < n_seg; sg += kRingThreads) {
+        float acc = 0.f;
+        for (int w = 0; w < kRingConsumers; ++w) acc += warp_part[w * n_seg + sg];
+        cta_part[(long)blockIdx.x * n_seg + sg] = acc;
+    }
+    __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
         const unsigned int ticket = atomicAdd(done_counter, 1u);
@@ -333,40 +358,12 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
     }
     __syncthreads();
     if (!is_last_s) return;
-    // Eight segments at a time: every thread first issues all its loads (thread t takes elements
-    // t, t + 544, ... of each segment), so the whole read costs about one L2 round trip; then one
-    // shuffle tree per segment, one exchange through shared memory, and warp g finishes segment g.
-    constexpr int kGroup = 8;
-    constexpr int kWarps = kRingThreads / 32;
-    for (int sg0 = 0; sg0 < n_seg; sg0 += kGroup) {
-        float acc[kGroup];
-#pragma unroll
-        for (int g = 0; g < kGroup; ++g) acc[g] = 0.f;
-#pragma unroll 2
-        for (int i0 = threadIdx.x; i0 < seg_rows; i0 += 4 * kRingThreads) {
-            float v[kGroup][4];
-#pragma unroll
-            for (int g = 0; g < kGroup; ++g)
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int i = i0 + r * kRingThreads;
-                    v[g][r] = (sg0 + g < n_seg && i < seg_rows) ? __ldcg(ent + (long)(sg0 + g) * seg_rows + i) : 0.f;
-                }
-#pragma unroll
-            for (int g = 0; g < kGroup; ++g) acc[g] += (v[g][0] + v[g][1]) + (v[g][2] + v[g][3]);
-        }
-#pragma unroll
-        for (int g = 0; g < kGroup; ++g) {
-            const float w = warp_sum(acc[g]);
-            if (lane == 0) part[g][warp] = w;
-        }
-        __syncthreads();
-        if (warp < kGroup && sg0 + warp < n_seg) {
-            float v = (lane < kWarps) ? part[warp][lane] : 0.f;
-            v = warp_sum(v);
-            if (lane == 0) mean[sg0 + warp] = v / (float)seg_rows;
-        }
-        __syncthreads();
+    // one warp per segment: lane l adds CTAs l, l + 32, ... in order, then the shuffle tree
+    for (int sg = warp; sg < n_seg; sg += kRingThreads / 32) {
+        float acc = 0.f;
+        for (int c = lane; c < (int)gridDim.x; c += 32) acc += __ldcg(cta_part + (long)c * n_seg + sg);
+        acc = warp_sum(acc);
+        if (lane == 0) mean[sg] = acc / (float)seg_rows;
     }
 }
 
@@ -429,7 +426,7 @@ nova_status launch_ring(nova_ctx* ctx, const void* logits, long rows, int V, lon
                         float* mean, int N, int S, cudaStream_t st)
 {
     constexpr int kSlots = kRingBytes / (VEC * 512);
-    const size_t smem = kRingBytes + 128 + 2 * sizeof(uint64_t) * kSlots;
+    const size_t smem = kRingBytes + 128 + 2 * sizeof(uint64_t) * kSlots + sizeof(float) * kRingConsumers * kMaxMeanSegments;
     static bool attr_done[64];
     if (ctx->device < 64 && !attr_done[ctx->device]) {
         NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(entropy_rows_ring<VEC, BF16>,
@@ -438,7 +435,8 @@ nova_status launch_ring(nova_ctx* ctx, const void* logits, long rows, int V, lon
     }
     const int grid = (int)(rows < ctx->num_sms ? rows : ctx->num_sms);
     entropy_rows_ring<VEC, BF16><<<grid, kRingThreads, smem, st>>>(
-        (const char*)logits, rows, V, stride_bytes, ent, mean, N, S, ctx->dev_status, ctx->dev_status + 1);
+        (const char*)logits, rows, V, stride_bytes, ent, mean, N, S, ctx->dev_status, ctx->dev_status + 1,
+        (float*)(ctx->dev_status + NOVA_STATUS_WORDS));
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }
@@ -461,7 +459,8 @@ extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nov
     cudaStream_t st = (cudaStream_t)stream;
     const int elt = (dt == NOVA_BF16) ? 2 : 4;
     const long row_bytes = (long)V * elt;
-    if ((row_bytes == 2048 || row_bytes == 4096 || row_bytes == 8192) && rows >= 64) {
+    if ((row_bytes == 2048 || row_bytes == 4096 || row_bytes == 8192) && rows >= 64 &&
+        (!mean || (S <= NOVA_MEAN_MAX_SEGMENTS && ctx->num_sms <= NOVA_MEAN_MAX_CTAS))) {
         // persistent ring kernel; the second word of the status allocation is its completion counter
         const long stride_bytes = (long)row_stride * elt;
         nova_launch_scope scope(ctx, NOVA_K_ENTROPY, st);
