@@ -35,7 +35,7 @@ UNIT = "images/s"
 # for any other workload, and reset to None whenever the kernel changes after the capture.
 # attention: one launch; gemm: average over the four launches of a layer (qkv, proj, fc1, fc2), the
 # unit `achieved` is taken over as well. Source: profiles/layer_kernels_c4_1024_batch4_keep0.5.txt.
-NCU_TRAFFIC_BYTES = {"attention": 342_493_952, "gemm": 171_636_672}
+NCU_TRAFFIC_BYTES = {"attention": 347_592_448, "gemm": 172_289_408}
 
 
 def parse_args():
