@@ -88,6 +88,21 @@ def scale_entropy(logits: np.ndarray):
     return ent, mean
 
 
+def head_entropy(x: np.ndarray, w: np.ndarray, b=None):
+    """Eq. 4 / Eq. 7 on the codebook head's output: logits = x @ w.T + b, never rounded.
+    x [S, N, C], w [V, C], b [V] or None -> (ent [S, N] f32, mean [S] f32)."""
+    x = _f32(x)
+    w = _f32(w)
+    S, N, C = x.shape
+    V = w.shape[0]
+    assert w.shape == (V, C)
+    bb = _f32(b) if b is not None else None
+    ent = np.empty((S, N), np.float32)
+    mean = np.empty((S,), np.float32)
+    _load().oracle_head_entropy(_p(x), _p(w), _p(bb) if bb is not None else None, S, N, C, V, _p(ent), _p(mean))
+    return ent, mean
+
+
 @dataclass
 class SchedParams:
     """Hyper-parameters of Eq. 9-11 (paper defaults) plus this build's clamps and overrides."""

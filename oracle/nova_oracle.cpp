@@ -60,6 +60,48 @@ void oracle_scale_entropy(const float* logits, int S, int N, int V,
 }
 
 // ---------------------------------------------------------------------------
+// Eq. 4 / Eq. 7 taken one step earlier: the predicted distribution of a token is the
+// softmax of the codebook head applied to its hidden state (the paper takes the
+// distributions "already produced during standard decoding"), so
+//   logits[v] = sum_c x[c] * w[v, c] + b[v],   p = softmax(logits),   H = -sum p ln p.
+// x [S, N, C], w [V, C] ([out, in] row-major), b [V] or null. The logits are never
+// rounded: double accumulation in index order, entropy as in oracle_scale_entropy.
+// ---------------------------------------------------------------------------
+void oracle_head_entropy(const float* x, const float* w, const float* b, int S, int N, int C, int V,
+                         float* ent, float* mean)
+{
+    const long rows = (long)S * N;
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < rows; ++r) {
+        const float* xr = x + r * (long)C;
+        std::vector<double> z((size_t)V);
+        for (int v = 0; v < V; ++v) {
+            double acc = b ? (double)b[v] : 0.0;
+            const float* wv = w + (long)v * C;
+            for (int c = 0; c < C; ++c) acc += (double)xr[c] * (double)wv[c];
+            z[v] = acc;
+        }
+        double zmax = -INFINITY;
+        for (int v = 0; v < V; ++v) zmax = std::max(zmax, z[v]);
+        double denom = 0.0;
+        for (int v = 0; v < V; ++v) denom += std::exp(z[v] - zmax);
+        double h = 0.0;
+        for (int v = 0; v < V; ++v) {
+            const double p = std::exp(z[v] - zmax) / denom;
+            if (p > 0.0) h -= p * std::log(p);
+        }
+        ent[r] = (float)h;
+    }
+    if (mean) {
+        for (int s = 0; s < S; ++s) {
+            double acc = 0.0;
+            for (int i = 0; i < N; ++i) acc += (double)ent[(long)s * N + i];
+            mean[s] = (float)(acc / (double)N);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Eq. 8-10 (growth rate, early baseline, smoothed rate, inflection scale),
 // Eq. 11 (scale-linkage ratio), Eq. 12-13 (layer-linkage ratio), and the keep
 // count that follows from a reduction ratio.

@@ -79,6 +79,51 @@ def test_entropy_neg_inf_logit_contributes_nothing():
     assert abs(ent[0, 0] - math.log(4)) < 1e-7
 
 
+# ----------------------------------------------------------- entropy of the codebook head
+def test_head_entropy_closed_forms():
+    """Zero head -> uniform -> ln V; bias only -> entropy of softmax(b) (two-level closed form);
+    a head whose rows are +-a along one hidden unit -> two-level distribution set by x."""
+    S, N, C, V = 1, 3, 8, 64
+    x = np.random.default_rng(0).standard_normal((S, N, C)).astype(np.float32)
+    ent, mean = oracle.head_entropy(x, np.zeros((V, C), np.float32))
+    assert np.allclose(ent, math.log(V), atol=1e-6) and np.allclose(mean, math.log(V), atol=1e-6)
+    b = np.zeros(V, np.float32)
+    b[:5] = 2.0
+    ent, _ = oracle.head_entropy(x, np.zeros((V, C), np.float32), b)
+    Z = 5 * math.exp(2.0) + (V - 5)
+    assert np.allclose(ent, math.log(Z) - 5 * 2.0 * math.exp(2.0) / Z, atol=1e-6)
+    w = np.zeros((V, C), np.float32)
+    w[: V // 2, 3] = 1.0                    # half of the codes see +x_3, the other half 0
+    ent, _ = oracle.head_entropy(x, w)
+    for i in range(N):
+        a = float(x[0, i, 3])
+        Z = (V // 2) * math.exp(a) + V // 2
+        want = math.log(Z) - (V // 2) * a * math.exp(a) / Z
+        assert abs(ent[0, i] - want) < 1e-6
+
+
+def test_head_entropy_equals_entropy_of_library_matmul_and_operand_order():
+    """Against numpy's float64 matmul followed by scipy's softmax entropy; a transposed or
+    mis-strided weight would fail (V != C, random values), so would a dropped bias."""
+    rng = np.random.default_rng(3)
+    S, N, C, V = 2, 5, 24, 40
+    x = rng.standard_normal((S, N, C)).astype(np.float32)
+    w = (0.3 * rng.standard_normal((V, C))).astype(np.float32)
+    b = rng.standard_normal(V).astype(np.float32)
+    ent, mean = oracle.head_entropy(x, w, b)
+    from scipy.special import softmax
+    from scipy.stats import entropy as sp_entropy
+    z = x.astype(np.float64) @ w.astype(np.float64).T + b.astype(np.float64)
+    want = sp_entropy(softmax(z, axis=-1), axis=-1)
+    assert np.abs(ent - want).max() < 1e-6
+    assert np.abs(mean - want.mean(axis=1)).max() < 1e-6
+    ent_nb, _ = oracle.head_entropy(x, w)
+    assert np.abs(ent_nb - want).max() > 1e-3          # the bias matters in this example
+    # and it is the same function as scale_entropy on the unrounded logits
+    ent2, _ = oracle.scale_entropy(z.astype(np.float32))
+    assert np.abs(ent - ent2).max() < 1e-5
+
+
 def test_mean_is_per_segment_and_permutation_invariant():
     rng = np.random.default_rng(1)
     z = rng.standard_normal((3, 16, 64)).astype(np.float32) * 3
