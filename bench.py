@@ -295,6 +295,24 @@ def run_ours(args):
         us = b0.elapsed_time(b1) * 1e3 / len(st["logits"])
         key = "gbs_back_to_back" if with_mean else "gbs_back_to_back_no_mean"
         kernels["entropy_rows"][key] = round(ent_bytes / us / 1e3, 1)
+    # Entropy fused with the codebook head (the step before the path: hidden states -> entropy, the
+    # 8 KiB/token of logits never stored), timed back to back over 8 calls outside the timed region.
+    head_w = synth.randn_bf16((synth.V_CODEBOOK, ms.C), 991, dev, std=3.0 / ms.C ** 0.5)
+    hidden = [synth.activations(B, N, ms.C, 900 + i, dev) for i in range(4)]
+    for _ in range(2):
+        nova.nova_head_entropy(ctx, hidden[0], head_w, None, ent_buf, mean_buf, stream=stream)
+    torch.cuda.synchronize()
+    b0.record(stream)
+    for i in range(8):
+        nova.nova_head_entropy(ctx, hidden[i % 4], head_w, None, ent_buf, mean_buf, stream=stream)
+    b1.record(stream)
+    torch.cuda.synchronize()
+    head_us = b0.elapsed_time(b1) * 1e3 / 8
+    head_tf = 2.0 * rows * ms.C * synth.V_CODEBOOK / head_us / 1e6
+    head_entropy = {"us_per_call": round(head_us, 1), "tflops": round(head_tf, 1),
+                    "frac_of_tensor_peak": round(head_tf / pk["tensor"], 4),
+                    "logits_bytes_not_written_or_read": int(2 * rows * synth.V_CODEBOOK * 2)}
+    assert ctx.device_status() == 0, "device status after the head-entropy timing"
     for k in ("entropy_rows", "restore"):
         if "gbs" in kernels.get(k, {}):
             kernels[k]["frac_of_hbm_peak"] = round(kernels[k]["gbs"] / pk["hbm"], 4)
@@ -307,6 +325,7 @@ def run_ours(args):
         "config": config_json(wd, world), "clocks": clk, "gpu_launches": int(launches),
         "tokens_per_s": round(world * B * N / (ms_per_step / 1e3), 1),
         "roofline": roofline, "roofline_second": other_roofline, "kernels": kernels,
+        "next_head_entropy": head_entropy,
     }
 
     # ---- end to end: inputs start in pinned host memory, result read back every step

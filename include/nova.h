@@ -6,6 +6,7 @@
  * at an accelerated scale:
  *
  *   nova_scale_entropy      Eq. 4, Eq. 7   per-token entropy and per-image mean
+ *   nova_head_entropy       Eq. 4, Eq. 7   the same from hidden states and the codebook head
  *   nova_keep_ratios        Eq. 8-13       inflection trigger, scale/layer ratios, keep counts
  *   nova_select_topk        text after Eq. 3 / Eq. 13: keep the highest-entropy tokens
  *   nova_pruned_block_forward   Eq. 14     the layer on the kept tokens only
@@ -94,6 +95,22 @@ nova_status nova_profile_end(nova_ctx* ctx, double* ms, long long* launches, int
 nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nova_dtype dt,
                                int S, int N, int V, int64_t row_stride,
                                float* ent, float* mean, void* stream);
+
+/* ---- Eq. 4 and Eq. 7 from the hidden states: codebook head fused with the entropy -- */
+/*
+ * The paper takes the predicted distributions "already produced during standard decoding"
+ * (complexity paragraph after Table 8); a decoder that has the hidden states at hand can skip
+ * writing the V-wide logits altogether. This call computes, per token,
+ *   logits = x W_head^T + b_head (bf16 operands, fp32 accumulation, never rounded or stored),
+ *   ent = -sum_v p(v) ln p(v), p = softmax(logits), and mean[s] = (1/N) sum_i ent[s, i].
+ * x:      device bf16 [S*N, C] contiguous.   w_head: device bf16 [V, C] ([out, in] row-major).
+ * b_head: device bf16 [V] or NULL.           ent: device f32 [S, N].   mean: device f32 [S] or NULL.
+ * C must be a multiple of 64 and V of 32. A non-finite logit makes the row's entropy NaN and
+ * records NOVA_ERR_NONFINITE in the device status word. S*N == 0 is a no-op.
+ * Errors: bad sizes -> INVALID_ARG / SHAPE; misaligned pointer -> ALIGNMENT.
+ */
+nova_status nova_head_entropy(nova_ctx* ctx, const void* x, const void* w_head, const void* b_head,
+                              int S, int N, int C, int V, float* ent, float* mean, void* stream);
 
 /* ---- Eq. 8-13: trigger, ratios, keep counts (host arithmetic, double) ---------- */
 typedef struct nova_sched_params {

@@ -6,7 +6,7 @@ missing or cannot be loaded, importing this package fails.
 """
 from .binding import (  # noqa: F401
     NovaError, Context, SchedParams, BlockWeights, BlockShape,
-    nova_scale_entropy, nova_keep_ratios, nova_select_topk,
+    nova_scale_entropy, nova_head_entropy, nova_keep_ratios, nova_select_topk,
     nova_pruned_block_forward, nova_restore_from_cache, nova_block_workspace_bytes,
     nova_pruned_block_forward_static, nova_static_scratch_bytes,
     lib_path, STATUS_NAMES,

@@ -194,6 +194,22 @@ def nova_scale_entropy(ctx: Context, logits, ent, mean=None, stream=None):
                                       logits.stride(1), _ptr(ent), _ptr(mean), _stream(stream)))
 
 
+_lib.nova_head_entropy.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]
+_lib.nova_head_entropy.restype = _i
+
+
+def nova_head_entropy(ctx: Context, x, w_head, b_head, ent, mean=None, stream=None):
+    """x [S, N, C] bf16, w_head [V, C] bf16, b_head [V] bf16 or None -> ent [S, N] f32, mean [S] f32:
+    entropy of softmax(x @ w_head.T + b_head) per token, logits never stored."""
+    S, N, Cc = x.shape
+    V = w_head.shape[0]
+    assert x.dtype == torch.bfloat16 and x.is_contiguous() and w_head.dtype == torch.bfloat16
+    assert w_head.is_contiguous() and w_head.shape[1] == Cc
+    assert ent.dtype == torch.float32 and ent.is_contiguous() and ent.numel() == S * N
+    ctx.check(_lib.nova_head_entropy(ctx.handle, _ptr(x), _ptr(w_head), _ptr(b_head), S, N, Cc, V,
+                                     _ptr(ent), _ptr(mean), _stream(stream)))
+
+
 def nova_keep_ratios(p: SchedParams, t: int, j: int, N_t: int, hbar_scale, hbar_layer=None):
     """Host arithmetic of the trigger and ratio functions. hbar_* are CPU float32 tensors.
 

@@ -110,7 +110,8 @@ static inline bool nova_aligned16(const void* p) { return (((uintptr_t)p) & 15u)
 enum nova_epilogue {
     NOVA_EPI_QKV = 0,       // +bias; columns [0,C) -> q, [C,2C) -> k cache rows, [2C,3C) -> v cache rows
     NOVA_EPI_BIAS_RES = 1,  // +bias + residual[res_row[r]] -> out
-    NOVA_EPI_BIAS_GELU = 2  // GELU_tanh(+bias) -> out
+    NOVA_EPI_BIAS_GELU = 2, // GELU_tanh(+bias) -> out
+    NOVA_EPI_ENTROPY = 3    // +bias (optional); nothing stored but ent[r] = entropy of softmax(row r) over all N columns
 };
 
 struct nova_gemm_args {
@@ -129,6 +130,7 @@ struct nova_gemm_args {
     __nv_bfloat16* k_cache;
     __nv_bfloat16* v_cache;
     const int32_t* kv_row;      // [M] destination cache row (b*Lmax + kv_len[b] + m), -1 = skip
+    float* ent;                 // entropy epilogue: [M] fp32
     // optional tail of the launch: kv_len[b] += cu_keep[b+1] - cu_keep[b] where it fits in Lmax
     const int32_t* adv_cu_keep;
     int32_t* adv_kv_len;

@@ -484,3 +484,34 @@ extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nov
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }
+
+// Eq. 4 / Eq. 7 one step earlier: entropy of softmax(x W^T + b) without the logits ever reaching
+// HBM. The head GEMM runs on the tensor cores (CTA-pair kernel) and its epilogue threads, one row
+// each, carry the row's running maximum and sums across the column tiles.
+extern "C" nova_status nova_head_entropy(nova_ctx* ctx, const void* x, const void* w_head, const void* b_head,
+                                         int S, int N, int C, int V, float* ent, float* mean, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if (S < 0 || N < 0 || C < 1 || V < 1) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_head_entropy: bad sizes");
+    const long rows = (long)S * N;
+    if (rows == 0) return NOVA_OK;
+    if (rows > 0x7fffffffL) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_head_entropy: too many rows");
+    if (!x || !w_head || !ent) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_head_entropy: null pointer");
+    if (C % 64 || V % 32) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_head_entropy: C must be a multiple of 64 and V of 32");
+    if (!nova_aligned16(x) || !nova_aligned16(w_head) || !nova_aligned16(b_head))
+        return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_head_entropy: tensors must be 16-byte aligned");
+    cudaStream_t st = (cudaStream_t)stream;
+    nova_gemm_args g;
+    memset(&g, 0, sizeof(g));
+    g.A = (const __nv_bfloat16*)x; g.W = (const __nv_bfloat16*)w_head; g.bias = (const __nv_bfloat16*)b_head;
+    g.M = (int)rows; g.N = V; g.K = C;
+    g.epilogue = NOVA_EPI_ENTROPY; g.cat = NOVA_K_ENTROPY; g.ent = ent;
+    const nova_status rc = nova_launch_gemm(ctx, g, st);
+    if (rc) return rc;
+    if (mean) {
+        nova_launch_scope scope(ctx, NOVA_K_ENTROPY_MEAN, st);
+        entropy_mean<<<S, 1024, 0, st>>>(ent, N, mean);
+    }
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    return NOVA_OK;
+}

@@ -61,6 +61,7 @@ struct GemmParams {
     const int32_t* adv_cu_keep;
     int32_t* adv_kv_len;
     int adv_B, adv_Lmax;
+    float* ent;
 };
 
 // Advance of the K/V cache lengths, done by one warp-sized loop of the launch's first CTA.
@@ -241,6 +242,7 @@ GemmParams make_params(nova_ctx* ctx, const nova_gemm_args& a)
     p.res = a.res; p.res_row = a.res_row; p.C = a.C; p.k_cache = a.k_cache; p.v_cache = a.v_cache;
     p.kv_row = a.kv_row; p.status = ctx->dev_status;
     p.adv_cu_keep = a.adv_cu_keep; p.adv_kv_len = a.adv_kv_len; p.adv_B = a.adv_B; p.adv_Lmax = a.adv_Lmax;
+    p.ent = a.ent;
     return p;
 }
 
@@ -285,6 +287,129 @@ __device__ __forceinline__ PairTile decode_tile(int entry, int span, int tiles_f
     return t;
 }
 
+// Entry of the work list that pair `pair` handles as its `local`-th tile, or -1 past the end.
+// group == 0: entries pair, pair + num_pairs, ... (any tile to any pair). group > 0 (entropy
+// epilogue, group = tiles along N, N-fastest order): a pair takes whole row blocks, all their `group`
+// column tiles in turn, so that the epilogue threads can carry a row's softmax state across them.
+__device__ __forceinline__ int pair_entry(int local, int pair, int num_pairs, int num_tiles, int group)
+{
+    int e;
+    if (group == 0) e = pair + local * num_pairs;
+    else e = (pair + (local / group) * num_pairs) * group + local % group;
+    return e < num_tiles ? e : -1;
+}
+
+// ---- entropy epilogue: running softmax-entropy state of one output row ----------------------
+// m = reference maximum, s = sum e^{z-m}, u = sum (z-m) e^{z-m} in the log2 domain (m2 = m log2 e),
+// the sums as two partial sums per 64-bit register (packed fp32 arithmetic).
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+struct EntropyState {
+    float m, m2;
+    uint64_t s2, u2;
+    __device__ __forceinline__ void reset()
+    {
+        m = -INFINITY; m2 = -INFINITY;
+        s2 = pack_f32x2(0.f, 0.f);
+        u2 = s2;
+    }
+    // 32 more logits of the row (fp32 accumulators plus bias)
+    __device__ __forceinline__ void add_chunk(const uint32_t (&acc)[32], const __nv_bfloat16* bias)
+    {
+        constexpr float kLog2e = 1.4426950408889634f;
+        float z[32];
+        if (bias) {
+            const uint4* bias4 = (const uint4*)bias;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 b = bias4[i];
+                const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    z[i * 8 + j * 2] = __uint_as_float(acc[i * 8 + j * 2]) + __uint_as_float(bw[j] << 16);
+                    z[i * 8 + j * 2 + 1] = __uint_as_float(acc[i * 8 + j * 2 + 1]) + __uint_as_float(bw[j] & 0xffff0000u);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(acc[i]);
+        }
+        float cm = z[0];
+#pragma unroll
+        for (int i = 1; i < 32; ++i) cm = fmaxf(cm, z[i]);
+        if (cm > m) {
+            // raise the reference: both sums scale by f = e^{m - m'}, u also shifts by (m - m') s
+            const float shift = (m - cm) * kLog2e;          // -inf the first time: f = 0
+            const float f = ex2_approx(shift);
+            float s_lo, s_hi, u_lo, u_hi;
+            unpack_f32x2(s2, s_lo, s_hi);
+            unpack_f32x2(u2, u_lo, u_hi);
+            if (m == -INFINITY) { u_lo = u_hi = 0.f; }
+            else {
+                u_lo = (u_lo + shift * s_lo) * f;
+                u_hi = (u_hi + shift * s_hi) * f;
+            }
+            s2 = pack_f32x2(s_lo * f, s_hi * f);
+            u2 = pack_f32x2(u_lo, u_hi);
+            m = cm;
+            m2 = cm * kLog2e;
+        }
+        const uint64_t log2e2 = pack_f32x2(kLog2e, kLog2e), neg_m2 = pack_f32x2(-m2, -m2);
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+            const uint64_t d2 = fma_f32x2(pack_f32x2(z[i], z[i + 1]), log2e2, neg_m2);
+            float d0, d1;
+            unpack_f32x2(d2, d0, d1);
+            const uint64_t e2 = pack_f32x2(ex2_approx(d0), ex2_approx(d1));
+            s2 = add_f32x2(s2, e2);
+            u2 = fma_f32x2(d2, e2, u2);
+        }
+    }
+    // H = ln s - u/s (u in log2 units); non-finite inputs give NaN and flag the status word
+    __device__ __forceinline__ float finish(unsigned int* status) const
+    {
+        float s_lo, s_hi, u_lo, u_hi;
+        unpack_f32x2(s2, s_lo, s_hi);
+        unpack_f32x2(u2, u_lo, u_hi);
+        const float s = s_lo + s_hi, u = u_lo + u_hi;
+        float h = logf(s) - (u / s) * 0.6931471805599453f;
+        if (!(fabsf(m) < INFINITY) || !(fabsf(h) < INFINITY)) {
+            h = __int_as_float(0x7fc00000);
+            atomicOr(status, NOVA_DEV_NONFINITE);
+        } else if (h <= 0.f) {
+            h = 0.f;
+        }
+        return h;
+    }
+};
+
 // Role layout as in gemm_bf16_tn. Barriers (all in each CTA's shared memory at equal offsets):
 //   full[s]       leader's copy is used: one arrival (its own expect_tx) + the bytes of both CTAs
 //   empty[s]      each CTA's copy, signalled in both CTAs by the leader's tcgen05.commit
@@ -294,7 +419,7 @@ template <int BN, int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                   const __grid_constant__ CUtensorMap tmap_w_half, const GemmParams p, const int span,
-                  const int tiles_full, const int num_tiles)
+                  const int tiles_full, const int num_tiles, const int group)
 {
     using L = PairSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
@@ -340,7 +465,9 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (lane == 0) {
             long it = 0;                         // k-blocks issued so far over all tiles of this pair
             bool ok = true;
-            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            for (int local = 0; ok; ++local) {
+                const int tile = pair_entry(local, pair, num_pairs, num_tiles, group);
+                if (tile < 0) break;
                 const PairTile t = decode_tile<BN>(tile, span, tiles_full);
                 const int m0 = t.m0 + (int)rank * 128;
                 const int n0 = t.n0 + (int)rank * (t.bn / 2);
@@ -386,7 +513,9 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             uint32_t par = 0;
             int local = 0;
             bool ok = true;
-            for (int tile = first_tile; tile < num_tiles && ok; tile += step, ++local) {
+            for (; ok; ++local) {
+                const int tile = pair_entry(local, first_tile, step, num_tiles, group);
+                if (tile < 0) break;
                 const int a = local & 1;
                 if (local >= 2) {
                     ok = mbar_wait_warp(&acc_empty[a], (uint32_t)((local >> 1) - 1) & 1, abort_flag, p.status);
@@ -420,7 +549,11 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const uint32_t acc_empty_leader = map_to_cta(smem_u32(&acc_empty[0]), 0);
         int local = 0;
         bool ok = true;
-        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++local) {
+        EntropyState est;
+        est.reset();
+        for (; ok; ++local) {
+            const int tile = pair_entry(local, pair, num_pairs, num_tiles, group);
+            if (tile < 0) break;
             const int a = local & 1;
             const PairTile t = decode_tile<BN>(tile, span, tiles_full);
             const int row = t.m0 + (int)rank * 128 + q * 32 + lane;
@@ -443,7 +576,13 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 tmem_ld32(t_addr + (uint32_t)(c * 32), acc);
                 tmem_ld_wait();
                 if (!row_ok || col0 >= p.N) continue;
-                epilogue_chunk(p, row, col0, acc, res_base, kv_base);
+                if (p.epilogue == NOVA_EPI_ENTROPY) est.add_chunk(acc, p.bias ? p.bias + col0 : nullptr);
+                else epilogue_chunk(p, row, col0, acc, res_base, kv_base);
+            }
+            if (p.epilogue == NOVA_EPI_ENTROPY && t.n0 + BN >= p.N) {
+                // last column tile of this row block: the row's entropy is complete
+                if (row_ok) p.ent[row] = est.finish(p.status);
+                est.reset();
             }
             // this warp has read its part of the buffer: tell the leader's MMA thread
             tc_fence_before();
@@ -480,15 +619,19 @@ nova_status launch_pair(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
     GemmParams p = make_params(ctx, a);
     const int tiles_m = (a.M + kPairBM - 1) / kPairBM, tiles_n = (a.N + BN - 1) / BN;
     const int tiles = tiles_m * tiles_n;
-    const int pairs = min(tiles, ctx->num_sms / 2);
+    const bool entropy = (a.epilogue == NOVA_EPI_ENTROPY);
+    // the entropy epilogue hands whole row blocks to pairs; otherwise any tile goes to any pair
+    const int pairs = min(entropy ? tiles_m : tiles, ctx->num_sms / 2);
     // a last partial wave that would occupy at most half of the pairs runs as half-width tiles
     const int rem = tiles % pairs;
-    const int tiles_full = (rem > 0 && 2 * rem <= pairs) ? tiles - rem : tiles;
+    const int tiles_full = (!entropy && rem > 0 && 2 * rem <= pairs) ? tiles - rem : tiles;
     const int entries = tiles_full + 2 * (tiles - tiles_full);
     {
         nova_launch_scope scope(ctx, a.cat, st);
-        const int span = ((long)a.M >= (long)a.N) ? -tiles_n : tiles_m;   // sweep the smaller operand
-        kern<<<dim3(2 * pairs), kThreads, L::kTotal, st>>>(ta, tw, tw_half, p, span, tiles_full, entries);
+        // sweep the smaller operand; the entropy epilogue needs the N-fastest order
+        const int span = (entropy || (long)a.M >= (long)a.N) ? -tiles_n : tiles_m;
+        kern<<<dim3(2 * pairs), kThreads, L::kTotal, st>>>(ta, tw, tw_half, p, span, tiles_full, entries,
+                                                           entropy ? tiles_n : 0);
     }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
@@ -527,6 +670,10 @@ nova_status nova_launch_gemm(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_
     // CTA pairs with 256 x 256 tiles once there is at least one tile per pair of SMs; below that the
     // single-CTA 128 x 128 tiles spread a small problem over more SMs.
     const long tiles_pair = (long)((a.M + 255) / 256) * ((a.N + 255) / 256);
+    if (a.epilogue == NOVA_EPI_ENTROPY) {
+        if (ctx->num_sms < 2) return nova_fail(ctx, NOVA_ERR_SHAPE, "gemm: the entropy epilogue needs the CTA-pair kernel");
+        return launch_pair<256, 6>(ctx, a, st);
+    }
     if (tiles_pair >= ctx->num_sms / 2 && ctx->num_sms >= 2) return launch_pair<256, 6>(ctx, a, st);
     return launch<128, 3>(ctx, a, st);
 }

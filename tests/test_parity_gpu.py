@@ -164,6 +164,65 @@ def test_entropy_empty_and_bad_args(ctx):
     assert ei.value.status == 3
 
 
+# ------------------------------------------------------- entropy fused with the codebook head
+def _head_case(ctx, S, N, C, V, seed, bias=True, sample=None):
+    x = synth.activations(S, N, C, seed, DEV)
+    w = synth.randn_bf16((V, C), seed + 1, DEV, std=3.0 / math.sqrt(C))     # logits of a few units: entropies spread out
+    b = synth.randn_bf16((V,), seed + 2, DEV, std=1.0) if bias else None
+    ent = torch.full((S, N), float("nan"), dtype=torch.float32, device=DEV)
+    mean = torch.full((S,), float("nan"), dtype=torch.float32, device=DEV)
+    nova.nova_head_entropy(ctx, x, w, b, ent, mean)
+    assert ctx.device_status() == 0
+    got = ent.cpu().numpy()
+    assert np.isfinite(got).all()
+    bb = f32(b) if bias else None
+    if sample is None:
+        want, want_mean = oracle.head_entropy(f32(x), f32(w), bb)
+        assert np.abs(got - want).max() <= ENT_TOL
+        assert np.abs(mean.cpu().numpy() - want_mean).max() <= ENT_TOL
+        assert want.max() - want.min() > 0.05
+    else:
+        flat = f32(x).reshape(S * N, C)
+        want, _ = oracle.head_entropy(flat[sample][None], f32(w), bb)
+        assert np.abs(got.reshape(-1)[sample] - want[0]).max() <= ENT_TOL
+        # the means are the fixed-order means of the entropies the kernel wrote
+        assert np.abs(mean.cpu().numpy() - got.astype(np.float64).mean(axis=1)).max() <= 1e-4
+
+
+@pytest.mark.parametrize("S,N,C,V,bias", [
+    (2, 300, 256, 4096, True),       # 600 rows: three 256-row blocks, the last one partial
+    (1, 77, 128, 992, False),        # fewer rows than one block; V not a multiple of the 256-column tile
+    (3, 256, 512, 2048, True),
+])
+def test_head_entropy_matches_oracle(ctx, S, N, C, V, bias):
+    _head_case(ctx, S, N, C, V, seed=31, bias=bias)
+
+
+def test_head_entropy_full_size_sampled_rows(ctx):
+    """Batch 4 at 64 x 64 tokens, width 2048, V = 4096 (the benchmark's launch): sampled rows."""
+    rows = np.array([0, 127, 128, 255, 256, 4095, 4096, 8191, 12287, 12288, 16383])
+    _head_case(ctx, 4, 4096, 2048, 4096, seed=37, sample=rows)
+
+
+def test_head_entropy_closed_form_flag_and_bad_args(ctx):
+    S, N, C, V = 1, 64, 128, 512
+    x = synth.activations(S, N, C, 3, DEV)
+    ent = torch.empty((S, N), dtype=torch.float32, device=DEV)
+    nova.nova_head_entropy(ctx, x, torch.zeros((V, C), dtype=torch.bfloat16, device=DEV), None, ent)
+    assert np.abs(ent.cpu().numpy() - math.log(V)).max() <= ENT_TOL       # zero head -> uniform
+    x[0, 5, 7] = float("inf")
+    w = synth.randn_bf16((V, C), 4, DEV, std=0.1)
+    nova.nova_head_entropy(ctx, x, w, None, ent)
+    e = ent.cpu().numpy()[0]
+    assert np.isnan(e[5]) and np.isfinite(np.delete(e, 5)).all()
+    assert ctx.device_status() == 5
+    with pytest.raises(nova.NovaError) as ei:                             # C not a multiple of 64
+        nova.nova_head_entropy(ctx, synth.activations(1, 8, 96, 1, DEV),
+                               torch.zeros((V, 96), dtype=torch.bfloat16, device=DEV), None,
+                               torch.empty((1, 8), dtype=torch.float32, device=DEV))
+    assert ei.value.status == 2
+
+
 # ---------------------------------------------------------------------------- select
 @pytest.mark.parametrize("S,N", [(1, 1), (3, 33), (2, 256), (5, 1000), (2, 4096), (2, 16384)])
 def test_select_bit_exact(ctx, S, N):
