@@ -333,10 +333,20 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         uint32_t v_par = 0, k_par_next = (kKStages > 1) ? 0u : 1u;
         for (int j = 0; j < n_tiles_u && ok; ++j) {
             const bool more = j + 1 < n_tiles_u;
-            ok = mbar_wait_warp(&v_full[vs], v_par, abort_flag, p.status);
-            if (ok && more) ok = mbar_wait_warp(&k_full[ks_next], k_par_next, abort_flag, p.status);
+            // The three barriers this step starts with are tried together, so their shared-memory
+            // round trips overlap; whatever is not complete yet gets a bounded wait of its own.
+            {
+                const bool v_ok = mbar_try_wait(&v_full[vs], v_par);
+                const bool k_ok = more ? mbar_try_wait(&k_full[ks_next], k_par_next) : true;
+                const bool p_ok = mbar_try_wait(&p_full[0], j & 1);
+                if (!__all_sync(0xffffffffu, v_ok && k_ok && p_ok)) {
+                    ok = mbar_wait_warp(&v_full[vs], v_par, abort_flag, p.status);
+                    if (ok && more) ok = mbar_wait_warp(&k_full[ks_next], k_par_next, abort_flag, p.status);
+                    if (ok) ok = mbar_wait_warp(&p_full[0], j & 1, abort_flag, p.status);
+                }
+            }
             for (int t = 0; t < n_q && ok; ++t) {
-                ok = mbar_wait_warp(&p_full[t], j & 1, abort_flag, p.status);
+                if (t > 0) ok = mbar_wait_warp(&p_full[t], j & 1, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
                 issue_pv(t, vs, j == 0);
