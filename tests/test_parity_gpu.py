@@ -334,6 +334,26 @@ def test_restore_matches_oracle(ctx, B, hp, wp, h, w, C, keep_frac):
     assert torch.equal(x_out2, x_out)
 
 
+def test_restore_full_size_1024_shape(ctx):
+    """The benchmark's restore launch: batch 4, 64 x 64 tokens from a 48 x 48 residual cache, width
+    2048, half of the tokens kept; every output row against the oracle."""
+    B, hp, wp, h, w, C = 4, 48, 48, 64, 64, 2048
+    N = h * w
+    x = synth.activations(B, N, C, seed=41, device=DEV)
+    cache = synth.residual_cache(B, hp, wp, C, seed=42, device=DEV)
+    ent = torch.rand((B, N), generator=torch.Generator(device="cpu").manual_seed(43))
+    ks = [2048, 2048, 1999, 2100]
+    keep_idx, prune_idx, cu, _ = gpu_select(ctx, ent.to(DEV), ks)
+    M = sum(ks)
+    y = synth.randn_bf16((M, C), 44, DEV)
+    x_out = torch.full_like(x, float("nan"))
+    cache_out = torch.full_like(x, float("nan"))
+    nova.nova_restore_from_cache(ctx, x, y, keep_idx, prune_idx, cu, cache, h, w, x_out, cache_out)
+    wx, wc = oracle.restore_from_cache(f32(x), f32(y), keep_idx.cpu().numpy(), prune_idx.cpu().numpy(),
+                                       cu.cpu().numpy(), f32(cache), h, w)
+    assert _bf16_ulp_ok(f32(x_out), wx) and _bf16_ulp_ok(f32(cache_out), wc)
+
+
 # ----------------------------------------------------------------------------- block
 def _run_block(ctx, shape, weights, x, keep_idx, cu, k_cache, v_cache, kv_len, append=True):
     ctx.ensure_workspace(shape)
