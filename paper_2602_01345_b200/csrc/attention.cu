@@ -28,7 +28,11 @@ using namespace tc;
 constexpr int BQ = 128;        // query rows per tile (two tiles per CTA)
 constexpr int BKV = 128;       // keys per tile
 constexpr int kThreads = 384;     // warpgroup 0: producer + MMA issuer (+2 idle warps); 1, 2: softmax of tile A, B
-constexpr int kRegsLow = 64, kRegsHigh = 216;   // 128 * 64 + 256 * 216 <= 64 K registers
+// setmaxnreg.inc waits until the registers are there, and nothing bounds that wait: the split must
+// leave slack in the 64 K register file (128 * 64 + 256 * 216 = 63488; a split that used all
+// 65536 never got its registers and the kernel hung).
+constexpr int kRegsLow = 64, kRegsHigh = 216;
+static_assert(128 * kRegsLow + 256 * kRegsHigh <= 65536 - 2048, "keep slack for setmaxnreg.inc");
 constexpr int kSlabBytes = 128 * 128;   // [128 rows][64 bf16]
 constexpr float kRescaleThreshold = 8.f;   // in log2 units
 
