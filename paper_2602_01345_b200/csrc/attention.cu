@@ -58,6 +58,11 @@ struct AttnParams {
     __nv_bfloat16* o;
     int B, C, Lmax, n_heads, num_sms;
     float scale_log2e;     // (1 / sqrt(dh)) * log2(e)
+    // key-split of a last partial wave: per split item two partial results [2][256 rows][DH + 4]
+    // fp32 (unnormalised O row, reference maximum, sum) and a ticket counter; part == NULL: no split
+    float* part;
+    unsigned int* tickets;
+    int part_slots;
     unsigned int* status;
 };
 
@@ -155,19 +160,23 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     // ---- which (image, 256-row query block, head) is this CTA? ----------------------------
     // Work items are (head, query block), blocks fastest so that CTAs running together share K/V
     // in L2. All items cost the same, so a grid of T items runs in ceil(T / SMs) waves and the last
-    // wave may be nearly empty: when it would fill at most half of the SMs, its items are split
-    // into their two 128-row tiles, each run by a CTA of its own (one tile, no ping-pong), which
-    // cuts the last wave to roughly 60 % of a full one.
+    // wave may be nearly empty: when it would fill at most half of the SMs, each of its items is
+    // run by two CTAs, one per half of the keys. Both leave their unnormalised result (O row,
+    // reference maximum, sum) in scratch memory and draw a ticket; the one that draws the second
+    // ticket finds the other's result complete, merges the two and writes the output. Nobody
+    // waits for anybody.
     int units = 0;
     for (int i = 0; i < p.B; ++i) units += (p.cu_keep[i + 1] - p.cu_keep[i] + 2 * BQ - 1) / (2 * BQ);
     const int items = units * p.n_heads;
     const int rem = items % p.num_sms;
-    const int whole_items = (rem > 0 && 2 * rem <= p.num_sms) ? items - rem : items;
-    int item = blockIdx.x, half = -1;
+    const bool split = p.part && rem > 0 && 2 * rem <= p.num_sms && rem <= p.part_slots;
+    const int whole_items = split ? items - rem : items;
+    int item = blockIdx.x, khalf = -1, tail_slot = 0;
     if (item >= whole_items) {
         const int h = item - whole_items;
         item = whole_items + (h >> 1);
-        half = h & 1;
+        khalf = h & 1;
+        tail_slot = h >> 1;
     }
     if (item >= items) return;
     const int head = item / units;
@@ -179,15 +188,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         if (slot < blocks) { q_begin = c0 + slot * 2 * BQ; break; }
         slot -= blocks;
     }
-    int rows_valid = min(2 * BQ, k_b - slot * 2 * BQ);
-    if (half >= 0) {
-        q_begin += half * BQ;
-        rows_valid = min(BQ, rows_valid - half * BQ);
-        if (rows_valid <= 0) return;
-    }
+    const int rows_valid = min(2 * BQ, k_b - slot * 2 * BQ);
     const bool tile_b_active = rows_valid > BQ;
     const int n_keys = min(p.kv_len[b] + k_b, p.Lmax);
-    const int n_tiles = (n_keys + BKV - 1) / BKV;
+    const int n_tiles_all = (n_keys + BKV - 1) / BKV;
+    if (khalf >= 0 && n_tiles_all < 4) {      // too few key tiles to share: the first CTA takes them all
+        if (khalf == 1) return;
+        khalf = -1;
+    }
+    // this CTA's key tiles are jt0 .. jt0 + n_tiles - 1; loops below count j from 0
+    int jt0 = 0, n_tiles = n_tiles_all;
+    if (khalf == 0) n_tiles = (n_tiles_all + 1) / 2;
+    if (khalf == 1) { jt0 = (n_tiles_all + 1) / 2; n_tiles = n_tiles_all - jt0; }
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -202,6 +214,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint64_t* o_done = p_full + 2;                    // 1
     uint32_t* tmem_slot = (uint32_t*)(o_done + 1);
     __shared__ int abort_flag_s;
+    __shared__ int ticket_s;
     volatile int* abort_flag = &abort_flag_s;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -256,13 +269,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 uint8_t* k_dst = smem + L::kKOff + ks * L::kTileBytes;
                 mbar_arrive_expect_tx(&k_full[ks], L::kTileBytes);
                 for (int sl = 0; sl < kSlabs; ++sl)
-                    tma_load_3d(k_dst + sl * kSlabBytes, &tmap_k, &k_full[ks], head * DH + sl * 64, j * BKV, b);
+                    tma_load_3d(k_dst + sl * kSlabBytes, &tmap_k, &k_full[ks], head * DH + sl * 64, (jt0 + j) * BKV, b);
                 k_issued = j + 1;
                 if (j >= kVStages && !mbar_wait(&v_empty[vs], ((j / kVStages) - 1) & 1, abort_flag, p.status)) break;
                 uint8_t* v_dst = smem + L::kVOff + vs * L::kTileBytes;
                 mbar_arrive_expect_tx(&v_full[vs], L::kTileBytes);
                 for (int sl = 0; sl < kSlabs; ++sl)
-                    tma_load_3d(v_dst + sl * kSlabBytes, &tmap_v, &v_full[vs], head * DH + sl * 64, j * BKV, b);
+                    tma_load_3d(v_dst + sl * kSlabBytes, &tmap_v, &v_full[vs], head * DH + sl * 64, (jt0 + j) * BKV, b);
                 v_issued = j + 1;
             }
             if (*abort_flag) {
@@ -388,7 +401,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 ok = mbar_wait_warp(&s_full[t], j & 1, abort_flag, p.status);
                 if (!ok) break;
                 tc_fence_after();
-                const int cols_valid = n_keys - j * BKV;      // >= 1; < BKV only on a ragged last tile
+                const int cols_valid = n_keys - (jt0 + j) * BKV;      // >= 1; < BKV only on a ragged last tile
                 // the whole row of S (128 scores) into registers with one round trip to tensor memory
                 uint32_t sv[128];
 #pragma unroll
@@ -479,11 +492,11 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 mbar_arrive(&p_full[t]);
             }
             if (ok) ok = mbar_wait_warp(o_done, 0, abort_flag, p.status);
-            if (ok) {
+            const int grow = t * BQ + row;
+            __nv_bfloat16* dst_row = p.o + (long)(q_begin + grow) * p.C + head * DH;
+            if (ok && khalf < 0) {
                 tc_fence_after();
                 const float inv = 1.f / l_run;
-                const int grow = t * BQ + row;
-                __nv_bfloat16* dst_row = p.o + (long)(q_begin + grow) * p.C + head * DH;
 #pragma unroll
                 for (int cch = 0; cch < DH / 32; ++cch) {
                     uint32_t ov[32];
@@ -498,6 +511,64 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                                 pack_bf16(__uint_as_float(ov[g * 8 + 2]) * inv, __uint_as_float(ov[g * 8 + 3]) * inv),
                                 pack_bf16(__uint_as_float(ov[g * 8 + 4]) * inv, __uint_as_float(ov[g * 8 + 5]) * inv),
                                 pack_bf16(__uint_as_float(ov[g * 8 + 6]) * inv, __uint_as_float(ov[g * 8 + 7]) * inv));
+                    }
+                }
+            } else if (khalf >= 0) {
+                // ---- half of the keys: publish the partial result, then merge if the other is there
+                // (all softmax threads of the CTA take part, also after a failed wait, so that the
+                // named barrier below is complete; a failed CTA publishes nothing useful and the
+                // status word says so)
+                constexpr int kStride = DH + 4;
+                float* mine = p.part + ((size_t)(tail_slot * 2 + khalf) * (2 * BQ) + grow) * kStride;
+                const float* other = p.part + ((size_t)(tail_slot * 2 + (khalf ^ 1)) * (2 * BQ) + grow) * kStride;
+                if (ok) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int cch = 0; cch < DH / 32; ++cch) {
+                        uint32_t ov[32];
+                        tmem_ld32(o_addr + cch * 32, ov);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            *(uint4*)(mine + cch * 32 + g * 4) = make_uint4(ov[g * 4], ov[g * 4 + 1], ov[g * 4 + 2], ov[g * 4 + 3]);
+                    }
+                    mine[DH] = m_ref;
+                    mine[DH + 1] = l_run;
+                }
+                __threadfence();
+                const int n_soft = tile_b_active ? 256 : 128;
+                asm volatile("bar.sync 1, %0;" ::"r"(n_soft) : "memory");
+                if (threadIdx.x == 128) {
+                    const unsigned int ticket = atomicAdd(&p.tickets[tail_slot], 1u);
+                    if (ticket == 1u) p.tickets[tail_slot] = 0;          // ready for the next launch
+                    ticket_s = (int)ticket;
+                }
+                asm volatile("bar.sync 1, %0;" ::"r"(n_soft) : "memory");
+                if (ok && ticket_s == 1) {
+                    // the other CTA fenced its partial result before it drew ticket 0
+                    const float m_o = __ldcg(other + DH), l_o = __ldcg(other + DH + 1);
+                    const float m_new = fmaxf(m_ref, m_o);
+                    const float a_me = ex2((m_ref - m_new) * c), a_o = ex2((m_o - m_new) * c);
+                    const float inv = 1.f / (l_run * a_me + l_o * a_o);
+                    const float w_me = a_me * inv, w_o = a_o * inv;
+#pragma unroll
+                    for (int cch = 0; cch < DH / 32; ++cch) {
+                        uint32_t ov[32];
+                        tmem_ld32(o_addr + cch * 32, ov);
+                        tmem_ld_wait();
+                        if (grow < rows_valid) {
+                            uint4* dst = (uint4*)(dst_row + cch * 32);
+#pragma unroll
+                            for (int g = 0; g < 4; ++g) {
+                                const float4 o0 = __ldcg((const float4*)(other + cch * 32 + g * 8));
+                                const float4 o1 = __ldcg((const float4*)(other + cch * 32 + g * 8 + 4));
+                                dst[g] = make_uint4(
+                                    pack_bf16(__uint_as_float(ov[g * 8]) * w_me + o0.x * w_o, __uint_as_float(ov[g * 8 + 1]) * w_me + o0.y * w_o),
+                                    pack_bf16(__uint_as_float(ov[g * 8 + 2]) * w_me + o0.z * w_o, __uint_as_float(ov[g * 8 + 3]) * w_me + o0.w * w_o),
+                                    pack_bf16(__uint_as_float(ov[g * 8 + 4]) * w_me + o1.x * w_o, __uint_as_float(ov[g * 8 + 5]) * w_me + o1.y * w_o),
+                                    pack_bf16(__uint_as_float(ov[g * 8 + 6]) * w_me + o1.z * w_o, __uint_as_float(ov[g * 8 + 7]) * w_me + o1.w * w_o));
+                            }
+                        }
                     }
                 }
             }
@@ -533,6 +604,12 @@ nova_status launch(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st)
     p.scale_log2e = (float)((1.0 / sqrt((double)DH)) * 1.4426950408889634);
     p.status = ctx->dev_status;
     p.n_heads = a.n_heads; p.num_sms = ctx->num_sms;
+    // scratch for a key-split last wave: [slots][2][256][DH + 4] fp32; tickets live in the context's
+    // status allocation (zero at creation, reset by the CTA that draws the second ticket)
+    const size_t slot_bytes = (size_t)2 * 2 * BQ * (DH + 4) * sizeof(float);
+    p.part = (float*)a.scratch;
+    p.part_slots = a.scratch ? (int)min((size_t)NOVA_ATTN_TICKETS, a.scratch_bytes / slot_bytes) : 0;
+    p.tickets = ctx->dev_status + NOVA_ATTN_TICKET_WORD0;
     // upper bound of the work items (the kept counts per image live on the device) plus the CTAs a
     // split last wave adds; CTAs past the end return at once
     dim3 grid(((a.M + 2 * BQ - 1) / (2 * BQ) + a.B) * a.n_heads + ctx->num_sms / 2);

@@ -17,9 +17,11 @@
 #define NOVA_DEV_SHAPE     4u
 
 // Layout of the context's one device allocation: NOVA_STATUS_WORDS 32-bit words (word 0 = status
-// bits, word 1 = completion counter of the entropy kernel), then the per-CTA partial sums of the
+// bits, word 1 = completion counter of the entropy kernel, words 16.. = attention tickets), then the per-CTA partial sums of the
 // entropy means, float[NOVA_MEAN_MAX_CTAS][NOVA_MEAN_MAX_SEGMENTS].
-#define NOVA_STATUS_WORDS 64
+#define NOVA_STATUS_WORDS 128
+#define NOVA_ATTN_TICKET_WORD0 16     // words 16 .. 16 + NOVA_ATTN_TICKETS - 1: tickets of key-split attention items
+#define NOVA_ATTN_TICKETS 96
 #define NOVA_MEAN_MAX_CTAS 192
 #define NOVA_MEAN_MAX_SEGMENTS 256
 #define NOVA_STATUS_BYTES (NOVA_STATUS_WORDS * 4 + NOVA_MEAN_MAX_CTAS * NOVA_MEAN_MAX_SEGMENTS * 4)
@@ -147,6 +149,8 @@ struct nova_attn_args {
     const int32_t* kv_len;         // [B] length before this call's rows
     __nv_bfloat16* o;              // [M, C]
     int B, C, n_heads, Lmax, M;
+    void* scratch;                 // device memory free during the launch (or NULL) for a key-split last wave
+    size_t scratch_bytes;
 };
 
 nova_status nova_launch_attention(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st);

@@ -453,6 +453,15 @@ def test_block_attention_ragged_mid_size(ctx):
                 rows=np.array(rows, np.int32))
 
 
+def test_block_1024_shape_batch1_keep025_sampled_rows(ctx):
+    """One image of the 1024x1024 shape at keep ratio 0.25: 1024 kept rows give only 64 attention work
+    items for 148 SMs, so every item is shared by two CTAs (one per half of the keys) whose partial
+    results are merged by whichever finishes second."""
+    rows = [0, 127, 128, 255, 256, 511, 512, 767, 768, 1023]
+    _block_case(ctx, B=1, N=4096, C=2048, heads=16, F=8192, Lmax=10521, ks=[1024], kv_lens=[6425], seed=47,
+                rows=np.array(rows, np.int32))
+
+
 def test_block_512_shape_sampled_rows(ctx):
     """VAR-d30-shaped 512x512 block: width 1920, 30 heads x 64, MLP 7680, last scale 32x32 over 1216
     prior tokens, batch 4, ragged keep counts. Widths that are not multiples of 256 (partial GEMM
