@@ -35,7 +35,7 @@ UNIT = "images/s"
 # for any other workload, and reset to None whenever the kernel changes after the capture.
 # attention: one launch; gemm: average over the four launches of a layer (qkv, proj, fc1, fc2), the
 # unit `achieved` is taken over as well. Source: profiles/layer_kernels_c4_1024_batch4_keep0.5.txt.
-NCU_TRAFFIC_BYTES = {"attention": 347_592_448, "gemm": 172_289_408}
+NCU_TRAFFIC_BYTES = {"attention": 351_096_576, "gemm": 171_372_416}
 
 
 def parse_args():
@@ -414,6 +414,8 @@ def oracle_sample(wd, st, keeps, rows_entropy=1024, rows_block=8):
     x = f32(st["x_in"][0:1])
     kc, vc = f32(st["k_caches"][0][0:1]), f32(st["v_caches"][0][0:1])
     kv_len = np.array([wd["P"]], np.int32)
+    # first call untimed: it also pays for the first touch of the converted K/V caches
+    oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=np.zeros(0, np.int32))
     t0 = time.perf_counter()
     oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=np.zeros(0, np.int32))
     t["block_kv"] = time.perf_counter() - t0
