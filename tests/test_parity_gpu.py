@@ -462,6 +462,15 @@ def test_block_1024_shape_batch1_keep025_sampled_rows(ctx):
                 rows=np.array(rows, np.int32))
 
 
+@pytest.mark.parametrize("kv_len", [517, 5])
+def test_block_key_split_small_cases(ctx, kv_len):
+    """Four attention work items on 148 SMs, so each is shared by two CTAs, one per half of the keys.
+    The second query block has 44 rows (only one of its two query tiles in use). With 517 prior keys
+    there are 7 key tiles (4 + 3, the last one ragged); with 5 there are only 3, too few to share, and
+    the first CTA of each pair does all the work."""
+    _block_case(ctx, B=1, N=600, C=256, heads=2, F=2048, Lmax=1024, ks=[300], kv_lens=[kv_len], seed=53)
+
+
 def test_block_512_shape_sampled_rows(ctx):
     """VAR-d30-shaped 512x512 block: width 1920, 30 heads x 64, MLP 7680, last scale 32x32 over 1216
     prior tokens, batch 4, ragged keep counts. Widths that are not multiples of 256 (partial GEMM
