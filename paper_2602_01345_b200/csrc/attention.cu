@@ -3,7 +3,8 @@
 //
 // One CTA = 256 query rows (two 128-row tiles A and B) of one image and one head, streaming
 // over 128-key tiles of K and V:
-//   warp 0        TMA producer: Q tiles once, then a ring of {K tile, V tile} stages
+//   warp 0        TMA producer: Q tiles once, then a ring of K tiles and a ring of V tiles
+//   warps 2-3     idle (they fill the producer/issuer warpgroup, which gives up registers)
 //   warp 1        tcgen05.mma issuer. Per key tile j:  O_A += P_A V_j ; S_A = Q_A K_{j+1}^T ;
 //                 O_B += P_B V_j ; S_B = Q_B K_{j+1}^T.  S and O are fp32 in tensor memory and
 //                 O accumulates there across all key tiles.
@@ -18,6 +19,8 @@
 // the MN-major B operand, i.e. V is consumed exactly as it lies in the cache ([keys, dh]).
 // MMAs issued by one thread execute in issue order, which orders "P_A read by O_A += P_A V" before
 // "S_A overwritten by the next Q_A K^T" and "O complete" before the next S of the same tile.
+// When the grid's last wave would be less than half full, each of its work items is shared by
+// two CTAs that take half of the key tiles each and merge their partial results (see below).
 // Every mbarrier wait is bounded.
 #include "tc_common.cuh"
 
