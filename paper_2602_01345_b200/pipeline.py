@@ -96,6 +96,50 @@ class PrunedScaleRunner:
         return x, keeps
 
 
+class MultiScaleRunner:
+    """All scales of one generation, in order: the state NOVA carries from scale to scale.
+
+    Per layer it owns the K/V caches (every scale appends the kept tokens' keys and values), the
+    residual cache written at the previous scale (Eq. 15; read, resized, at the next one, Eq. 16)
+    and, per image, the history of scale mean entropies that the trigger of Eq. 8-10 works on. A
+    scale that is not pruned yet is simply the same call sequence with every token kept.
+    The backbone around the layers (token embedding, sampling) is not part of this library: the
+    caller supplies each scale's layer input and logits.
+    """
+
+    def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, scales, eps: float = 1e-6):
+        self.ctx, self.weights, self.n_heads, self.B, self.eps = ctx, weights, n_heads, B, eps
+        self.scales = tuple(scales)
+        self.L = len(weights)
+        self.C = weights[0]["w_o"].shape[0]
+        self.Lmax = sum(s * s for s in self.scales)
+        dev = weights[0]["w_o"].device
+        self.k_caches = [torch.zeros((B, self.Lmax, self.C), dtype=torch.bfloat16, device=dev) for _ in range(self.L)]
+        self.v_caches = [torch.zeros((B, self.Lmax, self.C), dtype=torch.bfloat16, device=dev) for _ in range(self.L)]
+        self.kv_len = torch.zeros((self.L, B), dtype=torch.int32, device=dev)
+        self.res_cache = [None] * self.L          # previous scale's residual cache per layer, [B, h, w, C]
+        self.hbar_scale = torch.zeros((B, 0), dtype=torch.float32)
+        self._ent = None
+
+    def run_scale(self, t: int, x_in, scale_logits, layer_logits, sched: nv.SchedParams, stream=None):
+        """Scale t (1-based, in order). scale_logits [B, N_t, V] give the scale's mean entropy
+        (Eq. 7) that extends the history; layer_logits: L tensors [B, N_t, V]. Returns
+        (x_out, keeps, runner) where runner is the PrunedScaleRunner that ran the layers."""
+        assert t == self.hbar_scale.shape[1] + 1, "scales must be run in order"
+        side = self.scales[t - 1]
+        B, N = self.B, side * side
+        st = stream if stream is not None else torch.cuda.current_stream()
+        ent = torch.empty((B, N), dtype=torch.float32, device=x_in.device)
+        mean = torch.empty((B,), dtype=torch.float32, device=x_in.device)
+        nv.nova_scale_entropy(self.ctx, scale_logits, ent, mean, stream=st)
+        self.hbar_scale = torch.cat([self.hbar_scale, mean.cpu().view(B, 1)], dim=1)
+        runner = PrunedScaleRunner(self.ctx, self.weights, self.n_heads, B, side, side, self.Lmax, self.k_caches,
+                                   self.v_caches, self.kv_len, self.res_cache, eps=self.eps)
+        x_out, keeps = runner.run_scale(x_in, layer_logits, sched, t, self.hbar_scale.contiguous(), stream=st)
+        self.res_cache = [c.view(B, side, side, self.C) for c in runner.cache_out]
+        return x_out, keeps, runner
+
+
 def launch_count(ctx: nv.Context) -> int:
     nv._lib.nova_launch_count.restype = C.c_ulonglong
     nv._lib.nova_launch_count.argtypes = [C.c_void_p]

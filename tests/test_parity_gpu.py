@@ -637,3 +637,71 @@ def test_pipeline_literal_schedule_256_shape(ctx):
     # free-running over three layers: bf16 storage between stages on the GPU, fp32 in the oracle
     assert _rel_err(f32(x_out), x_ref) <= BLOCK_TOL
     assert kv_len.cpu().tolist() == [[P + int(k) for k in keeps[j].tolist()] for j in range(L)]
+
+
+def test_multi_scale_generation_256_shape(ctx):
+    """All ten scales of the VAR-d16 256x256 schedule (1, 2, 3, 4, 5, 6, 8, 10, 13, 16) through two
+    layers for two images, with the paper's hyper-parameters and nothing forced: mean entropies that
+    follow a seeded sigmoid per image, so the inflection test of Eq. 8-10 fires at a seed-determined
+    scale; from the scale after it tokens are pruned by Eq. 11-13; K/V caches grow scale by scale and
+    each scale's residual cache (Eq. 15) fills the next scale's pruned rows (Eq. 16). The oracle runs
+    the same generation with its own caches; decisions (inflection scale, keep counts, index lists)
+    are taken on the entropies the GPU measured and must agree exactly."""
+    from paper_2602_01345_b200 import pipeline
+    ms = synth.CONFIGS["c2_var_d16_256"]
+    B, L, T = 2, 2, len(ms.scales)
+    C, Lmax = ms.C, ms.total_tokens
+    weights = [synth.block_weights(C, ms.F, 100 + j, DEV) for j in range(L)]
+    wts = [{n: f32(v) for n, v in weights[j].items()} for j in range(L)]
+    a_env, _ = synth.scale_envelope_temperatures(B, T, seed=3)
+    beta = synth.layer_inverse_temperatures(L, 3)
+    gen = pipeline.MultiScaleRunner(ctx, weights, ms.heads, B, ms.scales)
+    sched, osched = nova.SchedParams(), oracle.SchedParams()
+    # the oracle's own state
+    ok_cache = [np.zeros((B, Lmax, C), np.float32) for _ in range(L)]
+    ov_cache = [np.zeros((B, Lmax, C), np.float32) for _ in range(L)]
+    o_len = np.zeros((L, B), np.int32)
+    o_res = [None] * L
+    pruned_scales = 0
+    for t in range(1, T + 1):
+        side = ms.scales[t - 1]
+        N = side * side
+        x_in = synth.activations(B, N, C, 200 + t, DEV)
+        a = a_env[:, t - 1].view(B, 1).expand(B, N).contiguous().to(DEV)
+        scale_logits = synth.logits_from_temperature(a, synth.V_CODEBOOK, 300 + t)
+        layer_logits = [synth.logits_from_temperature(a * float(beta[j]), synth.V_CODEBOOK, 400 + 10 * t + j)
+                        for j in range(L)]
+        x_out, keeps, runner = gen.run_scale(t, x_in, scale_logits, layer_logits, sched)
+        assert ctx.device_status() == 0
+        hist = gen.hbar_scale.numpy()
+        _, w_mean = oracle.scale_entropy(f32(scale_logits))
+        assert np.abs(hist[:, t - 1] - w_mean).max() <= ENT_TOL
+        x_ref = f32(x_in)
+        hbar_layer = np.zeros((B, L), np.float32)
+        for j in range(L):
+            ent_gpu = runner.ent[j].cpu().numpy()
+            hbar_layer[:, j] = runner.mean[j].cpu().numpy()
+            wr = oracle.keep_ratios(osched, t, j + 1, N, hist.copy(), hbar_layer[:, : j + 1].copy())
+            assert np.array_equal(keeps[j].numpy(), wr["keep"]), (t, j)
+            w_keep, w_prune, w_cu, _ = oracle.select_topk(ent_gpu, wr["keep"])
+            wy, wk, wv = oracle.pruned_block_forward(wts[j], 1e-6, ms.heads, x_ref, w_keep, w_cu,
+                                                     ok_cache[j], ov_cache[j], o_len[j].copy())
+            for b in range(B):
+                kb = int(wr["keep"][b])
+                ok_cache[j][b, o_len[j, b]:o_len[j, b] + kb] = wk[w_cu[b]:w_cu[b + 1]]
+                ov_cache[j][b, o_len[j, b]:o_len[j, b] + kb] = wv[w_cu[b]:w_cu[b + 1]]
+                o_len[j, b] += kb
+            prev = o_res[j] if o_res[j] is not None else np.zeros((B, 1, 1, C), np.float32)
+            x_ref, o_res_new = oracle.restore_from_cache(x_ref, wy, w_keep, w_prune, w_cu, prev, side, side)
+            o_res[j] = o_res_new.reshape(B, side, side, C)
+            if (wr["keep"] < N).any():
+                pruned_scales += 1 if j == 0 else 0
+        assert _rel_err(f32(x_out), x_ref) <= BLOCK_TOL, t
+        assert gen.kv_len.cpu().numpy().tolist() == o_len.tolist()
+    final = oracle.keep_ratios(osched, T, 1, ms.scales[-1] ** 2, gen.hbar_scale.numpy())
+    assert (final["act_scale"] > 0).any() and (final["act_scale"] <= T).any()     # the trigger fired in time
+    assert pruned_scales >= 1                                                      # and scales were pruned
+    # the caches the GPU carried agree with the oracle's after all scales
+    for j in range(L):
+        assert _rel_err(f32(gen.k_caches[j]), ok_cache[j]) <= BLOCK_TOL
+        assert _rel_err(f32(gen.res_cache[j]), o_res[j]) <= BLOCK_TOL
