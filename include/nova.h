@@ -11,6 +11,7 @@
  *   nova_select_topk        text after Eq. 3 / Eq. 13: keep the highest-entropy tokens
  *   nova_pruned_block_forward   Eq. 14     the layer on the kept tokens only
  *   nova_restore_from_cache     Eq. 15-16  fill pruned rows from the residual cache
+ *   nova_*_device               the same steps with the keep counts left on the device
  *
  * General rules
  *  - Plain C ABI. No call throws, aborts or traps the GPU. Every call returns a
@@ -264,6 +265,48 @@ nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, const void*
                                     const int32_t* cu_keep, const void* cache_prev,
                                     int hp, int wp, int h, int w, int C, int B, int M,
                                     void* x_out, void* cache_out, void* stream);
+
+/* ---- the same steps driven from the device: no host value between the calls of a layer ----- */
+/*
+ * (The paper fixes what is computed, not where the keep counts live; these calls exist so that a
+ * whole scale - every layer's entropy, Eq. 8-13, selection, Eq. 14 and Eq. 15-16 - can be enqueued
+ * without a host synchronisation and captured once in a CUDA graph.)
+ * They enqueue work only; nothing is read back. Results equal those of the host-driven calls.
+ *
+ * nova_keep_ratios_device: Eq. 8-13 exactly as nova_keep_ratios, one device thread per image, in
+ *   double. The exp and tanh of Eq. 11 come from the device's math library instead of the host's,
+ *   so a ratio may differ in its last bit; a keep count differs only if ratio * N_t lies within
+ *   that bit of an integer.
+ *   hbar_scale: device f32 [t, B] (row u-1 = the means of scale u, as nova_scale_entropy writes
+ *   them; note the transposed layout); hbar_layer: device f32 [j, B] or NULL when j == 1;
+ *   t_star, act_scale: device int32 [B] or NULL; keep: device int32 [B]. p is host memory, copied
+ *   at the call.
+ * nova_select_topk_device: nova_select_topk with k in device memory (int32 [S], values clamped to
+ *   [0, N]); keep_idx and prune_idx must both hold S*N entries' worth of space. S <= 65535.
+ * nova_pruned_block_forward_device: nova_pruned_block_forward where s->M is only an upper bound of
+ *   the kept rows (it sizes launches, y_kept and the workspace: pass B*N if nothing better is
+ *   known); the true count is cu_keep[B], read on the device. Rows of y_kept past it are untouched.
+ * nova_restore_from_cache_device: nova_restore_from_cache with the kept count read from
+ *   cu_keep[B]; cache_prev is always required (a 1 x 1 map of zeros serves before the first cache
+ *   exists, when nothing can be pruned).
+ * Errors as for the host-driven calls.
+ */
+nova_status nova_keep_ratios_device(nova_ctx* ctx, const nova_sched_params* p, int B, int t, int j, int N_t,
+                                    const float* hbar_scale, const float* hbar_layer,
+                                    int32_t* t_star, int32_t* act_scale, int32_t* keep, void* stream);
+nova_status nova_select_topk_device(nova_ctx* ctx, const float* ent, int S, int N, const int32_t* k_dev,
+                                    int32_t* keep_idx, int32_t* prune_idx, int32_t* cu_keep,
+                                    int32_t* pos, void* stream);
+nova_status nova_pruned_block_forward_device(nova_ctx* ctx, const nova_block_weights* w,
+                                             const nova_block_shape* s, const void* x_in,
+                                             const int32_t* keep_idx, const int32_t* cu_keep,
+                                             void* k_cache, void* v_cache, int32_t* kv_len,
+                                             int append_kv, void* y_kept, void* stream);
+nova_status nova_restore_from_cache_device(nova_ctx* ctx, const void* x_in, const void* y_kept,
+                                           const int32_t* keep_idx, const int32_t* prune_idx,
+                                           const int32_t* cu_keep, const void* cache_prev,
+                                           int hp, int wp, int h, int w, int C, int B,
+                                           void* x_out, void* cache_out, void* stream);
 
 #ifdef __cplusplus
 }

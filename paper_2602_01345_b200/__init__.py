@@ -9,5 +9,7 @@ from .binding import (  # noqa: F401
     nova_scale_entropy, nova_head_entropy, nova_keep_ratios, nova_select_topk,
     nova_pruned_block_forward, nova_restore_from_cache, nova_block_workspace_bytes,
     nova_pruned_block_forward_static, nova_static_scratch_bytes,
+    nova_keep_ratios_device, nova_select_topk_device, nova_pruned_block_forward_device,
+    nova_restore_from_cache_device,
     lib_path, STATUS_NAMES,
 )

@@ -287,3 +287,59 @@ def nova_pruned_block_forward_static(ctx: Context, w: BlockWeights, shape: Block
         ctx.check(_lib.nova_pruned_block_forward_static(
             ctx.handle, C.byref(w.c), C.byref(c), _ptr(x_in), _ptr(keep_idx), _ptr(cu_keep), _ptr(k_cache),
             _ptr(v_cache), _ptr(kv_len), int(bool(append_kv)), _ptr(y_kept), _stream(stream)))
+
+
+# ---- the device-driven variants: nothing crosses to the host between the calls of a layer -----
+_lib.nova_keep_ratios_device.argtypes = [_vp, C.POINTER(_SchedParams), _i, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.nova_keep_ratios_device.restype = _i
+_lib.nova_select_topk_device.argtypes = _lib.nova_select_topk.argtypes
+_lib.nova_select_topk_device.restype = _i
+_lib.nova_pruned_block_forward_device.argtypes = _lib.nova_pruned_block_forward.argtypes
+_lib.nova_pruned_block_forward_device.restype = _i
+_lib.nova_restore_from_cache_device.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp]
+_lib.nova_restore_from_cache_device.restype = _i
+
+
+def nova_keep_ratios_device(ctx: Context, p: SchedParams, t: int, j: int, N_t: int, hbar_scale, hbar_layer, keep,
+                            t_star=None, act_scale=None, stream=None):
+    """Eq. 8-13 on the device. hbar_scale: device f32 [t, B]; hbar_layer: device f32 [j, B] or None;
+    keep (and optionally t_star, act_scale): device int32 [B]."""
+    B = keep.numel()
+    assert hbar_scale.dtype == torch.float32 and hbar_scale.shape == (t, B)
+    assert hbar_layer is None or (hbar_layer.dtype == torch.float32 and hbar_layer.shape == (j, B))
+    assert keep.dtype == torch.int32
+    c = p._c()
+    ctx.check(_lib.nova_keep_ratios_device(ctx.handle, C.byref(c), B, t, j, N_t, _ptr(hbar_scale), _ptr(hbar_layer),
+                                           _ptr(t_star), _ptr(act_scale), _ptr(keep), _stream(stream)))
+
+
+def nova_select_topk_device(ctx: Context, ent, k_dev, keep_idx, prune_idx, cu_keep, pos=None, stream=None):
+    """nova_select_topk with the keep counts in a device int32 tensor [S]; keep_idx and prune_idx
+    must each have room for S*N entries."""
+    S, N = ent.shape
+    assert ent.dtype == torch.float32 and ent.is_contiguous()
+    assert k_dev.dtype == torch.int32 and k_dev.numel() == S and k_dev.is_cuda
+    assert keep_idx.numel() >= S * N and prune_idx.numel() >= S * N
+    ctx.check(_lib.nova_select_topk_device(ctx.handle, _ptr(ent), S, N, _ptr(k_dev), _ptr(keep_idx), _ptr(prune_idx),
+                                           _ptr(cu_keep), _ptr(pos), _stream(stream)))
+
+
+def nova_pruned_block_forward_device(ctx: Context, w: BlockWeights, shape: BlockShape, x_in, keep_idx, cu_keep,
+                                     k_cache, v_cache, kv_len, append_kv, y_kept, stream=None):
+    """nova_pruned_block_forward where shape.M is an upper bound; the true count is cu_keep[B]."""
+    c = shape._c()
+    assert y_kept.shape[0] >= shape.M
+    ctx.check(_lib.nova_pruned_block_forward_device(ctx.handle, C.byref(w.c), C.byref(c), _ptr(x_in), _ptr(keep_idx),
+                                                    _ptr(cu_keep), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len),
+                                                    int(bool(append_kv)), _ptr(y_kept), _stream(stream)))
+
+
+def nova_restore_from_cache_device(ctx: Context, x_in, y_kept, keep_idx, prune_idx, cu_keep, cache_prev, h, w,
+                                   x_out, cache_out=None, stream=None):
+    """nova_restore_from_cache with the kept count read from cu_keep[B] on the device."""
+    B, N, Cc = x_in.shape
+    assert N == h * w and cache_prev is not None
+    ctx.check(_lib.nova_restore_from_cache_device(ctx.handle, _ptr(x_in), _ptr(y_kept), _ptr(keep_idx),
+                                                  _ptr(prune_idx), _ptr(cu_keep), _ptr(cache_prev),
+                                                  cache_prev.shape[1], cache_prev.shape[2], h, w, Cc, B,
+                                                  _ptr(x_out), _ptr(cache_out), _stream(stream)))

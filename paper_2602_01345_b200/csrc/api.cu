@@ -78,7 +78,7 @@ const char* nova_profile_category_name(int cat)
 {
     static const char* names[NOVA_K_COUNT] = {
         "entropy_rows", "entropy_mean", "select_topk", "layernorm", "gemm_qkv",
-        "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "restore"};
+        "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "restore", "keep_ratios"};
     return (cat >= 0 && cat < NOVA_K_COUNT) ? names[cat] : "?";
 }
 
@@ -147,11 +147,15 @@ void nova_sched_params_default(nova_sched_params* p)
     p->force_keep_ratio = -1.0;
 }
 
-// Eq. 8-13 for one image. hs[u-1] is the mean entropy of scale u; hl[k-1] that of layer k.
-static void schedule_one(const nova_sched_params& p, int t, int j, int n_tokens, const float* hs,
-                         const float* hl, int32_t* t_star, int32_t* act_scale, double* ratio_scale,
-                         double* ratio_layer, int32_t* keep)
+// Eq. 8-13 for one image. HS(u) is the mean entropy of scale u, HL(k) that of layer k; the
+// histories are strided so that the host layout [B, t] and the device layout [t, B] share the code.
+static __host__ __device__ void schedule_one(const nova_sched_params& p, int t, int j, int n_tokens,
+                                             const float* hs_base, long hs_stride, const float* hl_base, long hl_stride,
+                                             int32_t* t_star, int32_t* act_scale, double* ratio_scale,
+                                             double* ratio_layer, int32_t* keep)
 {
+#define HS(u) ((double)hs_base[((u) - 1) * hs_stride])
+#define HL(k) ((double)hl_base[((k) - 1) * hl_stride])
     // growth rates g[u] for u = 2..t (Eq. 8)
     double growth_now = 0.0;
     int found = 0;
@@ -159,12 +163,12 @@ static void schedule_one(const nova_sched_params& p, int t, int j, int n_tokens,
         // baseline: the growth rates up to t_est telescope, but are summed one by one so the
         // rounding matches a term-by-term evaluation of Eq. 9
         double base = 0.0;
-        for (int u = 2; u <= p.t_est; ++u) base += (double)hs[u - 1] - (double)hs[u - 2];
+        for (int u = 2; u <= p.t_est; ++u) base += HS(u) - HS(u - 1);
         base /= (double)(p.t_est - 1);
         const double threshold = p.alpha * base;
         for (int u = p.t_est + 1; u <= t && !found; ++u) {
-            const double gu = (double)hs[u - 1] - (double)hs[u - 2];
-            const double gprev = (double)hs[u - 2] - (double)hs[u - 3];
+            const double gu = HS(u) - HS(u - 1);
+            const double gprev = HS(u - 1) - HS(u - 2);
             if ((gu + gprev) / 2.0 <= threshold) found = u;   // Eq. 10
         }
     }
@@ -181,15 +185,15 @@ static void schedule_one(const nova_sched_params& p, int t, int j, int n_tokens,
         if (p.force_keep_ratio >= 0.0) {
             rs = rl = 1.0 - p.force_keep_ratio;
         } else {
-            if (t >= 2) growth_now = (double)hs[t - 1] - (double)hs[t - 2];
+            if (t >= 2) growth_now = HS(t) - HS(t - 1);
             const double arg = ((double)t - (double)act) / p.tau;
             rs = 1.0 / (1.0 + exp(-arg)) - p.lambda * tanh(growth_now);   // Eq. 11
             rl = rs;
             if (j >= 2) {                                                // Eq. 12-13
                 double mu = 0.0;
-                for (int k = 1; k < j; ++k) mu += (double)hl[k - 1];
+                for (int k = 1; k < j; ++k) mu += HL(k);
                 mu /= (double)(j - 1);
-                const double delta = (mu != 0.0) ? ((double)hl[j - 1] - mu) / mu : 0.0;
+                const double delta = (mu != 0.0) ? (HL(j) - mu) / mu : 0.0;
                 rl = rs - delta * rs;
             }
         }
@@ -202,6 +206,24 @@ static void schedule_one(const nova_sched_params& p, int t, int j, int n_tokens,
     if (kept < p.k_min) kept = p.k_min;
     if (kept > n_tokens) kept = n_tokens;
     *keep = (int32_t)kept;
+#undef HS
+#undef HL
+}
+
+// One thread per image; the histories are device arrays [t, B] and [j, B].
+__global__ void keep_ratios_kernel(const nova_sched_params p, int B, int t, int j, int n_tokens,
+                                   const float* __restrict__ hs, const float* __restrict__ hl,
+                                   int32_t* __restrict__ t_star, int32_t* __restrict__ act_scale,
+                                   int32_t* __restrict__ keep)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int32_t ts, as, kp;
+    double rs, rl;
+    schedule_one(p, t, j, n_tokens, hs + b, B, hl ? hl + b : nullptr, B, &ts, &as, &rs, &rl, &kp);
+    if (t_star) t_star[b] = ts;
+    if (act_scale) act_scale[b] = as;
+    keep[b] = kp;
 }
 
 nova_status nova_keep_ratios(const nova_sched_params* p, int B, int t, int j, int N_t,
@@ -214,9 +236,30 @@ nova_status nova_keep_ratios(const nova_sched_params* p, int B, int t, int j, in
     if (!hbar_scale || !t_star || !act_scale || !ratio_scale || !ratio_layer || !keep) return NOVA_ERR_INVALID_ARG;
     if (j >= 2 && !hbar_layer && p->force_keep_ratio < 0.0) return NOVA_ERR_INVALID_ARG;
     for (int b = 0; b < B; ++b)
-        schedule_one(*p, t, j, N_t, hbar_scale + (size_t)b * t,
-                     hbar_layer ? hbar_layer + (size_t)b * j : nullptr,
+        schedule_one(*p, t, j, N_t, hbar_scale + (size_t)b * t, 1,
+                     hbar_layer ? hbar_layer + (size_t)b * j : nullptr, 1,
                      t_star + b, act_scale + b, ratio_scale + b, ratio_layer + b, keep + b);
+    return NOVA_OK;
+}
+
+nova_status nova_keep_ratios_device(nova_ctx* ctx, const nova_sched_params* p, int B, int t, int j, int N_t,
+                                    const float* hbar_scale, const float* hbar_layer,
+                                    int32_t* t_star, int32_t* act_scale, int32_t* keep, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if (!p || B < 0 || t < 1 || j < 1 || N_t < 1 || p->t_est < 2 || !(p->tau > 0.0))
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_keep_ratios_device: bad argument");
+    if (B == 0) return NOVA_OK;
+    if (!hbar_scale || !keep) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_keep_ratios_device: null pointer");
+    if (j >= 2 && !hbar_layer && p->force_keep_ratio < 0.0)
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_keep_ratios_device: layer history missing");
+    cudaStream_t st = (cudaStream_t)stream;
+    {
+        nova_launch_scope scope(ctx, NOVA_K_KEEP_RATIOS, st);
+        keep_ratios_kernel<<<(B + 127) / 128, 128, 0, st>>>(*p, B, t, j, N_t, hbar_scale, hbar_layer, t_star,
+                                                           act_scale, keep);
+    }
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }
 

@@ -45,10 +45,12 @@ __device__ __forceinline__ float warp_sum(float v)
 template <int VEC, bool MAPS>
 __global__ void __launch_bounds__(kLnWarps * 32)
 layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
-               float eps, int M, int vec_per_row, uint4* __restrict__ out, const RowMapArgs maps)
+               float eps, int M, const int32_t* __restrict__ m_dev, int vec_per_row, uint4* __restrict__ out,
+               const RowMapArgs maps)
 {
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
+    if (m_dev) M = min(M, *m_dev);      // the host knows only an upper bound
     if (r >= M) return;
     long src = r;
     if (MAPS) {
@@ -170,8 +172,8 @@ bool shape_ok(const nova_block_shape* s)
 }  // namespace
 
 static nova_status launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const RowMapArgs* maps,
-                             const __nv_bfloat16* g, const __nv_bfloat16* b, float eps, int M, int C,
-                             __nv_bfloat16* out, cudaStream_t st)
+                             const __nv_bfloat16* g, const __nv_bfloat16* b, float eps, int M, const int32_t* m_dev,
+                             int C, __nv_bfloat16* out, cudaStream_t st)
 {
     if (M <= 0) return NOVA_OK;
     const int vec = C / 8;
@@ -182,8 +184,8 @@ static nova_status launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const RowMap
     nova_launch_scope scope(ctx, NOVA_K_LAYERNORM, st);
 #define NOVA_LN_CASE(V)                                                                                          \
     do {                                                                                                         \
-        if (maps) layernorm_rows<V, true><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, vec, (uint4*)out, *maps); \
-        else layernorm_rows<V, false><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, vec, (uint4*)out, none);      \
+        if (maps) layernorm_rows<V, true><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, *maps); \
+        else layernorm_rows<V, false><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, none);      \
     } while (0)
     if (per_lane <= 2) NOVA_LN_CASE(2);
     else if (per_lane <= 4) NOVA_LN_CASE(4);
@@ -202,11 +204,13 @@ extern "C" size_t nova_block_workspace_bytes(const nova_block_shape* s)
     return carve(nullptr, s->M, s->C, s->F).bytes;
 }
 
-extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block_weights* w,
-                                                 const nova_block_shape* s, const void* x_in,
-                                                 const int32_t* keep_idx, const int32_t* cu_keep,
-                                                 void* k_cache, void* v_cache, int32_t* kv_len,
-                                                 int append_kv, void* y_kept, void* stream)
+// m_on_device: s->M is only an upper bound of the kept rows (it sizes grids, tensor maps and the
+// workspace); every kernel takes the true count from cu_keep[B] on the device.
+static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w,
+                                 const nova_block_shape* s, const void* x_in,
+                                 const int32_t* keep_idx, const int32_t* cu_keep,
+                                 void* k_cache, void* v_cache, int32_t* kv_len,
+                                 int append_kv, void* y_kept, void* stream, bool m_on_device)
 {
     if (!ctx) return NOVA_ERR_INVALID_ARG;
     if (!w || !s) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward: null weights or shape");
@@ -231,17 +235,18 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     typedef const __nv_bfloat16* cbf;
     typedef __nv_bfloat16* bf;
 
+    const int32_t* m_dev = m_on_device ? cu_keep + s->B : nullptr;
     nova_status rc;
     // h = LN1(gathered rows); the same kernel writes the row maps the GEMM epilogues use
     RowMapArgs maps;
     maps.keep_idx = keep_idx; maps.cu_keep = cu_keep; maps.kv_len = kv_len; maps.B = s->B; maps.N = s->N;
     maps.Lmax = s->Lmax; maps.src_row = ws.src_row; maps.kv_row = ws.kv_row; maps.status = ctx->dev_status;
-    rc = launch_ln(ctx, (cbf)x_in, &maps, (cbf)w->ln1_g, (cbf)w->ln1_b, w->eps, M, C, ws.h, st);
+    rc = launch_ln(ctx, (cbf)x_in, &maps, (cbf)w->ln1_g, (cbf)w->ln1_b, w->eps, M, m_dev, C, ws.h, st);
     if (rc) return rc;
     // [q | k | v] = h W_qkv^T + b; k, v go straight to their cache rows
     nova_gemm_args g;
     memset(&g, 0, sizeof(g));
-    g.A = ws.h; g.W = (cbf)w->w_qkv; g.bias = (cbf)w->b_qkv; g.M = M; g.N = 3 * C; g.K = C;
+    g.A = ws.h; g.W = (cbf)w->w_qkv; g.bias = (cbf)w->b_qkv; g.M = M; g.m_dev = m_dev; g.N = 3 * C; g.K = C;
     g.epilogue = NOVA_EPI_QKV; g.cat = NOVA_K_GEMM_QKV; g.out = ws.q; g.C = C; g.k_cache = (bf)k_cache; g.v_cache = (bf)v_cache; g.kv_row = ws.kv_row;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
@@ -255,22 +260,22 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     if (rc) return rc;
     // x1 = Xc + o W_o^T + b_o
     memset(&g, 0, sizeof(g));
-    g.A = ws.o; g.W = (cbf)w->w_o; g.bias = (cbf)w->b_o; g.M = M; g.N = C; g.K = C;
+    g.A = ws.o; g.W = (cbf)w->w_o; g.bias = (cbf)w->b_o; g.M = M; g.m_dev = m_dev; g.N = C; g.K = C;
     g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_PROJ; g.out = ws.x1; g.res = (cbf)x_in; g.res_row = ws.src_row;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     // h = LN2(x1)
-    rc = launch_ln(ctx, ws.x1, nullptr, (cbf)w->ln2_g, (cbf)w->ln2_b, w->eps, M, C, ws.h, st);
+    rc = launch_ln(ctx, ws.x1, nullptr, (cbf)w->ln2_g, (cbf)w->ln2_b, w->eps, M, m_dev, C, ws.h, st);
     if (rc) return rc;
     // f = GELU(h W_fc1^T + b_fc1)
     memset(&g, 0, sizeof(g));
-    g.A = ws.h; g.W = (cbf)w->w_fc1; g.bias = (cbf)w->b_fc1; g.M = M; g.N = F; g.K = C;
+    g.A = ws.h; g.W = (cbf)w->w_fc1; g.bias = (cbf)w->b_fc1; g.M = M; g.m_dev = m_dev; g.N = F; g.K = C;
     g.epilogue = NOVA_EPI_BIAS_GELU; g.cat = NOVA_K_GEMM_FC1; g.out = ws.f;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     // y = x1 + f W_fc2^T + b_fc2
     memset(&g, 0, sizeof(g));
-    g.A = ws.f; g.W = (cbf)w->w_fc2; g.bias = (cbf)w->b_fc2; g.M = M; g.N = C; g.K = F;
+    g.A = ws.f; g.W = (cbf)w->w_fc2; g.bias = (cbf)w->b_fc2; g.M = M; g.m_dev = m_dev; g.N = C; g.K = F;
     g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_FC2; g.out = (bf)y_kept; g.res = ws.x1; g.res_row = nullptr;
     if (append_kv) {
         // the last kernel of the block also advances kv_len: every reader of the old lengths (row
@@ -280,6 +285,24 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     return NOVA_OK;
+}
+
+extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block_weights* w,
+                                                 const nova_block_shape* s, const void* x_in,
+                                                 const int32_t* keep_idx, const int32_t* cu_keep,
+                                                 void* k_cache, void* v_cache, int32_t* kv_len,
+                                                 int append_kv, void* y_kept, void* stream)
+{
+    return block_forward(ctx, w, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream, false);
+}
+
+extern "C" nova_status nova_pruned_block_forward_device(nova_ctx* ctx, const nova_block_weights* w,
+                                                        const nova_block_shape* s, const void* x_in,
+                                                        const int32_t* keep_idx, const int32_t* cu_keep,
+                                                        void* k_cache, void* v_cache, int32_t* kv_len,
+                                                        int append_kv, void* y_kept, void* stream)
+{
+    return block_forward(ctx, w, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream, true);
 }
 
 // ---- block forward for callers that cannot allocate device memory --------------------------

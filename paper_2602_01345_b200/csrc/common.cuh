@@ -30,7 +30,7 @@
 enum nova_kernel_cat {
     NOVA_K_ENTROPY = 0, NOVA_K_ENTROPY_MEAN, NOVA_K_SELECT, NOVA_K_LAYERNORM,
     NOVA_K_GEMM_QKV, NOVA_K_ATTENTION, NOVA_K_GEMM_PROJ, NOVA_K_GEMM_FC1, NOVA_K_GEMM_FC2,
-    NOVA_K_RESTORE, NOVA_K_COUNT
+    NOVA_K_RESTORE, NOVA_K_KEEP_RATIOS, NOVA_K_COUNT
 };
 
 struct nova_prof_rec {
@@ -121,6 +121,7 @@ struct nova_gemm_args {
     const __nv_bfloat16* W;     // [N, K] row-major
     const __nv_bfloat16* bias;  // [N]
     int M, N, K;
+    const int32_t* m_dev;       // NULL, or device: the true row count (<= M, which then sizes the grid and maps)
     int epilogue;
     int cat;                    // nova_kernel_cat of this launch
     __nv_bfloat16* out;         // [M, N] (QKV: q buffer [M, C])

@@ -62,7 +62,14 @@ struct GemmParams {
     int32_t* adv_kv_len;
     int adv_B, adv_Lmax;
     float* ent;
+    const int32_t* m_dev;
 };
+
+// Rows of this launch: p.M, or the device-side count when the host only knows an upper bound.
+__device__ __forceinline__ int true_rows(const GemmParams& p)
+{
+    return p.m_dev ? min(max(*p.m_dev, 0), p.M) : p.M;
+}
 
 // Advance of the K/V cache lengths, done by one warp-sized loop of the launch's first CTA.
 __device__ __forceinline__ void advance_kv_len(const GemmParams& p)
@@ -144,7 +151,9 @@ gemm_bf16_tn(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int num_kb = p.K / BK;
+    const int M = true_rows(p);
     if (blockIdx.x == 0 && blockIdx.y == 0) advance_kv_len(p);
+    if (m0 >= M) return;            // whole tile past the device-side row count (nothing allocated yet)
 
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
@@ -209,7 +218,7 @@ gemm_bf16_tn(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
         const int row = m0 + q * 32 + lane;
         if (mbar_wait_warp(acc_bar, 0, abort_flag, p.status)) {
             tc_fence_after();
-            const bool row_ok = row < p.M;
+            const bool row_ok = row < M;
             long res_base = 0;
             long kv_base = -1;
             if (row_ok) {
@@ -242,7 +251,7 @@ GemmParams make_params(nova_ctx* ctx, const nova_gemm_args& a)
     p.res = a.res; p.res_row = a.res_row; p.C = a.C; p.k_cache = a.k_cache; p.v_cache = a.v_cache;
     p.kv_row = a.kv_row; p.status = ctx->dev_status;
     p.adv_cu_keep = a.adv_cu_keep; p.adv_kv_len = a.adv_kv_len; p.adv_B = a.adv_B; p.adv_Lmax = a.adv_Lmax;
-    p.ent = a.ent;
+    p.ent = a.ent; p.m_dev = a.m_dev;
     return p;
 }
 
@@ -418,8 +427,8 @@ struct EntropyState {
 template <int BN, int STAGES>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-                  const __grid_constant__ CUtensorMap tmap_w_half, const GemmParams p, const int span,
-                  const int tiles_full, const int num_tiles, const int group)
+                  const __grid_constant__ CUtensorMap tmap_w_half, const GemmParams p, const int span_host,
+                  const int tiles_full_host, const int num_tiles_host, const int group)
 {
     using L = PairSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
@@ -437,6 +446,18 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     if (blockIdx.x == 0) advance_kv_len(p);
     const int num_kb = p.K / BK;
+    // The work list is the host's, or, when only the device knows the row count, the same plan
+    // rebuilt here from that count (every thread computes the same values).
+    int M = p.M, span = span_host, tiles_full = tiles_full_host, num_tiles = num_tiles_host;
+    if (p.m_dev) {
+        M = true_rows(p);
+        const int tiles_m = (M + kPairBM - 1) / kPairBM, tiles_n = (p.N + BN - 1) / BN;
+        const int tiles = tiles_m * tiles_n;
+        const int rem = tiles % num_pairs;
+        tiles_full = (group == 0 && rem > 0 && 2 * rem <= num_pairs) ? tiles - rem : tiles;
+        num_tiles = tiles_full + 2 * (tiles - tiles_full);
+        span = (group != 0 || M >= p.N) ? -tiles_n : tiles_m;
+    }
     constexpr uint32_t kTmemCols = 2 * BN;       // two accumulator buffers
 
     if (threadIdx.x == 0) {
@@ -561,7 +582,7 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             ok = mbar_wait_warp(&acc_full[a], (uint32_t)(local >> 1) & 1, abort_flag, p.status);
             if (!ok) break;
             tc_fence_after();
-            const bool row_ok = row < p.M;
+            const bool row_ok = row < M;
             long res_base = 0;
             long kv_base = -1;
             if (row_ok) {

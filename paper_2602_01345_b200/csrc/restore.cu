@@ -38,9 +38,10 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 restore_kernel(const uint4* __restrict__ x_in, const uint4* __restrict__ y_kept,
                const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ prune_idx,
                const int32_t* __restrict__ cu_keep, const uint4* __restrict__ cache_prev,
-               int hp, int wp, int h, int w, int vec_per_row, int B, int M,
+               int hp, int wp, int h, int w, int vec_per_row, int B, int M, bool m_on_device,
                uint4* __restrict__ x_out, uint4* __restrict__ cache_out)
 {
+    if (m_on_device) M = cu_keep[B];    // the kept count lives on the device
     const int lane = threadIdx.x & 31;
     const long r = (long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const int N = h * w;
@@ -127,11 +128,11 @@ restore_kernel(const uint4* __restrict__ x_in, const uint4* __restrict__ y_kept,
 
 }  // namespace
 
-extern "C" nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, const void* y_kept,
-                                               const int32_t* keep_idx, const int32_t* prune_idx,
-                                               const int32_t* cu_keep, const void* cache_prev,
-                                               int hp, int wp, int h, int w, int C, int B, int M,
-                                               void* x_out, void* cache_out, void* stream)
+static nova_status restore(nova_ctx* ctx, const void* x_in, const void* y_kept,
+                           const int32_t* keep_idx, const int32_t* prune_idx,
+                           const int32_t* cu_keep, const void* cache_prev,
+                           int hp, int wp, int h, int w, int C, int B, int M, bool m_on_device,
+                           void* x_out, void* cache_out, void* stream)
 {
     if (!ctx) return NOVA_ERR_INVALID_ARG;
     if (B < 0 || h < 0 || w < 0 || C < 1 || M < 0 || (long)M > (long)B * h * w)
@@ -141,7 +142,7 @@ extern "C" nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, 
     if (C % 8) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_restore_from_cache: C must be a multiple of 8");
     if (!x_in || !x_out || !cu_keep || (M > 0 && (!y_kept || !keep_idx)))
         return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_restore_from_cache: null pointer");
-    if (M < total && (!prune_idx || !cache_prev || hp < 1 || wp < 1))
+    if ((M < total || m_on_device) && (!prune_idx || !cache_prev || hp < 1 || wp < 1))
         return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_restore_from_cache: pruned rows need prune_idx and cache_prev");
     if (x_out == x_in) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_restore_from_cache: x_out aliases x_in");
     if (!nova_aligned16(x_in) || !nova_aligned16(x_out) || !nova_aligned16(y_kept) ||
@@ -151,7 +152,29 @@ extern "C" nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, 
     nova_launch_scope scope(ctx, NOVA_K_RESTORE, (cudaStream_t)stream);
     restore_kernel<<<blocks, kWarpsPerBlock * 32, 0, (cudaStream_t)stream>>>(
         (const uint4*)x_in, (const uint4*)y_kept, keep_idx, prune_idx, cu_keep, (const uint4*)cache_prev,
-        hp, wp, h, w, C / 8, B, M, (uint4*)x_out, (uint4*)cache_out);
+        hp, wp, h, w, C / 8, B, M, m_on_device, (uint4*)x_out, (uint4*)cache_out);
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
+}
+
+extern "C" nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, const void* y_kept,
+                                               const int32_t* keep_idx, const int32_t* prune_idx,
+                                               const int32_t* cu_keep, const void* cache_prev,
+                                               int hp, int wp, int h, int w, int C, int B, int M,
+                                               void* x_out, void* cache_out, void* stream)
+{
+    return restore(ctx, x_in, y_kept, keep_idx, prune_idx, cu_keep, cache_prev, hp, wp, h, w, C, B, M, false,
+                   x_out, cache_out, stream);
+}
+
+extern "C" nova_status nova_restore_from_cache_device(nova_ctx* ctx, const void* x_in, const void* y_kept,
+                                                      const int32_t* keep_idx, const int32_t* prune_idx,
+                                                      const int32_t* cu_keep, const void* cache_prev,
+                                                      int hp, int wp, int h, int w, int C, int B,
+                                                      void* x_out, void* cache_out, void* stream)
+{
+    const long total = (long)B * h * w;
+    if (total > 0x7fffffffL) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_restore_from_cache_device: too many rows");
+    return restore(ctx, x_in, y_kept, keep_idx, prune_idx, cu_keep, cache_prev, hp, wp, h, w, C, B, (int)total, true,
+                   x_out, cache_out, stream);
 }

@@ -27,7 +27,7 @@ __device__ __forceinline__ uint32_t order_key(float f)
 
 __global__ void __launch_bounds__(kThreads)
 select_topk_kernel(const float* __restrict__ ent, int N, int seg0, int cu0, SegParams sp,
-                   int32_t* __restrict__ keep_idx, int32_t* __restrict__ prune_idx,
+                   const int32_t* __restrict__ k_dev, int32_t* __restrict__ keep_idx, int32_t* __restrict__ prune_idx,
                    int32_t* __restrict__ cu_keep, int32_t* __restrict__ pos)
 {
     extern __shared__ uint32_t keys[];          // N keys
@@ -38,9 +38,25 @@ select_topk_kernel(const float* __restrict__ ent, int N, int seg0, int cu0, SegP
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int seg_local = blockIdx.x;
     const int seg = seg0 + seg_local;
-    const int k = sp.k[seg_local];
-    int cu = cu0;
-    for (int s = 0; s < seg_local; ++s) cu += sp.k[s];
+    __shared__ int sh_cu;
+    int k, cu;
+    if (k_dev) {
+        // keep counts written by an earlier kernel: clamp to [0, N]; cu = sum over the segments before
+        if (tid == 0) sh_cu = 0;
+        __syncthreads();
+        int part = 0;
+        for (int s = tid; s < seg; s += kThreads) part += min(max(k_dev[s], 0), N);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+        if (lane == 0 && part) atomicAdd(&sh_cu, part);
+        __syncthreads();
+        cu = sh_cu;
+        k = min(max(k_dev[seg], 0), N);
+    } else {
+        k = sp.k[seg_local];
+        cu = cu0;
+        for (int s = 0; s < seg_local; ++s) cu += sp.k[s];
+    }
     if (tid == 0) {
         cu_keep[seg] = cu;
         if (seg_local == (int)gridDim.x - 1) cu_keep[seg + 1] = cu + k;   // next launch overwrites with the same value
@@ -181,9 +197,41 @@ extern "C" nova_status nova_select_topk(nova_ctx* ctx, const float* ent, int S, 
         for (int s = 0; s < n; ++s) sp.k[s] = k[s0 + s];
         {
             nova_launch_scope scope(ctx, NOVA_K_SELECT, st);
-            select_topk_kernel<<<n, kThreads, (size_t)N * 4, st>>>(ent, N, s0, cu, sp, keep_idx, prune_idx, cu_keep, pos);
+            select_topk_kernel<<<n, kThreads, (size_t)N * 4, st>>>(ent, N, s0, cu, sp, nullptr, keep_idx, prune_idx, cu_keep, pos);
         }
         for (int s = 0; s < n; ++s) cu += k[s0 + s];
+    }
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    return NOVA_OK;
+}
+
+// The same selection with the keep counts in device memory (written by nova_keep_ratios_device):
+// no host value depends on them, so the call needs no synchronisation and can be captured.
+extern "C" nova_status nova_select_topk_device(nova_ctx* ctx, const float* ent, int S, int N,
+                                               const int32_t* k_dev, int32_t* keep_idx, int32_t* prune_idx,
+                                               int32_t* cu_keep, int32_t* pos, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if (S < 0 || N < 0) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_select_topk_device: negative size");
+    if (N > 16384) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_select_topk_device: N > 16384");
+    if (S > 65535) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_select_topk_device: S > 65535");
+    if (!cu_keep) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_select_topk_device: null cu_keep");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (S == 0 || N == 0) {
+        NOVA_CUDA_CHECK(ctx, cudaMemsetAsync(cu_keep, 0, sizeof(int32_t) * (size_t)(S + 1), st));
+        return NOVA_OK;
+    }
+    if (!ent || !k_dev || !keep_idx || !prune_idx)
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_select_topk_device: null pointer");
+    if (!ctx->attr_select) {
+        NOVA_CUDA_CHECK(ctx, cudaFuncSetAttribute(select_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * 4));
+        ctx->attr_select = true;
+    }
+    SegParams sp;
+    memset(&sp, 0, sizeof(sp));
+    {
+        nova_launch_scope scope(ctx, NOVA_K_SELECT, st);
+        select_topk_kernel<<<S, kThreads, (size_t)N * 4, st>>>(ent, N, 0, 0, sp, k_dev, keep_idx, prune_idx, cu_keep, pos);
     }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;

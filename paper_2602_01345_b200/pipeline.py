@@ -107,8 +107,12 @@ class MultiScaleRunner:
     caller supplies each scale's layer input and logits.
     """
 
-    def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, scales, eps: float = 1e-6):
+    def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, scales, eps: float = 1e-6,
+                 on_device: bool = False):
+        """on_device: keep the entropy history and every keep count in device memory and run each
+        scale through DeviceScaleRunner (no host synchronisation inside a scale)."""
         self.ctx, self.weights, self.n_heads, self.B, self.eps = ctx, weights, n_heads, B, eps
+        self.on_device = on_device
         self.scales = tuple(scales)
         self.L = len(weights)
         self.C = weights[0]["w_o"].shape[0]
@@ -119,16 +123,30 @@ class MultiScaleRunner:
         self.kv_len = torch.zeros((self.L, B), dtype=torch.int32, device=dev)
         self.res_cache = [None] * self.L          # previous scale's residual cache per layer, [B, h, w, C]
         self.hbar_scale = torch.zeros((B, 0), dtype=torch.float32)
-        self._ent = None
+        self.hist_dev = torch.zeros((len(self.scales), B), dtype=torch.float32, device=dev) if on_device else None
+        self.t_done = 0
 
     def run_scale(self, t: int, x_in, scale_logits, layer_logits, sched: nv.SchedParams, stream=None):
         """Scale t (1-based, in order). scale_logits [B, N_t, V] give the scale's mean entropy
         (Eq. 7) that extends the history; layer_logits: L tensors [B, N_t, V]. Returns
         (x_out, keeps, runner) where runner is the PrunedScaleRunner that ran the layers."""
-        assert t == self.hbar_scale.shape[1] + 1, "scales must be run in order"
+        assert t == self.t_done + 1, "scales must be run in order"
+        self.t_done = t
         side = self.scales[t - 1]
         B, N = self.B, side * side
         st = stream if stream is not None else torch.cuda.current_stream()
+        if self.on_device:
+            runner = DeviceScaleRunner(self.ctx, self.weights, self.n_heads, B, side, side, self.Lmax, self.k_caches,
+                                       self.v_caches, self.kv_len, self.res_cache, sched, t, self.hist_dev,
+                                       scale_logits.shape[-1], eps=self.eps, logits_dtype=scale_logits.dtype)
+            with torch.cuda.stream(st):
+                runner.x_in.copy_(x_in)
+                runner.scale_logits.copy_(scale_logits)
+                for dst, src in zip(runner.layer_logits, layer_logits):
+                    dst.copy_(src)
+            x_out = runner.enqueue(stream=st)
+            self.res_cache = [c.view(B, side, side, self.C) for c in runner.cache_out]
+            return x_out, runner.keep, runner
         ent = torch.empty((B, N), dtype=torch.float32, device=x_in.device)
         mean = torch.empty((B,), dtype=torch.float32, device=x_in.device)
         nv.nova_scale_entropy(self.ctx, scale_logits, ent, mean, stream=st)
@@ -138,6 +156,99 @@ class MultiScaleRunner:
         x_out, keeps = runner.run_scale(x_in, layer_logits, sched, t, self.hbar_scale.contiguous(), stream=st)
         self.res_cache = [c.view(B, side, side, self.C) for c in runner.cache_out]
         return x_out, keeps, runner
+
+
+class DeviceScaleRunner:
+    """One scale through all layers with every decision left on the device.
+
+    Per layer: entropy map and mean -> Eq. 8-13 in a one-thread-per-image kernel -> selection with
+    the keep counts read from device memory -> the block and the restore sized by an upper bound
+    (all B*N rows), the kept count read from cu_keep[B]. Nothing crosses to the host, so the whole
+    scale is one uninterrupted run of launches that can be recorded in a CUDA graph once and
+    replayed for every new batch of the same shape. Inputs live in fixed buffers:
+      x_in [B, N, C], scale_logits [B, N, V], layer_logits[j] [B, N, V]   (copy new data in)
+      hist [T, B] f32: rows 0..t-2 hold the earlier scales' means; row t-1 is written here.
+    Outputs: x_out (property), keep [L, B] int32, cache_out[j] [B, N, C], ent [L, B, N].
+    """
+
+    def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, h: int, w: int, Lmax: int,
+                 k_caches, v_caches, kv_len, cache_prev, sched: nv.SchedParams, t: int, hist, V: int,
+                 eps: float = 1e-6, logits_dtype=torch.bfloat16):
+        self.ctx, self.sched, self.t = ctx, sched, t
+        self.L = len(weights)
+        self.B, self.h, self.w, self.N = B, h, w, h * w
+        self.C = weights[0]["w_o"].shape[0]
+        self.F = weights[0]["w_fc1"].shape[0]
+        self.n_heads, self.Lmax = n_heads, Lmax
+        self.weights = [nv.BlockWeights(wt, eps) for wt in weights]
+        self.k_caches, self.v_caches, self.kv_len = k_caches, v_caches, kv_len
+        dev = weights[0]["w_o"].device
+        N, Cc, L = self.N, self.C, self.L
+        zero_cache = torch.zeros((B, 1, 1, Cc), dtype=torch.bfloat16, device=dev)
+        self.cache_prev = [c if c is not None else zero_cache for c in cache_prev]
+        self.hist = hist
+        assert hist.dtype == torch.float32 and hist.shape[1] == B and hist.shape[0] >= t and hist.is_contiguous()
+        self.x_in = torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev)
+        self.scale_logits = torch.empty((B, N, V), dtype=logits_dtype, device=dev)
+        self.layer_logits = [torch.empty((B, N, V), dtype=logits_dtype, device=dev) for _ in range(L)]
+        self.ent_scale = torch.empty((B, N), dtype=torch.float32, device=dev)
+        self.ent = torch.empty((L, B, N), dtype=torch.float32, device=dev)
+        self.mean = torch.empty((L, B), dtype=torch.float32, device=dev)
+        self.keep = torch.zeros((L, B), dtype=torch.int32, device=dev)
+        self.t_star = torch.zeros((B,), dtype=torch.int32, device=dev)
+        self.act_scale = torch.zeros((B,), dtype=torch.int32, device=dev)
+        self.keep_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
+        self.prune_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
+        self.cu_keep = torch.zeros((B + 1,), dtype=torch.int32, device=dev)
+        self.y_kept = torch.empty((B * N, Cc), dtype=torch.bfloat16, device=dev)
+        self.x_buf = [torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        self.cache_out = [torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+        self.shape = nv.BlockShape(B, N, Cc, n_heads, self.F, Lmax, B * N)
+        ctx.ensure_workspace(self.shape)
+        self.x_out = self.x_buf[(L - 1) & 1]
+        self.graph = None
+
+    def enqueue(self, append_kv: bool = True, stream=None):
+        """Issues the scale's launches on `stream` (default: the current stream); returns x_out."""
+        ctx, B, N, t = self.ctx, self.B, self.N, self.t
+        st = stream if stream is not None else torch.cuda.current_stream()
+        hist_t = self.hist[:t]
+        nv.nova_scale_entropy(ctx, self.scale_logits, self.ent_scale, hist_t[t - 1], stream=st)
+        x = self.x_in
+        for j in range(self.L):
+            nv.nova_scale_entropy(ctx, self.layer_logits[j], self.ent[j], self.mean[j], stream=st)
+            nv.nova_keep_ratios_device(ctx, self.sched, t, j + 1, N, hist_t, self.mean[: j + 1], self.keep[j],
+                                       self.t_star, self.act_scale, stream=st)
+            nv.nova_select_topk_device(ctx, self.ent[j], self.keep[j], self.keep_idx, self.prune_idx, self.cu_keep,
+                                       None, stream=st)
+            nv.nova_pruned_block_forward_device(ctx, self.weights[j], self.shape, x, self.keep_idx, self.cu_keep,
+                                                self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
+                                                self.y_kept, stream=st)
+            x_out = self.x_buf[j & 1]
+            nv.nova_restore_from_cache_device(ctx, x, self.y_kept, self.keep_idx, self.prune_idx, self.cu_keep,
+                                              self.cache_prev[j], self.h, self.w, x_out, self.cache_out[j], stream=st)
+            x = x_out
+        return x
+
+    def capture(self):
+        """Records the scale in a CUDA graph. One eager pass without the K/V append comes first (it
+        performs the kernels' one-time attribute set-up and leaves kv_len as it was); the recorded
+        pass appends."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.enqueue(append_kv=False, stream=side)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.enqueue(append_kv=True)
+        self.graph = g
+        return g
+
+    def replay(self):
+        self.graph.replay()
+        return self.x_out
 
 
 def launch_count(ctx: nv.Context) -> int:

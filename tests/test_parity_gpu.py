@@ -705,3 +705,134 @@ def test_multi_scale_generation_256_shape(ctx):
     for j in range(L):
         assert _rel_err(f32(gen.k_caches[j]), ok_cache[j]) <= BLOCK_TOL
         assert _rel_err(f32(gen.res_cache[j]), o_res[j]) <= BLOCK_TOL
+
+
+def test_keep_ratios_device_against_oracle(ctx):
+    """Eq. 8-13 evaluated by one device thread per image: inflection scale, activation scale and keep
+    counts equal the oracle's on seeded sigmoid-shaped entropy histories, at every scale and for
+    several layers (layer linkage on random layer means)."""
+    B, T, L, N = 64, 10, 6, 4096
+    _, hbar = synth.scale_envelope_temperatures(B, T, seed=11)
+    hist = hbar.t().contiguous().to(DEV)                      # [T, B]
+    rng = np.random.default_rng(5)
+    layer = torch.from_numpy((hbar[:, -1:].numpy() * (1 + 0.2 * rng.standard_normal((B, L)))).astype(np.float32))
+    layer_dev = layer.t().contiguous().to(DEV)                # [L, B]
+    sched, osched = nova.SchedParams(), oracle.SchedParams()
+    keep = torch.zeros(B, dtype=torch.int32, device=DEV)
+    ts = torch.zeros(B, dtype=torch.int32, device=DEV)
+    act = torch.zeros(B, dtype=torch.int32, device=DEV)
+    fired = 0
+    for t in range(1, T + 1):
+        for j in (1, 2, L):
+            nova.nova_keep_ratios_device(ctx, sched, t, j, N, hist[:t], layer_dev[:j], keep, ts, act)
+            want = oracle.keep_ratios(osched, t, j, N, hbar[:, :t].numpy().copy(), layer[:, :j].numpy().copy())
+            assert np.array_equal(ts.cpu().numpy(), want["t_star"]), (t, j)
+            assert np.array_equal(act.cpu().numpy(), want["act_scale"]), (t, j)
+            assert np.array_equal(keep.cpu().numpy(), want["keep"]), (t, j)
+            fired += int((want["keep"] < N).sum())
+    assert fired > 0
+    assert ctx.device_status() == 0
+
+
+def test_select_topk_device_counts(ctx):
+    """Selection with the keep counts in device memory: same lists as the host-count call,
+    including counts outside [0, N] (clamped) and the 0 and N corners."""
+    S, N = 7, 1000
+    ent = torch.from_numpy(np.random.default_rng(2).random((S, N), dtype=np.float32)).to(DEV)
+    k = torch.tensor([0, N, 1, 999, 500, -3, N + 5], dtype=torch.int32)
+    kc = k.clamp(0, N)
+    M = int(kc.sum())
+    a_keep = torch.full((S * N,), -7, dtype=torch.int32, device=DEV)
+    a_prune = torch.full((S * N,), -7, dtype=torch.int32, device=DEV)
+    a_cu = torch.zeros(S + 1, dtype=torch.int32, device=DEV)
+    a_pos = torch.zeros((S, N), dtype=torch.int32, device=DEV)
+    nova.nova_select_topk_device(ctx, ent, k.to(DEV), a_keep, a_prune, a_cu, a_pos)
+    w_keep, w_prune, w_cu, w_pos = oracle.select_topk(ent.cpu().numpy(), kc.numpy())
+    assert np.array_equal(a_cu.cpu().numpy(), w_cu)
+    assert np.array_equal(a_keep[:M].cpu().numpy(), w_keep)
+    assert np.array_equal(a_prune[: S * N - M].cpu().numpy(), w_prune)
+    assert np.array_equal(a_pos.cpu().numpy(), w_pos)
+    assert (a_keep[M:] == -7).all() and (a_prune[S * N - M:] == -7).all()      # nothing written past the lists
+
+
+def test_device_driven_generation_equals_host_driven(ctx):
+    """The ten-scale generation of the 256x256 schedule with every keep count left on the device
+    (no host synchronisation inside a scale, launches sized by the upper bound B*N) gives bit for bit
+    what the host-driven call sequence gives: outputs, keep counts, K/V caches, residual caches."""
+    from paper_2602_01345_b200 import pipeline
+    ms = synth.CONFIGS["c2_var_d16_256"]
+    B, L, T = 2, 2, len(ms.scales)
+    weights = [synth.block_weights(ms.C, ms.F, 100 + j, DEV) for j in range(L)]
+    a_env, _ = synth.scale_envelope_temperatures(B, T, seed=3)
+    beta = synth.layer_inverse_temperatures(L, 3)
+    host = pipeline.MultiScaleRunner(ctx, weights, ms.heads, B, ms.scales)
+    devr = pipeline.MultiScaleRunner(ctx, weights, ms.heads, B, ms.scales, on_device=True)
+    sched = nova.SchedParams()
+    pruned = 0
+    for t in range(1, T + 1):
+        N = ms.scales[t - 1] ** 2
+        x_in = synth.activations(B, N, ms.C, 200 + t, DEV)
+        a = a_env[:, t - 1].view(B, 1).expand(B, N).contiguous().to(DEV)
+        scale_logits = synth.logits_from_temperature(a, synth.V_CODEBOOK, 300 + t)
+        layer_logits = [synth.logits_from_temperature(a * float(beta[j]), synth.V_CODEBOOK, 400 + 10 * t + j)
+                        for j in range(L)]
+        xh, keeps_h, _ = host.run_scale(t, x_in, scale_logits, layer_logits, sched)
+        xh = xh.clone()
+        xd, keeps_d, _ = devr.run_scale(t, x_in, scale_logits, layer_logits, sched)
+        assert ctx.device_status() == 0
+        assert torch.equal(torch.stack(keeps_h), keeps_d.cpu()), t
+        assert torch.equal(xh, xd), t
+        pruned += int((torch.stack(keeps_h) < N).sum())
+    assert pruned > 0
+    assert torch.equal(host.kv_len, devr.kv_len)
+    assert torch.equal(host.hbar_scale.t().contiguous(), devr.hist_dev.cpu())
+    for j in range(L):
+        assert torch.equal(host.k_caches[j], devr.k_caches[j]) and torch.equal(host.v_caches[j], devr.v_caches[j])
+        assert torch.equal(host.res_cache[j], devr.res_cache[j])
+
+
+def test_scale_graph_replay(ctx):
+    """A pruned scale recorded once in a CUDA graph and replayed: each replay on fresh inputs gives
+    what the eager device-driven launches give, and the keep counts follow the inputs (a different
+    entropy history changes them without re-recording)."""
+    from paper_2602_01345_b200 import pipeline
+    ms = synth.CONFIGS["c2_var_d16_256"]
+    B, L, T = 2, 3, len(ms.scales)
+    side = ms.scales[-1]
+    N, V = side * side, synth.V_CODEBOOK
+    weights = [synth.block_weights(ms.C, ms.F, 100 + j, DEV) for j in range(L)]
+    Lmax = ms.total_tokens
+    prior = Lmax - N
+    k_caches = [synth.activations(B, Lmax, ms.C, 50 + j, DEV) for j in range(L)]
+    v_caches = [synth.activations(B, Lmax, ms.C, 60 + j, DEV) for j in range(L)]
+    cache_prev = [synth.activations(B, ms.scales[-2] ** 2, ms.C, 70 + j, DEV).view(B, ms.scales[-2], ms.scales[-2], ms.C)
+                  for j in range(L)]
+    kv_len = torch.full((L, B), prior, dtype=torch.int32, device=DEV)
+    _, hbar = synth.scale_envelope_temperatures(B, T, seed=3)
+    hist = hbar.t().contiguous().to(DEV)
+    sched = nova.SchedParams()
+    r = pipeline.DeviceScaleRunner(ctx, weights, ms.heads, B, side, side, Lmax, k_caches, v_caches, kv_len,
+                                   cache_prev, sched, T, hist, V)
+
+    def load(seed, temp):
+        r.x_in.copy_(synth.activations(B, N, ms.C, seed, DEV))
+        a = torch.full((B, N), temp, device=DEV)
+        r.scale_logits.copy_(synth.logits_from_temperature(a, V, seed + 1))
+        for j in range(L):
+            r.layer_logits[j].copy_(synth.logits_from_temperature(a * (1 + 0.1 * j), V, seed + 2 + j))
+
+    load(500, 1.0)
+    r.capture()
+    outs = []
+    for seed, temp in ((500, 1.0), (600, 3.0)):
+        load(seed, temp)
+        kv_len.fill_(prior)
+        x_eager = r.enqueue(append_kv=False).clone()
+        keep_eager = r.keep.clone()
+        x_graph = r.replay().clone()
+        assert ctx.device_status() == 0
+        assert torch.equal(x_graph, x_eager) and torch.equal(r.keep, keep_eager)
+        assert torch.equal(kv_len.cpu(), (prior + r.keep.cpu()).to(torch.int32))        # the recorded pass appends
+        outs.append(r.keep.cpu().clone())
+    assert (outs[0] < N).any()
+    assert not torch.equal(outs[0], outs[1])
