@@ -313,6 +313,36 @@ def run_ours(args):
                     "frac_of_tensor_peak": round(head_tf / pk["tensor"], 4),
                     "logits_bytes_not_written_or_read": int(2 * rows * synth.V_CODEBOOK * 2)}
     assert ctx.device_status() == 0, "device status after the head-entropy timing"
+    # The same step with every decision left on the device (Eq. 8-13 in a kernel, kept counts read
+    # from device memory, launches sized by the upper bound B*N): issued eagerly, and recorded once
+    # in a CUDA graph and replayed. Same inputs and buffers as the timed region above.
+    hist_dev = hbar_scale.t().contiguous().to(dev)
+    drun = pipeline.DeviceScaleRunner(ctx, st["weights"], ms.heads, B, wd["h"], wd["w"], wd["Lmax"], st["k_caches"],
+                                      st["v_caches"], st["kv_len"], st["cache_prev"], sched, wd["t"], hist_dev,
+                                      synth.V_CODEBOOK, x_in=st["x_in"], layer_logits=st["logits"], scale_entropy=False)
+    st["kv_len"].copy_(st["kv_len0"])
+    l0 = pipeline.launch_count(ctx)
+    drun.capture()
+    dev_launches = (pipeline.launch_count(ctx) - l0) // 2          # one eager pass + one recorded pass
+    dev_ms = {}
+    for mode in ("eager", "graph"):
+        for it in range(args.warmup + args.steps):
+            if it == args.warmup:
+                torch.cuda.synchronize()
+                b0.record(stream)
+            st["kv_len"].copy_(st["kv_len0"])
+            if mode == "eager":
+                drun.enqueue(stream=stream)
+            else:
+                drun.replay()
+        b1.record(stream)
+        torch.cuda.synchronize()
+        dev_ms[mode] = b0.elapsed_time(b1) / args.steps
+    assert ctx.device_status() == 0, "device status after the device-driven timing"
+    same = bool(torch.equal(drun.x_out, x_out)) and bool(torch.equal(drun.keep.cpu(), torch.stack(keeps)))
+    device_schedule = {"ms_per_step_eager": round(dev_ms["eager"], 4), "ms_per_step_graph": round(dev_ms["graph"], 4),
+                       "ms_per_step_host_driven": round(ms_per_step, 4), "launches_per_step": int(dev_launches),
+                       "host_syncs_per_step": 0, "equals_host_driven_result": same}
     for k in ("entropy_rows", "restore"):
         if "gbs" in kernels.get(k, {}):
             kernels[k]["frac_of_hbm_peak"] = round(kernels[k]["gbs"] / pk["hbm"], 4)
@@ -325,7 +355,7 @@ def run_ours(args):
         "config": config_json(wd, world), "clocks": clk, "gpu_launches": int(launches),
         "tokens_per_s": round(world * B * N / (ms_per_step / 1e3), 1),
         "roofline": roofline, "roofline_second": other_roofline, "kernels": kernels,
-        "next_head_entropy": head_entropy,
+        "next_head_entropy": head_entropy, "next_device_schedule": device_schedule,
     }
 
     # ---- end to end: inputs start in pinned host memory, result read back every step

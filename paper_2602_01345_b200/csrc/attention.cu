@@ -549,11 +549,24 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 asm volatile("bar.sync 1, %0;" ::"r"(n_soft) : "memory");
                 if (ok && ticket_s == 1) {
                     // the other CTA fenced its partial result before it drew ticket 0
+                    // The merge is written in terms of (half 0, half 1), not (mine, other), with every
+                    // rounding spelled out: either CTA may be the one that merges, and the output must
+                    // not depend on which.
                     const float m_o = __ldcg(other + DH), l_o = __ldcg(other + DH + 1);
                     const float m_new = fmaxf(m_ref, m_o);
                     const float a_me = ex2((m_ref - m_new) * c), a_o = ex2((m_o - m_new) * c);
-                    const float inv = 1.f / (l_run * a_me + l_o * a_o);
-                    const float w_me = a_me * inv, w_o = a_o * inv;
+                    const bool first = (khalf == 0);
+                    const float a0 = first ? a_me : a_o, a1 = first ? a_o : a_me;
+                    const float l0 = first ? l_run : l_o, l1 = first ? l_o : l_run;
+                    const float inv = 1.f / __fmaf_rn(l0, a0, __fmul_rn(l1, a1));
+                    const float w0 = a0 * inv, w1 = a1 * inv;
+                    const float w_me = first ? w0 : w1, w_o = first ? w1 : w0;
+                    auto mix = [&](uint32_t mine_bits, float theirs) {
+                        const float me = __uint_as_float(mine_bits);
+                        // half 0's term is the multiply-add operand, half 1's the rounded product
+                        return first ? __fmaf_rn(me, w_me, __fmul_rn(theirs, w_o))
+                                     : __fmaf_rn(theirs, w_o, __fmul_rn(me, w_me));
+                    };
 #pragma unroll
                     for (int cch = 0; cch < DH / 32; ++cch) {
                         uint32_t ov[32];
@@ -566,10 +579,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                                 const float4 o0 = __ldcg((const float4*)(other + cch * 32 + g * 8));
                                 const float4 o1 = __ldcg((const float4*)(other + cch * 32 + g * 8 + 4));
                                 dst[g] = make_uint4(
-                                    pack_bf16(__uint_as_float(ov[g * 8]) * w_me + o0.x * w_o, __uint_as_float(ov[g * 8 + 1]) * w_me + o0.y * w_o),
-                                    pack_bf16(__uint_as_float(ov[g * 8 + 2]) * w_me + o0.z * w_o, __uint_as_float(ov[g * 8 + 3]) * w_me + o0.w * w_o),
-                                    pack_bf16(__uint_as_float(ov[g * 8 + 4]) * w_me + o1.x * w_o, __uint_as_float(ov[g * 8 + 5]) * w_me + o1.y * w_o),
-                                    pack_bf16(__uint_as_float(ov[g * 8 + 6]) * w_me + o1.z * w_o, __uint_as_float(ov[g * 8 + 7]) * w_me + o1.w * w_o));
+                                    pack_bf16(mix(ov[g * 8], o0.x), mix(ov[g * 8 + 1], o0.y)),
+                                    pack_bf16(mix(ov[g * 8 + 2], o0.z), mix(ov[g * 8 + 3], o0.w)),
+                                    pack_bf16(mix(ov[g * 8 + 4], o1.x), mix(ov[g * 8 + 5], o1.y)),
+                                    pack_bf16(mix(ov[g * 8 + 6], o1.z), mix(ov[g * 8 + 7], o1.w)));
                             }
                         }
                     }

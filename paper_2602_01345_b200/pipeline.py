@@ -173,7 +173,10 @@ class DeviceScaleRunner:
 
     def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, h: int, w: int, Lmax: int,
                  k_caches, v_caches, kv_len, cache_prev, sched: nv.SchedParams, t: int, hist, V: int,
-                 eps: float = 1e-6, logits_dtype=torch.bfloat16):
+                 eps: float = 1e-6, logits_dtype=torch.bfloat16, x_in=None, layer_logits=None,
+                 scale_entropy: bool = True):
+        """x_in / layer_logits: existing tensors to use as the fixed input buffers instead of new
+        ones. scale_entropy=False: hist row t-1 is already filled by the caller (no scale_logits)."""
         self.ctx, self.sched, self.t = ctx, sched, t
         self.L = len(weights)
         self.B, self.h, self.w, self.N = B, h, w, h * w
@@ -188,9 +191,10 @@ class DeviceScaleRunner:
         self.cache_prev = [c if c is not None else zero_cache for c in cache_prev]
         self.hist = hist
         assert hist.dtype == torch.float32 and hist.shape[1] == B and hist.shape[0] >= t and hist.is_contiguous()
-        self.x_in = torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev)
-        self.scale_logits = torch.empty((B, N, V), dtype=logits_dtype, device=dev)
-        self.layer_logits = [torch.empty((B, N, V), dtype=logits_dtype, device=dev) for _ in range(L)]
+        self.x_in = x_in if x_in is not None else torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev)
+        self.scale_logits = torch.empty((B, N, V), dtype=logits_dtype, device=dev) if scale_entropy else None
+        self.layer_logits = (list(layer_logits) if layer_logits is not None else
+                             [torch.empty((B, N, V), dtype=logits_dtype, device=dev) for _ in range(L)])
         self.ent_scale = torch.empty((B, N), dtype=torch.float32, device=dev)
         self.ent = torch.empty((L, B, N), dtype=torch.float32, device=dev)
         self.mean = torch.empty((L, B), dtype=torch.float32, device=dev)
@@ -213,7 +217,8 @@ class DeviceScaleRunner:
         ctx, B, N, t = self.ctx, self.B, self.N, self.t
         st = stream if stream is not None else torch.cuda.current_stream()
         hist_t = self.hist[:t]
-        nv.nova_scale_entropy(ctx, self.scale_logits, self.ent_scale, hist_t[t - 1], stream=st)
+        if self.scale_logits is not None:
+            nv.nova_scale_entropy(ctx, self.scale_logits, self.ent_scale, hist_t[t - 1], stream=st)
         x = self.x_in
         for j in range(self.L):
             nv.nova_scale_entropy(ctx, self.layer_logits[j], self.ent[j], self.mean[j], stream=st)

@@ -462,6 +462,27 @@ def test_block_1024_shape_batch1_keep025_sampled_rows(ctx):
                 rows=np.array(rows, np.int32))
 
 
+def test_block_output_does_not_depend_on_merge_order(ctx):
+    """With every attention work item shared by two CTAs, either CTA of a pair may finish second and
+    merge; the block output must be the same bits whichever does. Eight runs of the batch-1,
+    keep-0.25 shape (64 items, all shared) give identical outputs."""
+    B, N, C, heads, F, Lmax, k, prior = 1, 4096, 2048, 16, 8192, 10521, 1024, 6425
+    wt = nova.BlockWeights(synth.block_weights(C, F, 47, DEV), 1e-6)
+    x = synth.activations(B, N, C, 48, DEV)
+    k_cache, v_cache, _ = synth.kv_cache(B, Lmax, prior, C, 49, DEV)
+    ent = torch.rand((B, N), generator=torch.Generator(device="cpu").manual_seed(47))
+    keep_idx, _, cu, _ = gpu_select(ctx, ent.to(DEV), [k])
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, k)
+    first = None
+    for _ in range(8):
+        kv_len = torch.tensor([prior], dtype=torch.int32, device=DEV)
+        y = _run_block(ctx, shape, wt, x, keep_idx, cu, k_cache, v_cache, kv_len)
+        if first is None:
+            first = y.clone()
+        assert torch.equal(y, first)
+    assert ctx.device_status() == 0
+
+
 @pytest.mark.parametrize("kv_len", [517, 5])
 def test_block_key_split_small_cases(ctx, kv_len):
     """Four attention work items on 148 SMs, so each is shared by two CTAs, one per half of the keys.
