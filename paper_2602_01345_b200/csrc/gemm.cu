@@ -10,7 +10,9 @@
 // (clusters of two, tcgen05 cta_group::2), each pair computing 256 x BN tiles. Per tensor-core
 // instruction each CTA supplies only its 128 rows of A and BN/2 rows of W, which halves the
 // shared-memory and L2 traffic per flop of the single-CTA tile; the fp32 accumulator is double
-// buffered in tensor memory so that the epilogue of tile i overlaps the main loop of tile i+1.
+// buffered in tensor memory so that the epilogue of tile i overlaps the main loop of tile i+1, and
+// eight epilogue warps (two per tensor-memory lane quarter, alternate column chunks) keep the
+// epilogue shorter than the main loop even with GELU.
 // Every mbarrier wait is bounded; on expiry the CTA records a timeout and tears down.
 #include "tc_common.cuh"
 
@@ -32,12 +34,15 @@ struct GemmSmem {
 
 __device__ __forceinline__ float gelu_tanh(float x)
 {
+    // 0.5 x (1 + tanh(c (x + 0.044715 x^3))) with the hardware tanh (relative error 2^-11, an order
+    // of magnitude below the bf16 rounding of the result): six instructions per element. The FC1
+    // epilogue is bound by its instruction count, not by memory.
     const float c = 0.7978845608028654f;
-    const float inner = c * (x + 0.044715f * x * x * x);
-    // tanh(y) = 1 - 2 / (exp(2y) + 1); exp through ex2 keeps the error near 1e-6 relative
-    const float e = __expf(2.f * inner);
-    const float t = 1.f - __fdividef(2.f, e + 1.f);
-    return 0.5f * x * (1.f + t);
+    const float inner = x * fmaf(x * x, 0.044715f * c, c);
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(inner));
+    const float hx = 0.5f * x;
+    return fmaf(hx, t, hx);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
@@ -257,6 +262,7 @@ GemmParams make_params(nova_ctx* ctx, const nova_gemm_args& a)
 
 // ---- CTA-pair kernel ------------------------------------------------------------------------
 constexpr int kPairBM = 256;           // rows of one pair tile (128 per CTA)
+constexpr int kPairThreads = 320;      // producer warp, MMA warp, eight epilogue warps
 
 template <int BN, int STAGES>
 struct PairSmem {
@@ -423,9 +429,9 @@ struct EntropyState {
 //   full[s]       leader's copy is used: one arrival (its own expect_tx) + the bytes of both CTAs
 //   empty[s]      each CTA's copy, signalled in both CTAs by the leader's tcgen05.commit
 //   acc_full[a]   each CTA's copy, same; a = accumulator buffer of tile parity
-//   acc_empty[a]  leader's copy: one arrival per epilogue warp of both CTAs (8)
+//   acc_empty[a]  leader's copy: one arrival per epilogue warp of both CTAs (16)
 template <int BN, int STAGES>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                   const __grid_constant__ CUtensorMap tmap_w_half, const GemmParams p, const int span_host,
                   const int tiles_full_host, const int num_tiles_host, const int group)
@@ -468,7 +474,7 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&acc_full[a], 1);
-            mbar_init(&acc_empty[a], 8);
+            mbar_init(&acc_empty[a], 16);
         }
         fence_barrier_init();
         prefetch_tmap(&tmap_a);
@@ -565,8 +571,16 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
         }
     } else {
-        // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31 of this CTA's half of the tile
+        // epilogue: warp w may touch TMEM lanes 32*(w%4) .. +31 of this CTA's half of the tile. Two
+        // warps share each lane quarter and take alternate 32-column chunks: the epilogue of a tile
+        // is a long chain of dependent instructions per thread, and with one warp per quarter the
+        // GELU epilogue took longer than the tile's main loop. (The entropy epilogue carries a row's
+        // state from chunk to chunk in one thread, so there the second warp of a quarter only
+        // signals.)
         const int q = warp & 3;
+        const bool entropy_epi = (p.epilogue == NOVA_EPI_ENTROPY);
+        const int c_first = entropy_epi ? 0 : ((warp - 2) >> 2), c_step = entropy_epi ? 1 : 2;
+        const bool idle_warp = entropy_epi && warp >= 6;
         const uint32_t acc_empty_leader = map_to_cta(smem_u32(&acc_empty[0]), 0);
         int local = 0;
         bool ok = true;
@@ -591,7 +605,7 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * BN);
 #pragma unroll 1
-            for (int c = 0; c < n_chunks; ++c) {
+            for (int c = c_first; c < n_chunks && !idle_warp; c += c_step) {
                 const int col0 = n0 + c * 32;
                 uint32_t acc[32];
                 tmem_ld32(t_addr + (uint32_t)(c * 32), acc);
@@ -600,7 +614,7 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (p.epilogue == NOVA_EPI_ENTROPY) est.add_chunk(acc, p.bias ? p.bias + col0 : nullptr);
                 else epilogue_chunk(p, row, col0, acc, res_base, kv_base);
             }
-            if (p.epilogue == NOVA_EPI_ENTROPY && t.n0 + BN >= p.N) {
+            if (p.epilogue == NOVA_EPI_ENTROPY && !idle_warp && t.n0 + BN >= p.N) {
                 // last column tile of this row block: the row's entropy is complete
                 if (row_ok) p.ent[row] = est.finish(p.status);
                 est.reset();
@@ -651,7 +665,7 @@ nova_status launch_pair(nova_ctx* ctx, const nova_gemm_args& a, cudaStream_t st)
         nova_launch_scope scope(ctx, a.cat, st);
         // sweep the smaller operand; the entropy epilogue needs the N-fastest order
         const int span = (entropy || (long)a.M >= (long)a.N) ? -tiles_n : tiles_m;
-        kern<<<dim3(2 * pairs), kThreads, L::kTotal, st>>>(ta, tw, tw_half, p, span, tiles_full, entries,
+        kern<<<dim3(2 * pairs), kPairThreads, L::kTotal, st>>>(ta, tw, tw_half, p, span, tiles_full, entries,
                                                            entropy ? tiles_n : 0);
     }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
