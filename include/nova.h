@@ -58,9 +58,9 @@ typedef enum nova_dtype { NOVA_BF16 = 0, NOVA_F32 = 1 } nova_dtype;
 
 /* ---- context ------------------------------------------------------------------ */
 
-/* Creates a context bound to CUDA device `device`. Allocates about 200 KB of device memory for
- * the status word and the partial sums of the entropy means (the only allocation the library
- * ever makes). */
+/* Creates a context bound to CUDA device `device`. Allocates about 3 KB of device memory for
+ * the status word, tickets and the accumulators of the entropy means (the only allocation the
+ * library ever makes). */
 nova_status nova_create(nova_ctx** out, int device);
 void        nova_destroy(nova_ctx* ctx);
 const char* nova_last_error(const nova_ctx* ctx);

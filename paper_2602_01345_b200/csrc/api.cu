@@ -117,8 +117,8 @@ nova_status nova_device_status(nova_ctx* ctx, void* stream)
     unsigned int word = 0;
     NOVA_CUDA_CHECK(ctx, cudaMemcpyAsync(&word, ctx->dev_status, sizeof(word), cudaMemcpyDeviceToHost, st));
     NOVA_CUDA_CHECK(ctx, cudaStreamSynchronize(st));
-    // an aborted kernel may leave the entropy counter or attention tickets half way: clear all words
-    if (word) NOVA_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->dev_status, 0, NOVA_STATUS_WORDS * sizeof(word), st));
+    // an aborted kernel may leave the entropy accumulators or attention tickets half way: clear everything
+    if (word) NOVA_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->dev_status, 0, NOVA_STATUS_BYTES, st));
     if (word & NOVA_DEV_TIMEOUT) return nova_fail(ctx, NOVA_ERR_TIMEOUT, "a device-side wait expired");
     if (word & NOVA_DEV_SHAPE) return nova_fail(ctx, NOVA_ERR_SHAPE, "K/V cache overflow on the device");
     if (word & NOVA_DEV_NONFINITE) return nova_fail(ctx, NOVA_ERR_NONFINITE, "non-finite logit");

@@ -17,14 +17,14 @@
 #define NOVA_DEV_SHAPE     4u
 
 // Layout of the context's one device allocation: NOVA_STATUS_WORDS 32-bit words (word 0 = status
-// bits, word 1 = completion counter of the entropy kernel, words 16.. = attention tickets), then the per-CTA partial sums of the
-// entropy means, float[NOVA_MEAN_MAX_CTAS][NOVA_MEAN_MAX_SEGMENTS].
+// flags, a block of tickets for key-split attention items), then one 64-bit accumulator per segment
+// for the entropy means (NOVA_MEAN_MAX_SEGMENTS of them). All of it is zero between launches.
 #define NOVA_STATUS_WORDS 128
 #define NOVA_ATTN_TICKET_WORD0 16     // words 16 .. 16 + NOVA_ATTN_TICKETS - 1: tickets of key-split attention items
 #define NOVA_ATTN_TICKETS 96
-#define NOVA_MEAN_MAX_CTAS 192
+#define NOVA_MEAN_MAX_CTAS 192        // the accumulator's arrival count has 8 bits
 #define NOVA_MEAN_MAX_SEGMENTS 256
-#define NOVA_STATUS_BYTES (NOVA_STATUS_WORDS * 4 + NOVA_MEAN_MAX_CTAS * NOVA_MEAN_MAX_SEGMENTS * 4)
+#define NOVA_STATUS_BYTES (NOVA_STATUS_WORDS * 4 + NOVA_MEAN_MAX_SEGMENTS * 8)
 
 // Kernel categories for the launch counter and the optional per-kernel event timing.
 enum nova_kernel_cat {

@@ -238,8 +238,8 @@ entropy_rows_reg(const void* __restrict__ logits, long rows, int V, long row_str
 // cp.async.bulk, one copy per row, completion counted on an mbarrier; sixteen consumer warps take
 // rows from the ring in turn, move the row into registers, hand the slot back at once and then do
 // the arithmetic. HBM sees one deep, steady stream per SM instead of waves of CTAs that load, then
-// compute. The per-segment means are taken by whichever CTA finishes last (a counter in global
-// memory), always with the same summation tree, so the result does not depend on which CTA it is.
+// compute. The per-segment means are completed by whichever CTA arrives last at a fixed-point
+// accumulator in global memory; integer addition commutes, so the result does not depend on the order.
 // Row i of a CTA goes to slot i % kSlots and to consumer warp i % 16; kSlots is a multiple of 16, so
 // every use of a slot is consumed by the same warp, in order. That matters: a parity wait for use
 // n of a slot succeeds at once while use n-1 has not completed yet, and bulk copies may land out of
@@ -261,7 +261,7 @@ template <int VEC, bool BF16>
 __global__ void __launch_bounds__(kRingThreads, 1)
 entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_stride_bytes,
                   float* __restrict__ ent, float* __restrict__ mean, int seg_rows, int n_seg,
-                  unsigned int* status, unsigned int* done_counter, float* __restrict__ cta_part)
+                  unsigned int* status, unsigned long long* __restrict__ accum, int fix_shift)
 {
     using namespace tc;
     constexpr int kRowBytes = VEC * 512;
@@ -273,7 +273,6 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
     uint64_t* empty_bar = full_bar + kSlots;
     float* warp_part = (float*)(empty_bar + kSlots);       // [kRingConsumers][n_seg] partial sums per warp
     __shared__ int abort_flag_s;
-    __shared__ int is_last_s;
     volatile int* abort_flag = &abort_flag_s;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -326,7 +325,7 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
             if (lane == 0) {
                 const float h = finish_row(m, s_sum, u, ent, row, status);
                 if (mean) {
-                    const int seg = (int)(row / seg_rows);
+                    const int seg = (int)((unsigned int)row / (unsigned int)seg_rows);   // rows < 2^31 (checked by the launcher)
                     if (seg != cur_seg) {
                         if (cur_seg >= 0) warp_part[warp * n_seg + cur_seg] = seg_acc;
                         cur_seg = seg;
@@ -340,30 +339,29 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
     }
     if (!mean) return;
 
-    // ---- means: per-CTA partial sums, combined by the last CTA to finish ------------------------
-    // Every level adds in a fixed order (a warp's rows in row order, the 16 warps in warp order,
-    // the CTAs in CTA order with a fixed tree), so the means do not depend on which CTA is last.
+    // ---- means ---------------------------------------------------------------------------------
+    // A CTA's partial sum of a segment is added in a fixed order (a warp's rows in row order, the 16
+    // warps in warp order) and then joins the other CTAs' in ONE 64-bit atomic add per segment:
+    //   bits 63..56  CTAs that have arrived      bits 55..46  how many of them had a non-finite sum
+    //   bits 45..0   sum of the partial sums in fixed point (2^-fix_shift units)
+    // Integer addition commutes, so the total does not depend on the order of arrival, and the add
+    // that completes the count returns everything needed: that thread writes the mean and clears
+    // the accumulator for the next launch. No fence, no second pass over partial results.
     __syncthreads();
     for (int sg = threadIdx.x; sg < n_seg; sg += kRingThreads) {
         float acc = 0.f;
         for (int w = 0; w < kRingConsumers; ++w) acc += warp_part[w * n_seg + sg];
-        cta_part[(long)blockIdx.x * n_seg + sg] = acc;
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int ticket = atomicAdd(done_counter, 1u);
-        is_last_s = (ticket == gridDim.x - 1);
-        if (is_last_s) *done_counter = 0;      // ready for the next launch
-    }
-    __syncthreads();
-    if (!is_last_s) return;
-    // one warp per segment: lane l adds CTAs l, l + 32, ... in order, then the shuffle tree
-    for (int sg = warp; sg < n_seg; sg += kRingThreads / 32) {
-        float acc = 0.f;
-        for (int c = lane; c < (int)gridDim.x; c += 32) acc += __ldcg(cta_part + (long)c * n_seg + sg);
-        acc = warp_sum(acc);
-        if (lane == 0) mean[sg] = acc / (float)seg_rows;
+        const bool finite = (acc >= 0.f) && (acc < INFINITY);
+        unsigned long long add = 1ull << 56;
+        if (finite) add += (unsigned long long)__float2ll_rn(ldexpf(acc, fix_shift));
+        else add += 1ull << 46;
+        const unsigned long long old = atomicAdd(&accum[sg], add);
+        if ((old >> 56) == gridDim.x - 1) {
+            const unsigned long long tot = old + add;
+            const double sum = (double)(tot & ((1ull << 46) - 1)) * exp2(-(double)fix_shift);
+            mean[sg] = ((tot >> 46) & 0x3ffull) ? __int_as_float(0x7fc00000) : (float)(sum / (double)seg_rows);
+            accum[sg] = 0ull;
+        }
     }
 }
 
@@ -434,9 +432,13 @@ nova_status launch_ring(nova_ctx* ctx, const void* logits, long rows, int V, lon
         attr_done[ctx->device] = true;
     }
     const int grid = (int)(rows < ctx->num_sms ? rows : ctx->num_sms);
+    // fixed-point scale of the mean accumulators: a segment's sum is below N * ln(V) <= 24 N, and
+    // has to stay below 2^46
+    int fix_shift = 30;
+    while (fix_shift > 0 && 24.0 * (double)N * exp2((double)fix_shift) >= 70368744177664.0 /* 2^46 */) --fix_shift;
     entropy_rows_ring<VEC, BF16><<<grid, kRingThreads, smem, st>>>(
-        (const char*)logits, rows, V, stride_bytes, ent, mean, N, S, ctx->dev_status, ctx->dev_status + 1,
-        (float*)(ctx->dev_status + NOVA_STATUS_WORDS));
+        (const char*)logits, rows, V, stride_bytes, ent, mean, N, S, ctx->dev_status,
+        (unsigned long long*)(ctx->dev_status + NOVA_STATUS_WORDS), fix_shift);
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }
@@ -459,7 +461,7 @@ extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nov
     cudaStream_t st = (cudaStream_t)stream;
     const int elt = (dt == NOVA_BF16) ? 2 : 4;
     const long row_bytes = (long)V * elt;
-    if ((row_bytes == 2048 || row_bytes == 4096 || row_bytes == 8192) && rows >= 64 &&
+    if ((row_bytes == 2048 || row_bytes == 4096 || row_bytes == 8192) && rows >= 64 && rows <= 0x7fffffffL &&
         (!mean || (S <= NOVA_MEAN_MAX_SEGMENTS && ctx->num_sms <= NOVA_MEAN_MAX_CTAS))) {
         // persistent ring kernel; the second word of the status allocation is its completion counter
         const long stride_bytes = (long)row_stride * elt;
