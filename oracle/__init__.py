@@ -53,6 +53,13 @@ class _BlockWeights(ctypes.Structure):
         "ln2_g", "ln2_b", "w_fc1", "b_fc1", "w_fc2", "b_fc2")] + [("eps", ctypes.c_float)]
 
 
+MODULATION_NAMES = ("shift1", "scale1", "gate1", "shift2", "scale2", "gate2")
+
+
+class _BlockModulation(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in MODULATION_NAMES]
+
+
 def _load():
     global _lib
     if _lib is None:
@@ -162,11 +169,13 @@ WEIGHT_NAMES = ("ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_o", "b_o",
 
 
 def pruned_block_forward(weights: dict, eps: float, n_heads: int, x_in, keep_idx, cu_keep,
-                         k_cache, v_cache, kv_len, rows=None):
+                         k_cache, v_cache, kv_len, rows=None, modulation=None):
     """Eq. 14 on the kept tokens (pre-LN block; keys = cache ++ kept tokens' own k/v).
 
     x_in [B, N, C]; k_cache/v_cache [B, Lmax, C]; kv_len [B]; rows: optional compacted
-    row numbers to evaluate. Returns (y [R, C], k_new [M, C], v_new [M, C]).
+    row numbers to evaluate. modulation: optional dict of per-image [B, C] arrays named in
+    MODULATION_NAMES (adaptive LayerNorm: LN output * (1 + scale) + shift, branch * gate); a
+    missing name means no such term. Returns (y [R, C], k_new [M, C], v_new [M, C]).
     """
     x = _f32(x_in)
     B, N, C = x.shape
@@ -185,8 +194,17 @@ def pruned_block_forward(weights: dict, eps: float, n_heads: int, x_in, keep_idx
     k_new = np.empty((M, C), np.float32)
     v_new = np.empty((M, C), np.float32)
     cw = _BlockWeights(*[_p(w[n]) for n in WEIGHT_NAMES], eps)
-    _load().oracle_pruned_block_forward(
-        ctypes.byref(cw), B, N, C, n_heads, F, Lmax, _p(x), _p(ki), _p(cu),
+    if modulation is None:
+        _load().oracle_pruned_block_forward(
+            ctypes.byref(cw), B, N, C, n_heads, F, Lmax, _p(x), _p(ki), _p(cu),
+            _p(kc), _p(vc), _p(kl), _p(rr), R, _p(y), _p(k_new), _p(v_new))
+        return y, k_new, v_new
+    md = {n: _f32(modulation[n]) for n in MODULATION_NAMES if modulation.get(n) is not None}
+    for a in md.values():
+        assert a.shape == (B, C)
+    cm = _BlockModulation(*[_p(md[n]) if n in md else None for n in MODULATION_NAMES])
+    _load().oracle_pruned_block_forward_mod(
+        ctypes.byref(cw), ctypes.byref(cm), B, N, C, n_heads, F, Lmax, _p(x), _p(ki), _p(cu),
         _p(kc), _p(vc), _p(kl), _p(rr), R, _p(y), _p(k_new), _p(v_new))
     return y, k_new, v_new
 

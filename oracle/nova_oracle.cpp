@@ -289,7 +289,48 @@ static inline double gelu_tanh(double x)
     return 0.5 * x * (1.0 + std::tanh(c * (x + 0.044715 * x * x * x)));
 }
 
+// Per-image modulation of the block (adaptive LayerNorm as in the class-conditional VAR
+// backbones; the NOVA paper names the layer's two parts but gives no block equations, so this
+// is the backbone's published form): every array is [B, C], any of the six may be NULL.
+//   h1 = LN1(x) * (1 + scale1[b]) + shift1[b]        x1 = x  + gate1[b] * (attention branch)
+//   h2 = LN2(x1) * (1 + scale2[b]) + shift2[b]       y  = x1 + gate2[b] * (MLP branch)
+struct oracle_block_modulation {
+    const float *shift1, *scale1, *gate1, *shift2, *scale2, *gate2;
+};
+
+static void modulate_row(float* h, const float* scale, const float* shift, int b, int C)
+{
+    for (int c = 0; c < C; ++c) {
+        double v = (double)h[c];
+        if (scale) v *= 1.0 + (double)scale[(long)b * C + c];
+        if (shift) v += (double)shift[(long)b * C + c];
+        h[c] = (float)v;
+    }
+}
+
+void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle_block_modulation* mod,
+                                     int B, int N, int C, int n_heads, int F, int Lmax,
+                                     const float* x_in, const int32_t* keep_idx,
+                                     const int32_t* cu_keep,
+                                     const float* k_cache, const float* v_cache,
+                                     const int32_t* kv_len,
+                                     const int32_t* rows, int n_rows,
+                                     float* y, float* k_new, float* v_new);
+
 void oracle_pruned_block_forward(const oracle_block_weights* w,
+                                 int B, int N, int C, int n_heads, int F, int Lmax,
+                                 const float* x_in, const int32_t* keep_idx,
+                                 const int32_t* cu_keep,
+                                 const float* k_cache, const float* v_cache,
+                                 const int32_t* kv_len,
+                                 const int32_t* rows, int n_rows,
+                                 float* y, float* k_new, float* v_new)
+{
+    oracle_pruned_block_forward_mod(w, nullptr, B, N, C, n_heads, F, Lmax, x_in, keep_idx, cu_keep, k_cache,
+                                    v_cache, kv_len, rows, n_rows, y, k_new, v_new);
+}
+
+void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle_block_modulation* mod,
                                  int B, int N, int C, int n_heads, int F, int Lmax,
                                  const float* x_in, const int32_t* keep_idx,
                                  const int32_t* cu_keep,
@@ -311,6 +352,7 @@ void oracle_pruned_block_forward(const oracle_block_weights* w,
         const int b = seg_of[m];
         const float* x = x_in + ((long)b * N + keep_idx[m]) * C;
         layer_norm_row(x, w->ln1_g, w->ln1_b, w->eps, C, &h1[(size_t)m * C]);
+        if (mod) modulate_row(&h1[(size_t)m * C], mod->scale1, mod->shift1, b, C);
         linear_row(&h1[(size_t)m * C], w->w_qkv + (long)C * C, w->b_qkv + C, C, C,
                    k_new + (long)m * C);
         linear_row(&h1[(size_t)m * C], w->w_qkv + 2L * C * C, w->b_qkv + 2 * C, C, C,
@@ -358,13 +400,20 @@ void oracle_pruned_block_forward(const oracle_block_weights* w,
             }
         }
         linear_row(o.data(), w->w_o, w->b_o, C, C, x1.data());
-        for (int c = 0; c < C; ++c) x1[c] = (float)((double)x[c] + (double)x1[c]);
+        for (int c = 0; c < C; ++c) {
+            const double g1 = (mod && mod->gate1) ? (double)mod->gate1[(long)b * C + c] : 1.0;
+            x1[c] = (float)((double)x[c] + g1 * (double)x1[c]);
+        }
 
         layer_norm_row(x1.data(), w->ln2_g, w->ln2_b, w->eps, C, h2.data());
+        if (mod) modulate_row(h2.data(), mod->scale2, mod->shift2, b, C);
         linear_row(h2.data(), w->w_fc1, w->b_fc1, C, F, f1.data());
         for (int i = 0; i < F; ++i) f1[i] = (float)gelu_tanh((double)f1[i]);
         linear_row(f1.data(), w->w_fc2, w->b_fc2, F, C, f2.data());
-        for (int c = 0; c < C; ++c) y[(long)ri * C + c] = (float)((double)x1[c] + (double)f2[c]);
+        for (int c = 0; c < C; ++c) {
+            const double g2 = (mod && mod->gate2) ? (double)mod->gate2[(long)b * C + c] : 1.0;
+            y[(long)ri * C + c] = (float)((double)x1[c] + g2 * (double)f2[c]);
+        }
     }
 }
 

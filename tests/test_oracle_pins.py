@@ -357,6 +357,76 @@ def test_block_matches_library_composition_ragged():
         assert np.allclose(v_new[cu[b]:cu[b + 1]], wv, atol=1e-5)
 
 
+def _torch_block_modulated(w, eps, heads, x_kept, k_old, v_old, md):
+    """The adaptive-LayerNorm block of one image from library ops (torch fp64): md holds the
+    image's six [C] vectors."""
+    t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    x = t(x_kept)
+    C = x.shape[1]
+    dh = C // heads
+    h = TF.layer_norm(x, (C,), t(w["ln1_g"]), t(w["ln1_b"]), eps) * (1 + t(md["scale1"])) + t(md["shift1"])
+    q, k, v = TF.linear(h, t(w["w_qkv"]), t(w["b_qkv"])).split(C, dim=1)
+    K, Vv = torch.cat([t(k_old), k]), torch.cat([t(v_old), v])
+    sh = lambda a: a.view(a.shape[0], heads, dh).transpose(0, 1)
+    o = TF.scaled_dot_product_attention(sh(q), sh(K), sh(Vv)).transpose(0, 1).reshape(x.shape[0], C)
+    x1 = x + t(md["gate1"]) * TF.linear(o, t(w["w_o"]), t(w["b_o"]))
+    h2 = TF.layer_norm(x1, (C,), t(w["ln2_g"]), t(w["ln2_b"]), eps) * (1 + t(md["scale2"])) + t(md["shift2"])
+    f = TF.linear(TF.gelu(TF.linear(h2, t(w["w_fc1"]), t(w["b_fc1"])), approximate="tanh"),
+                  t(w["w_fc2"]), t(w["b_fc2"]))
+    return (x1 + t(md["gate2"]) * f).numpy(), k.numpy(), v.numpy()
+
+
+def _rand_modulation(B, C, rng):
+    return {n: (0.5 * rng.standard_normal((B, C))).astype(np.float32) for n in oracle.MODULATION_NAMES}
+
+
+def test_modulated_block_matches_library_composition():
+    """Adaptive LayerNorm (per-image scale/shift after each LayerNorm, per-image gate on each branch)
+    against the same block composed from library ops per image, ragged keep counts."""
+    w, x, kc, vc, kv_len = _block_case(seed=4)
+    md = _rand_modulation(2, 16, np.random.default_rng(40))
+    ent = np.random.default_rng(9).standard_normal((2, 12)).astype(np.float32)
+    keep_idx, _, cu, _ = oracle.select_topk(ent, [7, 3])
+    y, k_new, v_new = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len, modulation=md)
+    for b in range(2):
+        idx = keep_idx[cu[b]:cu[b + 1]]
+        mb = {n: a[b] for n, a in md.items()}
+        wy, wk, wv = _torch_block_modulated(w, 1e-6, 2, x[b, idx], kc[b, :kv_len[b]], vc[b, :kv_len[b]], mb)
+        assert np.allclose(y[cu[b]:cu[b + 1]], wy, atol=2e-5, rtol=1e-5)
+        assert np.allclose(k_new[cu[b]:cu[b + 1]], wk, atol=1e-5)
+        assert np.allclose(v_new[cu[b]:cu[b + 1]], wv, atol=1e-5)
+
+
+def test_modulated_block_special_cases():
+    """What the modulation terms must reduce to: no scale, no shift, unit gates = the plain block,
+    bit for bit; both gates 0 = the identity on the kept rows whatever the rest holds; gate2 = 0 leaves
+    the attention half only, which does not depend on the second LayerNorm's modulation; a missing
+    entry means no such term."""
+    w, x, kc, vc, kv_len = _block_case(seed=6)
+    B, N, C = x.shape
+    ent = np.random.default_rng(3).standard_normal((B, N)).astype(np.float32)
+    keep_idx, _, cu, _ = oracle.select_topk(ent, [5, 9])
+    plain, pk, pv = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len)
+    zeros, ones = np.zeros((B, C), np.float32), np.ones((B, C), np.float32)
+    ident = dict(shift1=zeros, scale1=zeros, gate1=ones, shift2=zeros, scale2=zeros, gate2=ones)
+    y, k_new, v_new = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len, modulation=ident)
+    assert np.array_equal(y, plain) and np.array_equal(k_new, pk) and np.array_equal(v_new, pv)
+    y, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len, modulation={})
+    assert np.array_equal(y, plain)
+    md = _rand_modulation(B, C, np.random.default_rng(41))
+    md["gate1"], md["gate2"] = zeros, zeros
+    y, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len, modulation=md)
+    xk = np.concatenate([x[b, keep_idx[cu[b]:cu[b + 1]]] for b in range(B)])
+    assert np.array_equal(y, xk)
+    md = _rand_modulation(B, C, np.random.default_rng(42))
+    md["gate2"] = zeros
+    ya, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len, modulation=md)
+    md2 = dict(md, scale2=md["scale2"] + 3, shift2=md["shift2"] - 2)
+    yb, _, _ = oracle.pruned_block_forward(w, 1e-6, 2, x, keep_idx, cu, kc, vc, kv_len, modulation=md2)
+    assert np.array_equal(ya, yb)
+    assert not np.allclose(ya, plain, atol=1e-3)
+
+
 def test_block_keep_all_equals_dense_block_and_row_subset():
     w, x, kc, vc, kv_len = _block_case(seed=2)
     B, N, _ = x.shape
