@@ -215,6 +215,31 @@ nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block_weights* w
                                       void* k_cache, void* v_cache, int32_t* kv_len,
                                       int append_kv, void* y_kept, void* stream);
 
+/* ---- Eq. 14 with per-image adaptive LayerNorm (class-conditional VAR backbones) ------ */
+/*
+ * The paper accelerates existing VAR backbones and names only the layer's two parts (attention,
+ * FFN; Table 8). The class-conditional VAR models modulate each block per image from the
+ * condition embedding: LayerNorm output * (1 + scale) + shift before each part and a gate on each
+ * part's output. This call is nova_pruned_block_forward with those six per-image vectors:
+ *   h  = LN1(Xc) * (1 + scale1[b]) + shift1[b];   x1 = Xc + gate1[b] * (attention(h) W_o^T + b_o)
+ *   h2 = LN2(x1) * (1 + scale2[b]) + shift2[b];   y  = x1 + gate2[b] * (MLP(h2))
+ * where b is the image of the row and LN1/LN2 keep their own affine parameters from `w` (pass
+ * ones and zeros for a LayerNorm without them). Each pointer is device bf16 [B, C] or NULL (term
+ * absent); mod == NULL is the plain block. m_on_device != 0 makes s->M an upper bound as in
+ * nova_pruned_block_forward_device. Everything else as nova_pruned_block_forward.
+ */
+typedef struct nova_block_modulation {
+    const void *shift1, *scale1, *gate1;   /* attention half */
+    const void *shift2, *scale2, *gate2;   /* MLP half       */
+} nova_block_modulation;
+
+nova_status nova_pruned_block_forward_adaln(nova_ctx* ctx, const nova_block_weights* w,
+                                            const nova_block_modulation* mod,
+                                            const nova_block_shape* s, const void* x_in,
+                                            const int32_t* keep_idx, const int32_t* cu_keep,
+                                            void* k_cache, void* v_cache, int32_t* kv_len,
+                                            int append_kv, void* y_kept, int m_on_device, void* stream);
+
 /* ---- the same block for callers that cannot allocate device memory ------------------ */
 /*
  * (The paper has no counterpart to this call; it exists for deployment.)

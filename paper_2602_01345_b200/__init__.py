@@ -10,6 +10,6 @@ from .binding import (  # noqa: F401
     nova_pruned_block_forward, nova_restore_from_cache, nova_block_workspace_bytes,
     nova_pruned_block_forward_static, nova_static_scratch_bytes,
     nova_keep_ratios_device, nova_select_topk_device, nova_pruned_block_forward_device,
-    nova_restore_from_cache_device,
+    nova_restore_from_cache_device, nova_pruned_block_forward_adaln, MODULATION_NAMES,
     lib_path, STATUS_NAMES,
 )

@@ -343,3 +343,34 @@ def nova_restore_from_cache_device(ctx: Context, x_in, y_kept, keep_idx, prune_i
                                                   _ptr(prune_idx), _ptr(cu_keep), _ptr(cache_prev),
                                                   cache_prev.shape[1], cache_prev.shape[2], h, w, Cc, B,
                                                   _ptr(x_out), _ptr(cache_out), _stream(stream)))
+
+
+# ---- adaptive-LayerNorm block (per-image scale / shift / gate) ----------------------------------
+MODULATION_NAMES = ("shift1", "scale1", "gate1", "shift2", "scale2", "gate2")
+
+
+class _BlockModulation(C.Structure):
+    _fields_ = [(n, _vp) for n in MODULATION_NAMES]
+
+
+_lib.nova_pruned_block_forward_adaln.argtypes = [_vp, C.POINTER(_BlockWeights), C.POINTER(_BlockModulation),
+                                                 C.POINTER(_BlockShape), _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _i, _vp]
+_lib.nova_pruned_block_forward_adaln.restype = _i
+
+
+def nova_pruned_block_forward_adaln(ctx: Context, w: BlockWeights, modulation: dict, shape: BlockShape, x_in,
+                                    keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept,
+                                    m_on_device: bool = False, stream=None):
+    """nova_pruned_block_forward with per-image modulation: `modulation` maps names from
+    MODULATION_NAMES to device bf16 tensors [B, C] (a missing name or None = no such term)."""
+    ptrs = []
+    for n in MODULATION_NAMES:
+        t = modulation.get(n) if modulation else None
+        if t is not None:
+            assert t.dtype == torch.bfloat16 and t.shape == (shape.B, shape.C)
+        ptrs.append(_ptr(t))
+    cm = _BlockModulation(*ptrs)
+    c = shape._c()
+    ctx.check(_lib.nova_pruned_block_forward_adaln(
+        ctx.handle, C.byref(w.c), C.byref(cm), C.byref(c), _ptr(x_in), _ptr(keep_idx), _ptr(cu_keep), _ptr(k_cache),
+        _ptr(v_cache), _ptr(kv_len), int(bool(append_kv)), _ptr(y_kept), int(bool(m_on_device)), _stream(stream)))

@@ -19,7 +19,16 @@ struct RowMapArgs {
     int B, N, Lmax;
     int32_t* src_row;
     int32_t* kv_row;
+    int32_t* img_row;     // image of compacted row r
     unsigned int* status;
+};
+
+// Per-image modulation of a LayerNorm's output (adaptive LayerNorm): out * (1 + scale[b]) + shift[b].
+// scale / shift: [B, C] bf16 or NULL; img_row gives b for the kernels that do not build the maps.
+struct LnModArgs {
+    const uint4* scale;
+    const uint4* shift;
+    const int32_t* img_row;
 };
 
 // ---- LayerNorm ----------------------------------------------------------------------------
@@ -46,13 +55,15 @@ template <int VEC, bool MAPS>
 __global__ void __launch_bounds__(kLnWarps * 32)
 layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                float eps, int M, const int32_t* __restrict__ m_dev, int vec_per_row, uint4* __restrict__ out,
-               const RowMapArgs maps)
+               const RowMapArgs maps, const LnModArgs mod)
 {
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * kLnWarps + (threadIdx.x >> 5);
     if (m_dev) M = min(M, *m_dev);      // the host knows only an upper bound
     if (r >= M) return;
     long src = r;
+    int img = 0;
+    if (!MAPS && (mod.scale || mod.shift)) img = mod.img_row[r];
     if (MAPS) {
         // image of compacted row r: largest b with cu_keep[b] <= r
         int lo = 0, hi = maps.B;
@@ -62,8 +73,10 @@ layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, con
         }
         const int b = lo, c0 = maps.cu_keep[b];
         src = (long)b * maps.N + maps.keep_idx[r];
+        img = b;
         if (lane == 0) {
             maps.src_row[r] = (int32_t)src;
+            maps.img_row[r] = b;
             const int k_b = maps.cu_keep[b + 1] - c0, len = maps.kv_len[b];
             if (len + k_b > maps.Lmax) {
                 maps.kv_row[r] = -1;
@@ -117,13 +130,20 @@ layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, con
             const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
             const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, bw[4] = {bt.x, bt.y, bt.z, bt.w};
             uint32_t o[4];
+            uint32_t sc[4] = {0, 0, 0, 0}, sh[4] = {0, 0, 0, 0};        // bf16 zeros: no modulation
+            if (mod.scale) { const uint4 t = mod.scale[(long)img * vec_per_row + c]; sc[0] = t.x; sc[1] = t.y; sc[2] = t.z; sc[3] = t.w; }
+            if (mod.shift) { const uint4 t = mod.shift[(long)img * vec_per_row + c]; sh[0] = t.x; sh[1] = t.y; sh[2] = t.z; sh[3] = t.w; }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 // (x - mean) * rstd = x * rstd + shift
                 const float n0 = fmaf(__uint_as_float(w[q] << 16), rstd, shift);
                 const float n1 = fmaf(__uint_as_float(w[q] & 0xffff0000u), rstd, shift);
-                const float y0 = fmaf(n0, __uint_as_float(gw[q] << 16), __uint_as_float(bw[q] << 16));
-                const float y1 = fmaf(n1, __uint_as_float(gw[q] & 0xffff0000u), __uint_as_float(bw[q] & 0xffff0000u));
+                float y0 = fmaf(n0, __uint_as_float(gw[q] << 16), __uint_as_float(bw[q] << 16));
+                float y1 = fmaf(n1, __uint_as_float(gw[q] & 0xffff0000u), __uint_as_float(bw[q] & 0xffff0000u));
+                if (mod.scale || mod.shift) {
+                    y0 = fmaf(y0, 1.f + __uint_as_float(sc[q] << 16), __uint_as_float(sh[q] << 16));
+                    y1 = fmaf(y1, 1.f + __uint_as_float(sc[q] & 0xffff0000u), __uint_as_float(sh[q] & 0xffff0000u));
+                }
                 __nv_bfloat162 t = __floats2bfloat162_rn(y0, y1);
                 o[q] = *reinterpret_cast<uint32_t*>(&t);
             }
@@ -135,6 +155,7 @@ layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, con
 struct Workspace {
     int32_t* src_row;
     int32_t* kv_row;
+    int32_t* img_row;
     __nv_bfloat16 *h, *q, *o, *x1, *f;
     size_t bytes;
 };
@@ -154,6 +175,7 @@ Workspace carve(void* base, int M, int C, int F)
     w.o = (__nv_bfloat16*)take(Mp * C * 2);
     w.x1 = (__nv_bfloat16*)take(Mp * C * 2);
     w.f = (__nv_bfloat16*)take(Mp * (size_t)F * 2);
+    w.img_row = (int32_t*)take(Mp * 4);
     w.bytes = off;
     return w;
 }
@@ -171,7 +193,7 @@ bool shape_ok(const nova_block_shape* s)
 
 }  // namespace
 
-static nova_status launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const RowMapArgs* maps,
+static nova_status launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const RowMapArgs* maps, const LnModArgs& mod,
                              const __nv_bfloat16* g, const __nv_bfloat16* b, float eps, int M, const int32_t* m_dev,
                              int C, __nv_bfloat16* out, cudaStream_t st)
 {
@@ -184,8 +206,8 @@ static nova_status launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const RowMap
     nova_launch_scope scope(ctx, NOVA_K_LAYERNORM, st);
 #define NOVA_LN_CASE(V)                                                                                          \
     do {                                                                                                         \
-        if (maps) layernorm_rows<V, true><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, *maps); \
-        else layernorm_rows<V, false><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, none);      \
+        if (maps) layernorm_rows<V, true><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, *maps, mod); \
+        else layernorm_rows<V, false><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, none, mod);      \
     } while (0)
     if (per_lane <= 2) NOVA_LN_CASE(2);
     else if (per_lane <= 4) NOVA_LN_CASE(4);
@@ -206,7 +228,7 @@ extern "C" size_t nova_block_workspace_bytes(const nova_block_shape* s)
 
 // m_on_device: s->M is only an upper bound of the kept rows (it sizes grids, tensor maps and the
 // workspace); every kernel takes the true count from cu_keep[B] on the device.
-static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w,
+static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, const nova_block_modulation* mod,
                                  const nova_block_shape* s, const void* x_in,
                                  const int32_t* keep_idx, const int32_t* cu_keep,
                                  void* k_cache, void* v_cache, int32_t* kv_len,
@@ -236,12 +258,20 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w,
     typedef __nv_bfloat16* bf;
 
     const int32_t* m_dev = m_on_device ? cu_keep + s->B : nullptr;
+    nova_block_modulation md;
+    memset(&md, 0, sizeof(md));
+    if (mod) md = *mod;
+    const void* mp[] = {md.shift1, md.scale1, md.gate1, md.shift2, md.scale2, md.gate2};
+    for (const void* ptr : mp)
+        if (!nova_aligned16(ptr)) return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_pruned_block_forward: modulation not 16-byte aligned");
+    LnModArgs ln1_mod = {(const uint4*)md.scale1, (const uint4*)md.shift1, ws.img_row};
+    LnModArgs ln2_mod = {(const uint4*)md.scale2, (const uint4*)md.shift2, ws.img_row};
     nova_status rc;
     // h = LN1(gathered rows); the same kernel writes the row maps the GEMM epilogues use
     RowMapArgs maps;
     maps.keep_idx = keep_idx; maps.cu_keep = cu_keep; maps.kv_len = kv_len; maps.B = s->B; maps.N = s->N;
-    maps.Lmax = s->Lmax; maps.src_row = ws.src_row; maps.kv_row = ws.kv_row; maps.status = ctx->dev_status;
-    rc = launch_ln(ctx, (cbf)x_in, &maps, (cbf)w->ln1_g, (cbf)w->ln1_b, w->eps, M, m_dev, C, ws.h, st);
+    maps.Lmax = s->Lmax; maps.src_row = ws.src_row; maps.kv_row = ws.kv_row; maps.img_row = ws.img_row; maps.status = ctx->dev_status;
+    rc = launch_ln(ctx, (cbf)x_in, &maps, ln1_mod, (cbf)w->ln1_g, (cbf)w->ln1_b, w->eps, M, m_dev, C, ws.h, st);
     if (rc) return rc;
     // [q | k | v] = h W_qkv^T + b; k, v go straight to their cache rows
     nova_gemm_args g;
@@ -262,10 +292,11 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w,
     memset(&g, 0, sizeof(g));
     g.A = ws.o; g.W = (cbf)w->w_o; g.bias = (cbf)w->b_o; g.M = M; g.m_dev = m_dev; g.N = C; g.K = C;
     g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_PROJ; g.out = ws.x1; g.res = (cbf)x_in; g.res_row = ws.src_row;
+    g.gate = (cbf)md.gate1; g.img_row = ws.img_row;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
     // h = LN2(x1)
-    rc = launch_ln(ctx, ws.x1, nullptr, (cbf)w->ln2_g, (cbf)w->ln2_b, w->eps, M, m_dev, C, ws.h, st);
+    rc = launch_ln(ctx, ws.x1, nullptr, ln2_mod, (cbf)w->ln2_g, (cbf)w->ln2_b, w->eps, M, m_dev, C, ws.h, st);
     if (rc) return rc;
     // f = GELU(h W_fc1^T + b_fc1)
     memset(&g, 0, sizeof(g));
@@ -277,6 +308,7 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w,
     memset(&g, 0, sizeof(g));
     g.A = ws.f; g.W = (cbf)w->w_fc2; g.bias = (cbf)w->b_fc2; g.M = M; g.m_dev = m_dev; g.N = C; g.K = F;
     g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_FC2; g.out = (bf)y_kept; g.res = ws.x1; g.res_row = nullptr;
+    g.gate = (cbf)md.gate2; g.img_row = ws.img_row;
     if (append_kv) {
         // the last kernel of the block also advances kv_len: every reader of the old lengths (row
         // maps, attention) ran in an earlier kernel of this call
@@ -293,7 +325,7 @@ extern "C" nova_status nova_pruned_block_forward(nova_ctx* ctx, const nova_block
                                                  void* k_cache, void* v_cache, int32_t* kv_len,
                                                  int append_kv, void* y_kept, void* stream)
 {
-    return block_forward(ctx, w, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream, false);
+    return block_forward(ctx, w, nullptr, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream, false);
 }
 
 extern "C" nova_status nova_pruned_block_forward_device(nova_ctx* ctx, const nova_block_weights* w,
@@ -302,7 +334,18 @@ extern "C" nova_status nova_pruned_block_forward_device(nova_ctx* ctx, const nov
                                                         void* k_cache, void* v_cache, int32_t* kv_len,
                                                         int append_kv, void* y_kept, void* stream)
 {
-    return block_forward(ctx, w, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream, true);
+    return block_forward(ctx, w, nullptr, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream, true);
+}
+
+extern "C" nova_status nova_pruned_block_forward_adaln(nova_ctx* ctx, const nova_block_weights* w,
+                                                       const nova_block_modulation* mod,
+                                                       const nova_block_shape* s, const void* x_in,
+                                                       const int32_t* keep_idx, const int32_t* cu_keep,
+                                                       void* k_cache, void* v_cache, int32_t* kv_len,
+                                                       int append_kv, void* y_kept, int m_on_device, void* stream)
+{
+    return block_forward(ctx, w, mod, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream,
+                         m_on_device != 0);
 }
 
 // ---- block forward for callers that cannot allocate device memory --------------------------

@@ -128,6 +128,8 @@ struct nova_gemm_args {
     // residual epilogue
     const __nv_bfloat16* res;   // residual rows of width N
     const int32_t* res_row;     // row map into res, or NULL for identity
+    const __nv_bfloat16* gate;  // NULL, or [images, N]: out = res + gate[img_row[r]] * (acc + bias)
+    const int32_t* img_row;     // [M] image of each row (needed with gate)
     // QKV epilogue
     int C;
     __nv_bfloat16* k_cache;

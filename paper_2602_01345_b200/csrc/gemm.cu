@@ -68,6 +68,8 @@ struct GemmParams {
     int adv_B, adv_Lmax;
     float* ent;
     const int32_t* m_dev;
+    const __nv_bfloat16* gate;
+    const int32_t* img_row;
 };
 
 // Rows of this launch: p.M, or the device-side count when the host only knows an upper bound.
@@ -110,6 +112,20 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int row, int
         for (int i = 0; i < 32; ++i) v[i] = gelu_tanh(v[i]);
         dst = p.out + (long)row * p.N + col0;
     } else if (p.epilogue == NOVA_EPI_BIAS_RES) {
+        if (p.gate) {
+            // per-image gate of the branch: out = residual + gate * (acc + bias)
+            const uint4* g4 = (const uint4*)(p.gate + (long)p.img_row[row] * p.N + col0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 g = g4[i];
+                const uint32_t gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    v[i * 8 + j * 2] *= __uint_as_float(gw[j] << 16);
+                    v[i * 8 + j * 2 + 1] *= __uint_as_float(gw[j] & 0xffff0000u);
+                }
+            }
+        }
         const uint4* r4 = (const uint4*)(p.res + res_base + col0);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -256,7 +272,7 @@ GemmParams make_params(nova_ctx* ctx, const nova_gemm_args& a)
     p.res = a.res; p.res_row = a.res_row; p.C = a.C; p.k_cache = a.k_cache; p.v_cache = a.v_cache;
     p.kv_row = a.kv_row; p.status = ctx->dev_status;
     p.adv_cu_keep = a.adv_cu_keep; p.adv_kv_len = a.adv_kv_len; p.adv_B = a.adv_B; p.adv_Lmax = a.adv_Lmax;
-    p.ent = a.ent; p.m_dev = a.m_dev;
+    p.ent = a.ent; p.m_dev = a.m_dev; p.gate = a.gate; p.img_row = a.img_row;
     return p;
 }
 

@@ -513,6 +513,90 @@ def test_block_2048_shape_sampled_rows(ctx):
                 rows=np.array(rows, np.int32))
 
 
+def _modulation(B, C, seed, names=nova.MODULATION_NAMES):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    return {n: (0.5 * torch.randn((B, C), generator=g)).to(torch.bfloat16).to(DEV) for n in names}
+
+
+@pytest.mark.parametrize("case", ["small_dh64_ragged", "var_d16_256_shape", "gates_only", "device_count"])
+def test_block_adaptive_layernorm_matches_oracle(ctx, case):
+    """The block with per-image adaptive-LayerNorm modulation (scale and shift after each LayerNorm,
+    a gate on each branch) against the oracle: a small ragged case, the 256x256 VAR-d16 shape (last
+    scale, batch 4, half kept, sampled rows), a subset of the terms, and the launch sized by an upper
+    bound with the kept count read on the device."""
+    if case == "var_d16_256_shape":
+        ms = synth.CONFIGS["c2_var_d16_256"]
+        B, N, C, heads, F, Lmax = 4, ms.scales[-1] ** 2, ms.C, ms.heads, ms.F, ms.total_tokens
+        ks, kv_lens = [128, 97, 128, 160], [Lmax - N] * 4
+        rows = np.array([0, 127, 128, 224, 225, 352, 353, sum(ks) - 1], np.int32)
+    else:
+        B, N, C, heads, F, Lmax = 3, 200, 128, 2, 256, 512
+        ks, kv_lens, rows = [200, 77, 1], [0, 130, 300], None
+    names = ("gate1", "gate2") if case == "gates_only" else nova.MODULATION_NAMES
+    md = _modulation(B, C, 77, names)
+    wt = synth.block_weights(C, F, 31, DEV)
+    x = synth.activations(B, N, C, 32, DEV)
+    k_cache, v_cache, _ = synth.kv_cache(B, Lmax, max(kv_lens), C, 33, DEV)
+    kv_len = torch.tensor(kv_lens, dtype=torch.int32, device=DEV)
+    ent = torch.rand((B, N), generator=torch.Generator(device="cpu").manual_seed(31))
+    keep_idx, _, cu, _ = gpu_select(ctx, ent.to(DEV), ks)
+    M = sum(ks)
+    on_device = case == "device_count"
+    cap = B * N if on_device else M
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, cap)
+    ctx.ensure_workspace(shape)
+    y = torch.full((cap, C), float("nan"), dtype=torch.bfloat16, device=DEV)
+    k0, v0 = k_cache.clone(), v_cache.clone()
+    idx_buf = torch.zeros(cap, dtype=torch.int32, device=DEV)
+    idx_buf[:M] = keep_idx
+    nova.nova_pruned_block_forward_adaln(ctx, nova.BlockWeights(wt, 1e-6), md, shape, x, idx_buf, cu, k_cache, v_cache,
+                                         kv_len, True, y, m_on_device=on_device)
+    assert ctx.device_status() == 0
+    wy, wk, wv = oracle.pruned_block_forward({n: f32(t) for n, t in wt.items()}, 1e-6, heads, f32(x),
+                                             keep_idx.cpu().numpy(), cu.cpu().numpy(), f32(k0), f32(v0),
+                                             np.array(kv_lens, np.int32), rows=rows,
+                                             modulation={n: f32(t) for n, t in md.items()})
+    gy = f32(y[:M])
+    if rows is not None:
+        gy = gy[rows]
+    assert np.isfinite(gy).all()
+    assert _rel_err(gy, wy) <= BLOCK_TOL
+    cuu = cu.cpu().numpy()
+    for b in range(B):
+        n0, kb = kv_lens[b], ks[b]
+        assert _rel_err(f32(k_cache)[b, n0:n0 + kb], wk[cuu[b]:cuu[b + 1]]) <= BLOCK_TOL
+        assert _rel_err(f32(v_cache)[b, n0:n0 + kb], wv[cuu[b]:cuu[b + 1]]) <= BLOCK_TOL
+    if on_device:
+        assert torch.isnan(y[M:].float()).all()          # rows past the device-side count are untouched
+    # and the terms really act: the plain block gives something else
+    y_plain = _run_block(ctx, nova.BlockShape(B, N, C, heads, F, Lmax, M), nova.BlockWeights(wt, 1e-6), x, keep_idx, cu,
+                         k0.clone(), v0.clone(), torch.tensor(kv_lens, dtype=torch.int32, device=DEV))
+    assert _rel_err(f32(y_plain)[rows] if rows is not None else f32(y_plain), wy) > 2 * BLOCK_TOL
+
+
+def test_block_adaptive_layernorm_identity_equals_plain_block(ctx):
+    """Zero scale and shift with unit gates, and a NULL modulation, give the plain block bit for bit."""
+    B, N, C, heads, F, Lmax = 2, 256, 1024, 16, 4096, 680
+    ks, kv_lens = [128, 101], [424, 424]
+    wt = nova.BlockWeights(synth.block_weights(C, F, 3, DEV), 1e-6)
+    x = synth.activations(B, N, C, 4, DEV)
+    k_cache, v_cache, _ = synth.kv_cache(B, Lmax, 424, C, 5, DEV)
+    ent = torch.rand((B, N), generator=torch.Generator(device="cpu").manual_seed(3))
+    keep_idx, _, cu, _ = gpu_select(ctx, ent.to(DEV), ks)
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, sum(ks))
+    kv = lambda: torch.tensor(kv_lens, dtype=torch.int32, device=DEV)
+    y_plain = _run_block(ctx, shape, wt, x, keep_idx, cu, k_cache.clone(), v_cache.clone(), kv())
+    zeros = torch.zeros((B, C), dtype=torch.bfloat16, device=DEV)
+    ones = torch.ones((B, C), dtype=torch.bfloat16, device=DEV)
+    ident = dict(shift1=zeros, scale1=zeros, gate1=ones, shift2=zeros, scale2=zeros, gate2=ones)
+    for md in (ident, None):
+        y = torch.empty_like(y_plain)
+        nova.nova_pruned_block_forward_adaln(ctx, wt, md, shape, x, keep_idx, cu, k_cache.clone(), v_cache.clone(),
+                                             kv(), True, y)
+        assert torch.equal(y, y_plain)
+    assert ctx.device_status() == 0
+
+
 def test_block_without_append_leaves_kv_len(ctx):
     B, N, C, heads, F, Lmax = 1, 64, 128, 2, 256, 256
     wt = synth.block_weights(C, F, 1, DEV)
