@@ -35,7 +35,7 @@ UNIT = "images/s"
 # for any other workload, and reset to None whenever the kernel changes after the capture.
 # attention: one launch; gemm: average over the four launches of a layer (qkv, proj, fc1, fc2), the
 # unit `achieved` is taken over as well. Source: profiles/layer_kernels_c4_1024_batch4_keep0.5.txt.
-NCU_TRAFFIC_BYTES = {"attention": 351_096_576, "gemm": 171_372_416}
+NCU_TRAFFIC_BYTES = {"attention": 351_413_504, "gemm": 172_203_776}
 
 
 def parse_args():
@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="override the number of layers (small profiling cases)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-next", action="store_true",
+                    help="skip the extra timings after the timed region (fused head entropy, device-driven step)")
     return ap.parse_args()
 
 
@@ -295,54 +297,56 @@ def run_ours(args):
         us = b0.elapsed_time(b1) * 1e3 / len(st["logits"])
         key = "gbs_back_to_back" if with_mean else "gbs_back_to_back_no_mean"
         kernels["entropy_rows"][key] = round(ent_bytes / us / 1e3, 1)
-    # Entropy fused with the codebook head (the step before the path: hidden states -> entropy, the
-    # 8 KiB/token of logits never stored), timed back to back over 8 calls outside the timed region.
-    head_w = synth.randn_bf16((synth.V_CODEBOOK, ms.C), 991, dev, std=3.0 / ms.C ** 0.5)
-    hidden = [synth.activations(B, N, ms.C, 900 + i, dev) for i in range(4)]
-    for _ in range(2):
-        nova.nova_head_entropy(ctx, hidden[0], head_w, None, ent_buf, mean_buf, stream=stream)
-    torch.cuda.synchronize()
-    b0.record(stream)
-    for i in range(8):
-        nova.nova_head_entropy(ctx, hidden[i % 4], head_w, None, ent_buf, mean_buf, stream=stream)
-    b1.record(stream)
-    torch.cuda.synchronize()
-    head_us = b0.elapsed_time(b1) * 1e3 / 8
-    head_tf = 2.0 * rows * ms.C * synth.V_CODEBOOK / head_us / 1e6
-    head_entropy = {"us_per_call": round(head_us, 1), "tflops": round(head_tf, 1),
-                    "frac_of_tensor_peak": round(head_tf / pk["tensor"], 4),
-                    "logits_bytes_not_written_or_read": int(2 * rows * synth.V_CODEBOOK * 2)}
-    assert ctx.device_status() == 0, "device status after the head-entropy timing"
-    # The same step with every decision left on the device (Eq. 8-13 in a kernel, kept counts read
-    # from device memory, launches sized by the upper bound B*N): issued eagerly, and recorded once
-    # in a CUDA graph and replayed. Same inputs and buffers as the timed region above.
-    hist_dev = hbar_scale.t().contiguous().to(dev)
-    drun = pipeline.DeviceScaleRunner(ctx, st["weights"], ms.heads, B, wd["h"], wd["w"], wd["Lmax"], st["k_caches"],
-                                      st["v_caches"], st["kv_len"], st["cache_prev"], sched, wd["t"], hist_dev,
-                                      synth.V_CODEBOOK, x_in=st["x_in"], layer_logits=st["logits"], scale_entropy=False)
-    st["kv_len"].copy_(st["kv_len0"])
-    l0 = pipeline.launch_count(ctx)
-    drun.capture()
-    dev_launches = (pipeline.launch_count(ctx) - l0) // 2          # one eager pass + one recorded pass
-    dev_ms = {}
-    for mode in ("eager", "graph"):
-        for it in range(args.warmup + args.steps):
-            if it == args.warmup:
-                torch.cuda.synchronize()
-                b0.record(stream)
-            st["kv_len"].copy_(st["kv_len0"])
-            if mode == "eager":
-                drun.enqueue(stream=stream)
-            else:
-                drun.replay()
+    head_entropy = device_schedule = None
+    if not args.no_next:
+        # Entropy fused with the codebook head (the step before the path: hidden states -> entropy, the
+        # 8 KiB/token of logits never stored), timed back to back over 8 calls outside the timed region.
+        head_w = synth.randn_bf16((synth.V_CODEBOOK, ms.C), 991, dev, std=3.0 / ms.C ** 0.5)
+        hidden = [synth.activations(B, N, ms.C, 900 + i, dev) for i in range(4)]
+        for _ in range(2):
+            nova.nova_head_entropy(ctx, hidden[0], head_w, None, ent_buf, mean_buf, stream=stream)
+        torch.cuda.synchronize()
+        b0.record(stream)
+        for i in range(8):
+            nova.nova_head_entropy(ctx, hidden[i % 4], head_w, None, ent_buf, mean_buf, stream=stream)
         b1.record(stream)
         torch.cuda.synchronize()
-        dev_ms[mode] = b0.elapsed_time(b1) / args.steps
-    assert ctx.device_status() == 0, "device status after the device-driven timing"
-    same = bool(torch.equal(drun.x_out, x_out)) and bool(torch.equal(drun.keep.cpu(), torch.stack(keeps)))
-    device_schedule = {"ms_per_step_eager": round(dev_ms["eager"], 4), "ms_per_step_graph": round(dev_ms["graph"], 4),
-                       "ms_per_step_host_driven": round(ms_per_step, 4), "launches_per_step": int(dev_launches),
-                       "host_syncs_per_step": 0, "equals_host_driven_result": same}
+        head_us = b0.elapsed_time(b1) * 1e3 / 8
+        head_tf = 2.0 * rows * ms.C * synth.V_CODEBOOK / head_us / 1e6
+        head_entropy = {"us_per_call": round(head_us, 1), "tflops": round(head_tf, 1),
+                        "frac_of_tensor_peak": round(head_tf / pk["tensor"], 4),
+                        "logits_bytes_not_written_or_read": int(2 * rows * synth.V_CODEBOOK * 2)}
+        assert ctx.device_status() == 0, "device status after the head-entropy timing"
+        # The same step with every decision left on the device (Eq. 8-13 in a kernel, kept counts read
+        # from device memory, launches sized by the upper bound B*N): issued eagerly, and recorded once
+        # in a CUDA graph and replayed. Same inputs and buffers as the timed region above.
+        hist_dev = hbar_scale.t().contiguous().to(dev)
+        drun = pipeline.DeviceScaleRunner(ctx, st["weights"], ms.heads, B, wd["h"], wd["w"], wd["Lmax"], st["k_caches"],
+                                          st["v_caches"], st["kv_len"], st["cache_prev"], sched, wd["t"], hist_dev,
+                                          synth.V_CODEBOOK, x_in=st["x_in"], layer_logits=st["logits"], scale_entropy=False)
+        st["kv_len"].copy_(st["kv_len0"])
+        l0 = pipeline.launch_count(ctx)
+        drun.capture()
+        dev_launches = (pipeline.launch_count(ctx) - l0) // 2          # one eager pass + one recorded pass
+        dev_ms = {}
+        for mode in ("eager", "graph"):
+            for it in range(args.warmup + args.steps):
+                if it == args.warmup:
+                    torch.cuda.synchronize()
+                    b0.record(stream)
+                st["kv_len"].copy_(st["kv_len0"])
+                if mode == "eager":
+                    drun.enqueue(stream=stream)
+                else:
+                    drun.replay()
+            b1.record(stream)
+            torch.cuda.synchronize()
+            dev_ms[mode] = b0.elapsed_time(b1) / args.steps
+        assert ctx.device_status() == 0, "device status after the device-driven timing"
+        same = bool(torch.equal(drun.x_out, x_out)) and bool(torch.equal(drun.keep.cpu(), torch.stack(keeps)))
+        device_schedule = {"ms_per_step_eager": round(dev_ms["eager"], 4), "ms_per_step_graph": round(dev_ms["graph"], 4),
+                           "ms_per_step_host_driven": round(ms_per_step, 4), "launches_per_step": int(dev_launches),
+                           "host_syncs_per_step": 0, "equals_host_driven_result": same}
     for k in ("entropy_rows", "restore"):
         if "gbs" in kernels.get(k, {}):
             kernels[k]["frac_of_hbm_peak"] = round(kernels[k]["gbs"] / pk["hbm"], 4)

@@ -51,7 +51,7 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-template <int VEC, bool MAPS>
+template <int VEC, bool MAPS, bool MOD>
 __global__ void __launch_bounds__(kLnWarps * 32)
 layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                float eps, int M, const int32_t* __restrict__ m_dev, int vec_per_row, uint4* __restrict__ out,
@@ -63,7 +63,7 @@ layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, con
     if (r >= M) return;
     long src = r;
     int img = 0;
-    if (!MAPS && (mod.scale || mod.shift)) img = mod.img_row[r];
+    if (MOD && !MAPS) img = mod.img_row[r];
     if (MAPS) {
         // image of compacted row r: largest b with cu_keep[b] <= r
         int lo = 0, hi = maps.B;
@@ -131,8 +131,8 @@ layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, con
             const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, bw[4] = {bt.x, bt.y, bt.z, bt.w};
             uint32_t o[4];
             uint32_t sc[4] = {0, 0, 0, 0}, sh[4] = {0, 0, 0, 0};        // bf16 zeros: no modulation
-            if (mod.scale) { const uint4 t = mod.scale[(long)img * vec_per_row + c]; sc[0] = t.x; sc[1] = t.y; sc[2] = t.z; sc[3] = t.w; }
-            if (mod.shift) { const uint4 t = mod.shift[(long)img * vec_per_row + c]; sh[0] = t.x; sh[1] = t.y; sh[2] = t.z; sh[3] = t.w; }
+            if (MOD && mod.scale) { const uint4 t = mod.scale[(long)img * vec_per_row + c]; sc[0] = t.x; sc[1] = t.y; sc[2] = t.z; sc[3] = t.w; }
+            if (MOD && mod.shift) { const uint4 t = mod.shift[(long)img * vec_per_row + c]; sh[0] = t.x; sh[1] = t.y; sh[2] = t.z; sh[3] = t.w; }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 // (x - mean) * rstd = x * rstd + shift
@@ -140,7 +140,7 @@ layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, con
                 const float n1 = fmaf(__uint_as_float(w[q] & 0xffff0000u), rstd, shift);
                 float y0 = fmaf(n0, __uint_as_float(gw[q] << 16), __uint_as_float(bw[q] << 16));
                 float y1 = fmaf(n1, __uint_as_float(gw[q] & 0xffff0000u), __uint_as_float(bw[q] & 0xffff0000u));
-                if (mod.scale || mod.shift) {
+                if (MOD) {
                     y0 = fmaf(y0, 1.f + __uint_as_float(sc[q] << 16), __uint_as_float(sh[q] << 16));
                     y1 = fmaf(y1, 1.f + __uint_as_float(sc[q] & 0xffff0000u), __uint_as_float(sh[q] & 0xffff0000u));
                 }
@@ -204,17 +204,23 @@ static nova_status launch_ln(nova_ctx* ctx, const __nv_bfloat16* x, const RowMap
     RowMapArgs none;
     memset(&none, 0, sizeof(none));
     nova_launch_scope scope(ctx, NOVA_K_LAYERNORM, st);
+#define NOVA_LN_LAUNCH(V, MAPS, MOD, MAPARG)                                                                     \
+    layernorm_rows<V, MAPS, MOD><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, MAPARG, mod)
 #define NOVA_LN_CASE(V)                                                                                          \
     do {                                                                                                         \
-        if (maps) layernorm_rows<V, true><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, *maps, mod); \
-        else layernorm_rows<V, false><<<grid, block, 0, st>>>((const uint4*)x, (const uint4*)g, (const uint4*)b, eps, M, m_dev, vec, (uint4*)out, none, mod);      \
+        if (maps && modulated) NOVA_LN_LAUNCH(V, true, true, *maps);                                             \
+        else if (maps) NOVA_LN_LAUNCH(V, true, false, *maps);                                                    \
+        else if (modulated) NOVA_LN_LAUNCH(V, false, true, none);                                                \
+        else NOVA_LN_LAUNCH(V, false, false, none);                                                              \
     } while (0)
+    const bool modulated = mod.scale || mod.shift;
     if (per_lane <= 2) NOVA_LN_CASE(2);
     else if (per_lane <= 4) NOVA_LN_CASE(4);
     else if (per_lane <= 8) NOVA_LN_CASE(8);
     else if (per_lane <= 16) NOVA_LN_CASE(16);
     else if (per_lane <= 32) NOVA_LN_CASE(32);
     else return nova_fail(ctx, NOVA_ERR_SHAPE, "layernorm: C > 8192");
+#undef NOVA_LN_LAUNCH
 #undef NOVA_LN_CASE
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
