@@ -239,6 +239,7 @@ def run_ours(args):
     value = replica_throughput(world, B, ms_per_step)
     status = ctx.device_status()
     assert status == 0, f"device status after the timed region: {nova.STATUS_NAMES.get(status, status)}"
+    assert bool(torch.isfinite(x_out.float()).all()), "the timed step produced non-finite outputs"
 
     # ---- rooflines from the events recorded around every launch inside the timed region. The two
     # contractions (the attention kernel and the GEMM kernel, four launches per layer) take about

@@ -29,6 +29,22 @@ if not os.path.exists(_LIB_PATH):
     raise ImportError(
         f"{_LIB_PATH} not found: build it with `python -m paper_2602_01345_b200.build` "
         "(there is no CPU fallback for the NOVA kernels)")
+
+
+def _stale_sources():
+    """Source files newer than the built library (a library built from other sources than the
+    ones on disk gives results nobody can account for)."""
+    here = os.path.dirname(os.path.abspath(__file__))
+    built = os.path.getmtime(_LIB_PATH)
+    srcs = [os.path.join(here, "csrc", f) for f in os.listdir(os.path.join(here, "csrc"))]
+    srcs.append(os.path.join(os.path.dirname(here), "include", "nova.h"))
+    return [p for p in srcs if os.path.exists(p) and os.path.getmtime(p) > built + 1.0]
+
+
+if _stale_sources() and not os.environ.get("NOVA_ALLOW_STALE_LIBRARY"):
+    import warnings
+    warnings.warn("libnova.so is older than " + ", ".join(os.path.basename(p) for p in _stale_sources()) +
+                  ": rebuild with `python -m paper_2602_01345_b200.build`", RuntimeWarning, stacklevel=2)
 _lib = C.CDLL(_LIB_PATH)
 
 

@@ -440,6 +440,17 @@ def test_block_full_size_1024_shape_sampled_rows(ctx):
                 rows=np.array(rows, np.int32))
 
 
+def test_block_benchmark_configuration_sampled_rows(ctx):
+    """Exactly the launch the benchmark times: batch 4, 2048 of 4096 tokens kept per image, 6425 prior
+    keys. 512 attention work items on 148 SMs leave a last wave of 68, which is the partly key-split
+    case (444 whole items, 68 shared by two CTAs each); sampled rows include the first and last query
+    blocks of every image and heads on both sides of the split."""
+    ks = [2048] * 4
+    rows = [0, 255, 256, 1791, 1792, 2047, 2048, 4095, 4096, 6143, 6144, 6400, 7935, 7936, 8191]
+    _block_case(ctx, B=4, N=4096, C=2048, heads=16, F=8192, Lmax=10521, ks=ks, kv_lens=[6425] * 4, seed=19,
+                rows=np.array(rows, np.int32))
+
+
 def test_block_attention_ragged_mid_size(ctx):
     """Thousands of kept rows per image at head size 128, with keep counts and cache lengths that
     leave partial 256-row query blocks, blocks with only one of the two query tiles in use, and
