@@ -345,9 +345,11 @@ def run_ours(args):
             dev_ms[mode] = b0.elapsed_time(b1) / args.steps
         assert ctx.device_status() == 0, "device status after the device-driven timing"
         same = bool(torch.equal(drun.x_out, x_out)) and bool(torch.equal(drun.keep.cpu(), torch.stack(keeps)))
+        max_diff = float((drun.x_out.float() - x_out.float()).abs().max())
         device_schedule = {"ms_per_step_eager": round(dev_ms["eager"], 4), "ms_per_step_graph": round(dev_ms["graph"], 4),
                            "ms_per_step_host_driven": round(ms_per_step, 4), "launches_per_step": int(dev_launches),
-                           "host_syncs_per_step": 0, "equals_host_driven_result": same}
+                           "host_syncs_per_step": 0, "equals_host_driven_result": same,
+                           "max_abs_diff_vs_host_driven": max_diff}
     for k in ("entropy_rows", "restore"):
         if "gbs" in kernels.get(k, {}):
             kernels[k]["frac_of_hbm_peak"] = round(kernels[k]["gbs"] / pk["hbm"], 4)

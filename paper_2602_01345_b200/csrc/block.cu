@@ -290,8 +290,10 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
     nova_attn_args a;
     a.q = ws.q; a.k_cache = (cbf)k_cache; a.v_cache = (cbf)v_cache; a.cu_keep = cu_keep; a.kv_len = kv_len;
     a.o = ws.o; a.B = s->B; a.C = C; a.n_heads = s->n_heads; a.Lmax = s->Lmax; a.M = M;
-    a.scratch = ws.f;              // the MLP's hidden buffer is not in use yet
-    a.scratch_bytes = (size_t)((M + 127) / 128) * 128 * (size_t)F * 2;
+    // neither the projection's output buffer nor the MLP's hidden buffer is in use yet, and they lie
+    // next to each other: together they hold the partial results of a key-split last wave
+    a.scratch = ws.x1;
+    a.scratch_bytes = (size_t)((char*)ws.f - (char*)ws.x1) + (size_t)((M + 127) / 128) * 128 * (size_t)F * 2;
     rc = nova_launch_attention(ctx, a, st);
     if (rc) return rc;
     // x1 = Xc + o W_o^T + b_o
