@@ -23,8 +23,12 @@ class PrunedScaleRunner:
     """
 
     def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, h: int, w: int, Lmax: int,
-                 k_caches, v_caches, kv_len, cache_prev, eps: float = 1e-6, keep_cache_out: bool = True):
+                 k_caches, v_caches, kv_len, cache_prev, eps: float = 1e-6, keep_cache_out: bool = True,
+                 modulation=None):
+        """modulation: optional list of L dicts of per-image [B, C] bf16 tensors (adaptive LayerNorm
+        of the class-conditional backbones, see nova_pruned_block_forward_adaln)."""
         self.ctx = ctx
+        self.modulation = modulation
         self.L = len(weights)
         self.B, self.h, self.w, self.N = B, h, w, h * w
         self.C = weights[0]["w_o"].shape[0]
@@ -84,9 +88,15 @@ class PrunedScaleRunner:
                 nv.nova_select_topk(ctx, self.ent[j], keep, self.keep_idx[:M], self.prune_idx[: B * N - M],
                                     self.cu_keep, None, stream=st)
                 shape = nv.BlockShape(B, N, self.C, self.n_heads, self.F, self.Lmax, M)
-                nv.nova_pruned_block_forward(ctx, self.weights[j], shape, x, self.keep_idx[:M], self.cu_keep,
-                                             self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
-                                             self.y_kept[:M], stream=st)
+                if self.modulation is None:
+                    nv.nova_pruned_block_forward(ctx, self.weights[j], shape, x, self.keep_idx[:M], self.cu_keep,
+                                                 self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
+                                                 self.y_kept[:M], stream=st)
+                else:
+                    nv.nova_pruned_block_forward_adaln(ctx, self.weights[j], self.modulation[j], shape, x,
+                                                       self.keep_idx[:M], self.cu_keep, self.k_caches[j],
+                                                       self.v_caches[j], self.kv_len[j], append_kv, self.y_kept[:M],
+                                                       stream=st)
                 x_out = self.x_buf[j & 1] if x is not self.x_buf[j & 1] else self.x_buf[(j + 1) & 1]
                 nv.nova_restore_from_cache(ctx, x, self.y_kept[:M], self.keep_idx[:M], self.prune_idx[: B * N - M],
                                            self.cu_keep, self.cache_prev[j], self.h, self.w, x_out,
@@ -174,10 +184,11 @@ class DeviceScaleRunner:
     def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, h: int, w: int, Lmax: int,
                  k_caches, v_caches, kv_len, cache_prev, sched: nv.SchedParams, t: int, hist, V: int,
                  eps: float = 1e-6, logits_dtype=torch.bfloat16, x_in=None, layer_logits=None,
-                 scale_entropy: bool = True):
+                 scale_entropy: bool = True, modulation=None):
         """x_in / layer_logits: existing tensors to use as the fixed input buffers instead of new
         ones. scale_entropy=False: hist row t-1 is already filled by the caller (no scale_logits)."""
         self.ctx, self.sched, self.t = ctx, sched, t
+        self.modulation = modulation          # optional list of L dicts of [B, C] bf16 tensors (fixed buffers)
         self.L = len(weights)
         self.B, self.h, self.w, self.N = B, h, w, h * w
         self.C = weights[0]["w_o"].shape[0]
@@ -226,9 +237,14 @@ class DeviceScaleRunner:
                                        self.t_star, self.act_scale, stream=st)
             nv.nova_select_topk_device(ctx, self.ent[j], self.keep[j], self.keep_idx, self.prune_idx, self.cu_keep,
                                        None, stream=st)
-            nv.nova_pruned_block_forward_device(ctx, self.weights[j], self.shape, x, self.keep_idx, self.cu_keep,
-                                                self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
-                                                self.y_kept, stream=st)
+            if self.modulation is None:
+                nv.nova_pruned_block_forward_device(ctx, self.weights[j], self.shape, x, self.keep_idx, self.cu_keep,
+                                                    self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
+                                                    self.y_kept, stream=st)
+            else:
+                nv.nova_pruned_block_forward_adaln(ctx, self.weights[j], self.modulation[j], self.shape, x,
+                                                   self.keep_idx, self.cu_keep, self.k_caches[j], self.v_caches[j],
+                                                   self.kv_len[j], append_kv, self.y_kept, m_on_device=True, stream=st)
             x_out = self.x_buf[j & 1]
             nv.nova_restore_from_cache_device(ctx, x, self.y_kept, self.keep_idx, self.prune_idx, self.cu_keep,
                                               self.cache_prev[j], self.h, self.w, x_out, self.cache_out[j], stream=st)

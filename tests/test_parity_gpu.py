@@ -952,3 +952,60 @@ def test_scale_graph_replay(ctx):
         outs.append(r.keep.cpu().clone())
     assert (outs[0] < N).any()
     assert not torch.equal(outs[0], outs[1])
+
+
+def test_runners_with_modulation_agree_and_match_oracle(ctx):
+    """The scale runners pass per-image adaptive-LayerNorm modulation through: host-driven and
+    device-driven runs of two layers of the 256x256 shape agree, and the first layer's output equals
+    the oracle's modulated block followed by its restore."""
+    from paper_2602_01345_b200 import pipeline
+    ms = synth.CONFIGS["c2_var_d16_256"]
+    B, L, T = 2, 2, len(ms.scales)
+    side = ms.scales[-1]
+    N, V, C, Lmax = side * side, synth.V_CODEBOOK, ms.C, ms.total_tokens
+    prior = Lmax - N
+    weights = [synth.block_weights(C, ms.F, 100 + j, DEV) for j in range(L)]
+    mods = [_modulation(B, C, 900 + j) for j in range(L)]
+    hp = ms.scales[-2]
+    cache_prev = [synth.residual_cache(B, hp, hp, C, 70 + j, DEV) for j in range(L)]
+    x_in = synth.activations(B, N, C, 7, DEV)
+    a = synth.smooth_temperature_field(B, side, side, 5, a_lo=0.5, a_hi=6.0, device=DEV)
+    logits = [synth.logits_from_temperature(a * (1 + 0.1 * j), V, 20 + j) for j in range(L)]
+    sched = nova.SchedParams(force_act_scale=T, force_keep_ratio=0.5)
+    hbar = torch.linspace(2.0, 7.0, T).repeat(B, 1).contiguous()
+
+    def caches():
+        ks, vs = [], []
+        for j in range(L):
+            k, v, _ = synth.kv_cache(B, Lmax, prior, C, 50 + 2 * j, DEV)
+            ks.append(k)
+            vs.append(v)
+        return ks, vs, torch.full((L, B), prior, dtype=torch.int32, device=DEV)
+
+    k1, v1, len1 = caches()
+    host = pipeline.PrunedScaleRunner(ctx, weights, ms.heads, B, side, side, Lmax, k1, v1, len1, cache_prev,
+                                      modulation=mods)
+    xh, keeps = host.run_scale(x_in, logits, sched, T, hbar)
+    xh = xh.clone()
+    k2, v2, len2 = caches()
+    devr = pipeline.DeviceScaleRunner(ctx, weights, ms.heads, B, side, side, Lmax, k2, v2, len2, cache_prev, sched, T,
+                                      hbar.t().contiguous().to(DEV), V, x_in=x_in, layer_logits=logits,
+                                      scale_entropy=False, modulation=mods)
+    xd = devr.enqueue()
+    assert ctx.device_status() == 0
+    # Same keep counts and, for the first layer, the same appended keys bit for bit. The outputs may
+    # differ by bf16 rounding: the device-driven launch is sized by the upper bound B*N, which here
+    # gives the attention kernel enough scratch to share its 32 work items between CTA pairs, while
+    # the host-driven launch (sized by the true 256 rows) runs them unsplit.
+    assert torch.equal(torch.stack(keeps), devr.keep.cpu())
+    assert torch.equal(k1[0], k2[0])
+    assert _rel_err(f32(xd), f32(xh)) <= BLOCK_TOL / 2
+    # layer 1 against the oracle (teacher-forced on the GPU's entropies)
+    k0, v0, _ = synth.kv_cache(B, Lmax, prior, C, 50, DEV)
+    w_keep, w_prune, w_cu, _ = oracle.select_topk(host.ent[0].cpu().numpy(), keeps[0].numpy())
+    wy, _, _ = oracle.pruned_block_forward({n: f32(t) for n, t in weights[0].items()}, 1e-6, ms.heads, f32(x_in), w_keep,
+                                           w_cu, f32(k0), f32(v0), np.full(B, prior, np.int32),
+                                           modulation={n: f32(t) for n, t in mods[0].items()})
+    w_x1, _ = oracle.restore_from_cache(f32(x_in), wy, w_keep, w_prune, w_cu, f32(cache_prev[0]), side, side)
+    # the runner's layer-1 output is x_buf[0]; layer 2 wrote x_buf[1]
+    assert _rel_err(f32(host.x_buf[0]), w_x1) <= BLOCK_TOL
