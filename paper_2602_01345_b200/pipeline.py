@@ -54,11 +54,15 @@ class PrunedScaleRunner:
         self.last_keep = None
 
     def run_scale(self, x_in, layer_logits, sched: nv.SchedParams, t: int, hbar_scale, append_kv: bool = True,
-                  stream=None, logits_ready=None):
+                  stream=None, logits_ready=None, select_ent=None):
         """x_in [B, N, C] bf16; layer_logits: sequence of L tensors [B, N, V]; hbar_scale: CPU
         float32 [B, t] with the mean entropies of scales 1..t. Returns (x_out, keeps) where keeps
         is the list of per-layer keep-count tensors. `logits_ready`, if given, is a list of
         torch.cuda.Event to wait for before layer j's logits are read (upload overlap).
+        select_ent: optional device f32 [B, N] entropy map of the scale. If given, every layer selects
+        on this one map (the layers' kept sets are then nested: a smaller keep count keeps a subset)
+        and the layers' own logits only provide the means of Eq. 12-13; by default layer j selects
+        on the entropy map of its own logits.
         """
         ctx, B, N = self.ctx, self.B, self.N
         st = stream if stream is not None else torch.cuda.current_stream()
@@ -85,8 +89,8 @@ class PrunedScaleRunner:
                 keep = r["keep"]
                 M = int(keep.sum())
                 keeps.append(keep)
-                nv.nova_select_topk(ctx, self.ent[j], keep, self.keep_idx[:M], self.prune_idx[: B * N - M],
-                                    self.cu_keep, None, stream=st)
+                nv.nova_select_topk(ctx, self.ent[j] if select_ent is None else select_ent, keep, self.keep_idx[:M],
+                                    self.prune_idx[: B * N - M], self.cu_keep, None, stream=st)
                 shape = nv.BlockShape(B, N, self.C, self.n_heads, self.F, self.Lmax, M)
                 if self.modulation is None:
                     nv.nova_pruned_block_forward(ctx, self.weights[j], shape, x, self.keep_idx[:M], self.cu_keep,

@@ -1009,3 +1009,56 @@ def test_runners_with_modulation_agree_and_match_oracle(ctx):
     w_x1, _ = oracle.restore_from_cache(f32(x_in), wy, w_keep, w_prune, w_cu, f32(cache_prev[0]), side, side)
     # the runner's layer-1 output is x_buf[0]; layer 2 wrote x_buf[1]
     assert _rel_err(f32(host.x_buf[0]), w_x1) <= BLOCK_TOL
+
+
+def test_selection_on_one_scale_map_gives_nested_sets(ctx):
+    """The other reading of how layers get their entropy map: one map per scale, selected on by every
+    layer with that layer's keep count. Kept sets of layers with fewer kept tokens are subsets of
+    those with more, index lists equal the oracle's on the same map, and the layers' own logits still
+    drive the keep counts through their means (Eq. 12-13)."""
+    from paper_2602_01345_b200 import pipeline
+    ms = synth.CONFIGS["c2_var_d16_256"]
+    B, L, T = 2, 3, len(ms.scales)
+    side = ms.scales[-1]
+    N, V, C, Lmax = side * side, synth.V_CODEBOOK, ms.C, ms.total_tokens
+    prior = Lmax - N
+    weights = [synth.block_weights(C, ms.F, 100 + j, DEV) for j in range(L)]
+    ks, vs = [], []
+    for j in range(L):
+        k, v, _ = synth.kv_cache(B, Lmax, prior, C, 50 + 2 * j, DEV)
+        ks.append(k)
+        vs.append(v)
+    kv_len = torch.full((L, B), prior, dtype=torch.int32, device=DEV)
+    cache_prev = [synth.residual_cache(B, ms.scales[-2], ms.scales[-2], C, 70 + j, DEV) for j in range(L)]
+    x_in = synth.activations(B, N, C, 7, DEV)
+    a = synth.smooth_temperature_field(B, side, side, 5, a_lo=0.5, a_hi=6.0, device=DEV)
+    beta = [1.0, 0.8, 1.25]
+    logits = [synth.logits_from_temperature(a * beta[j], V, 20 + j) for j in range(L)]
+    scale_ent = torch.empty((B, N), dtype=torch.float32, device=DEV)
+    nova.nova_scale_entropy(ctx, synth.logits_from_temperature(a, V, 19), scale_ent, None)
+    _, hbar = synth.scale_envelope_temperatures(B, T, seed=3)
+    sched = nova.SchedParams(force_act_scale=T - 1)          # Eq. 11-13 decide the ratios
+    runner = pipeline.PrunedScaleRunner(ctx, weights, ms.heads, B, side, side, Lmax, ks, vs, kv_len, cache_prev)
+    kept = []
+    orig = nova.nova_select_topk
+
+    def spy(ctx_, ent, k, keep_idx, prune_idx, cu_keep, pos=None, stream=None):
+        orig(ctx_, ent, k, keep_idx, prune_idx, cu_keep, pos, stream=stream)
+        assert ent.data_ptr() == scale_ent.data_ptr()
+        w_keep, w_prune, w_cu, _ = oracle.select_topk(scale_ent.cpu().numpy(), k.numpy())
+        assert np.array_equal(keep_idx.cpu().numpy(), w_keep) and np.array_equal(cu_keep.cpu().numpy(), w_cu)
+        cu = cu_keep.cpu().numpy()
+        kept.append([set(keep_idx[cu[b]:cu[b + 1]].cpu().tolist()) for b in range(B)])
+
+    pipeline.nv.nova_select_topk = spy
+    try:
+        _, keeps = runner.run_scale(x_in, logits, sched, T, hbar.contiguous(), select_ent=scale_ent)
+    finally:
+        pipeline.nv.nova_select_topk = orig
+    assert ctx.device_status() == 0
+    counts = torch.stack(keeps)
+    assert len({tuple(c.tolist()) for c in counts}) > 1          # the layers' means moved the counts
+    for b in range(B):
+        order = sorted(range(L), key=lambda j: int(counts[j, b]))
+        for lo, hi in zip(order, order[1:]):
+            assert kept[lo][b] <= kept[hi][b]
