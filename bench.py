@@ -30,12 +30,35 @@ import nova_synth as synth  # noqa: E402
 
 METRIC = "pruned_scale_images_per_s"
 UNIT = "images/s"
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the committed ncu captures
-# under profiles/, taken on the default workload's launch shapes (batch 4, 4096 tokens, keep 0.5); None
-# for any other workload, and reset to None whenever the kernel changes after the capture.
-# attention: one launch; gemm: average over the four launches of a layer (qkv, proj, fc1, fc2), the
-# unit `achieved` is taken over as well. Source: profiles/layer_kernels_c4_1024_batch4_keep0.5.txt.
-NCU_TRAFFIC_BYTES = {"attention": 351_413_504, "gemm": 172_203_776}
+NOMINAL_PEAKS = {"hbm": 8000.0, "tensor": 2250.0}      # GB/s, dense bf16 TFLOP/s (context; `peak` is the measured one)
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic_c4_1024_batch4_keep0.5.txt")
+
+
+def source_digest(paths):
+    import hashlib
+    h = hashlib.sha256()
+    for p in paths:
+        with open(os.path.join(ROOT, p), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic():
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the committed ncu capture
+    on the default workload's launch shapes, per kernel key. Each line of the summary file names the
+    sources the kernel is built from and their digest at capture time: a kernel whose sources have
+    changed since reports no traffic (None) until it is captured again."""
+    out = {}
+    try:
+        for line in open(TRAFFIC_FILE):
+            f = line.split()
+            if len(f) < 4 or line.startswith("#"):
+                continue
+            key, nbytes, digest, srcs = f[0], int(f[1]), f[2], f[3].split(",")
+            out[key] = nbytes if source_digest(srcs) == digest else None
+    except (OSError, ValueError):
+        pass
+    return out
 
 
 def parse_args():
@@ -264,10 +287,13 @@ def run_ours(args):
             gemm_n += prof[k][1]
     gemm_tf = sum(gemm_flops.values()) / (gemm_ms / (gemm_n / 4) * 1e-3) / 1e12 if gemm_n else 0.0
 
+    traffic = ncu_traffic() if default_shape else {}
+
     def tensor_roofline(name, achieved, launches_per_layer, traffic_key):
         return {"kernel": name, "bound": "tensor", "achieved": round(achieved, 2), "peak": pk["tensor"],
                 "unit": "TFLOP/s", "frac": round(achieved / pk["tensor"], 4),
-                "traffic": NCU_TRAFFIC_BYTES[traffic_key] if default_shape else None,
+                "frac_of_nominal": round(achieved / NOMINAL_PEAKS["tensor"], 4), "nominal_peak": NOMINAL_PEAKS["tensor"],
+                "traffic": traffic.get(traffic_key),
                 "launches_per_layer": launches_per_layer, "peak_source": pk["source"] + " (bf16 sustained)"}
 
     roof_attn = tensor_roofline("attention_kernel", attn_tf, 1, "attention")
@@ -350,9 +376,13 @@ def run_ours(args):
                            "ms_per_step_host_driven": round(ms_per_step, 4), "launches_per_step": int(dev_launches),
                            "host_syncs_per_step": 0, "equals_host_driven_result": same,
                            "max_abs_diff_vs_host_driven": max_diff}
-    for k in ("entropy_rows", "restore"):
-        if "gbs" in kernels.get(k, {}):
+    for k in kernels:
+        if "gbs" in kernels[k]:
             kernels[k]["frac_of_hbm_peak"] = round(kernels[k]["gbs"] / pk["hbm"], 4)
+            kernels[k]["frac_of_nominal_hbm"] = round(kernels[k]["gbs"] / NOMINAL_PEAKS["hbm"], 4)
+        if "tflops" in kernels[k]:
+            kernels[k]["frac_of_tensor_peak"] = round(kernels[k]["tflops"] / pk["tensor"], 4)
+            kernels[k]["frac_of_nominal_tensor"] = round(kernels[k]["tflops"] / NOMINAL_PEAKS["tensor"], 4)
     kernels["entropy_rows"]["frac_of_hbm_peak_back_to_back"] = round(kernels["entropy_rows"]["gbs_back_to_back"] / pk["hbm"], 4)
 
     out = {
@@ -428,15 +458,26 @@ def run_e2e(args, wd, st, runner, sched, hbar_scale, barrier, dist, dev, world):
 
 
 # ---------------------------------------------------------------------- CPU baseline (oracle)
-def oracle_sample(wd, st, keeps, rows_entropy=1024, rows_block=8):
+def oracle_sample_sizes(threads: int):
+    """Row counts of one oracle sample: enough rows for every OpenMP thread to stay busy (the oracle
+    parallelises over rows only)."""
+    return dict(rows_entropy=max(256, 32 * threads), rows_block=4 * threads)
+
+
+def oracle_sample(wd, st, keeps):
     """Times the oracle, as it stands, on one layer of one image and extrapolates to the whole
     pruned scale: entropy on a row sample, selection on the full map, K/V of every kept token
-    (exact), attention + MLP on a row sample, restore on the full map."""
+    (exact), attention + MLP on a row sample (4 rows per thread, timed as the difference between a
+    call with those rows and a call with none), restore on the full map. Returns (seconds per
+    image-layer, parts, threads, sizes)."""
     import numpy as np
 
     import oracle
     ms, N = wd["ms"], wd["N"]
     f32 = synth.to_f32_numpy
+    threads = oracle.num_threads()
+    sz = oracle_sample_sizes(threads)
+    rows_entropy = min(sz["rows_entropy"], N)
     t = {}
     logits = f32(st["logits"][0][0:1, :rows_entropy])
     t0 = time.perf_counter()
@@ -444,6 +485,7 @@ def oracle_sample(wd, st, keeps, rows_entropy=1024, rows_block=8):
     t["entropy"] = (time.perf_counter() - t0) * (N / rows_entropy)
     ent_full = np.random.default_rng(0).random((1, N)).astype(np.float32)
     k = int(keeps[0][0])
+    rows_block = min(sz["rows_block"], k)
     t0 = time.perf_counter()
     keep_idx, prune_idx, cu, _ = oracle.select_topk(ent_full, [k])
     t["select"] = time.perf_counter() - t0
@@ -451,36 +493,47 @@ def oracle_sample(wd, st, keeps, rows_entropy=1024, rows_block=8):
     x = f32(st["x_in"][0:1])
     kc, vc = f32(st["k_caches"][0][0:1]), f32(st["v_caches"][0][0:1])
     kv_len = np.array([wd["P"]], np.int32)
+    none = np.zeros(0, np.int32)
     # first call untimed: it also pays for the first touch of the converted K/V caches
-    oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=np.zeros(0, np.int32))
+    oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=none)
     t0 = time.perf_counter()
-    oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=np.zeros(0, np.int32))
+    oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=none)
     t["block_kv"] = time.perf_counter() - t0
     rows = np.linspace(0, k - 1, rows_block).astype(np.int32)
     t0 = time.perf_counter()
-    y, _, _ = oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=rows)
+    oracle.pruned_block_forward(wts, 1e-6, ms.heads, x, keep_idx, cu, kc, vc, kv_len, rows=rows)
     t["block_rows"] = max(time.perf_counter() - t0 - t["block_kv"], 0.0) * (k / rows_block)
     y_full = np.zeros((k, ms.C), np.float32)
     t0 = time.perf_counter()
     oracle.restore_from_cache(x, y_full, keep_idx, prune_idx, cu, f32(st["cache_prev"][0][0:1]), wd["h"], wd["w"])
     t["restore"] = time.perf_counter() - t0
-    per_image_layer = sum(t.values())
-    return per_image_layer, t, oracle.num_threads()
+    return sum(t.values()), t, threads, dict(rows_entropy=rows_entropy, rows_block=rows_block, kept=k)
 
 
-def cpu_baseline(wd, st, keeps):
-    per_image_layer, parts, cores = oracle_sample(wd, st, keeps)
+def sample_text(sizes, threads, L):
+    return (f"one layer of one image: entropy on {sizes['rows_entropy']} rows, top-k on the full map, K/V of all "
+            f"{sizes['kept']} kept tokens, attention+MLP on {sizes['rows_block']} kept rows "
+            f"({sizes['rows_block'] // max(threads, 1)} per thread, all {threads} threads busy), restore on the full map; "
+            f"each part scaled to the full row count, then x{L} layers")
+
+
+def cpu_baseline(wd, st, keeps, repeats=3):
+    """The oracle on the host cores: `repeats` samples, the median per part."""
+    runs = [oracle_sample(wd, st, keeps) for _ in range(repeats)]
+    parts = {k: statistics.median(r[1][k] for r in runs) for k in runs[0][1]}
+    totals = sorted(r[0] for r in runs)
+    threads, sizes = runs[0][2], runs[0][3]
     ms = wd["ms"]
-    sec_per_image = per_image_layer * ms.L
-    return {"value": round(1.0 / sec_per_image, 6), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "one layer of one image: entropy on 1024 of the rows, top-k on the full map, K/V of all kept "
-                      "tokens, attention+MLP on 8 kept rows, restore on the full map; each part scaled to the full "
-                      f"row count, then x{ms.L} layers",
-            "seconds_per_image_layer": {k: round(v, 3) for k, v in parts.items()}}
+    sec_per_image = sum(parts.values()) * ms.L
+    return {"value": round(1.0 / sec_per_image, 6), "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": sample_text(sizes, threads, ms.L) + f"; median of {repeats} samples",
+            "seconds_per_image_layer": {k: round(v, 3) for k, v in parts.items()},
+            "spread_seconds_per_image_layer": [round(totals[0], 3), round(totals[-1], 3)]}
 
 
 def run_reference(args):
-    """The oracle as the reference arm: same metric and workload, bounded sample per step."""
+    """The oracle as the reference arm: same metric and workload, bounded sample per step (the same
+    sample, of the same size, as the `cpu_baseline` leg of the other arm)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -491,20 +544,20 @@ def run_reference(args):
     k = wd["N"] - int((1.0 - wd["keep"]) * wd["N"])
     keeps = [torch.tensor([k], dtype=torch.int32)]
     times = []
-    cores = 1
+    threads, sizes = 1, {}
     for i in range(args.warmup + args.steps):
-        per_image_layer, _, cores = oracle_sample(wd_small, st, keeps, rows_entropy=256, rows_block=2)
+        per_image_layer, _, threads, sizes = oracle_sample(wd_small, st, keeps)
         if i >= args.warmup:
             times.append(per_image_layer * ms.L)
-    sec_per_image = sum(times) / len(times)
+    sec_per_image = statistics.median(times)
     value = 1.0 / sec_per_image
-    sample = ("per step: one layer of one image (entropy on 256 rows, full top-k, K/V of all kept tokens, "
-              f"attention+MLP on 2 kept rows, full restore), parts scaled to full row counts, x{ms.L} layers")
+    sample = "per step: " + sample_text(sizes, threads, ms.L) + f"; median of {len(times)} steps"
     out = {"impl": "reference", "metric": METRIC, "value": round(value, 6), "unit": UNIT,
            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
            "ms_per_step": round(sec_per_image * wd["B"] * 1e3, 1), "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config_json(wd, 1),
-           "cpu_baseline": {"value": round(value, 6), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+           "cpu_baseline": {"value": round(value, 6), "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                            "spread_seconds_per_image": [round(min(times), 1), round(max(times), 1)]},
            "e2e": {"value": round(value, 6), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out))
@@ -517,7 +570,7 @@ def build_state_cpu_one_layer(wd):
     k, v, _ = synth.kv_cache(1, wd["Lmax"], wd["P"], ms.C, 0, "cpu")
     return dict(weights=[synth.block_weights(ms.C, ms.F, 0, "cpu")], k_caches=[k], v_caches=[v],
                 cache_prev=[synth.residual_cache(1, wd["hp"], wd["wp"], ms.C, 0, "cpu")],
-                logits=[synth.logits_from_temperature(a[:, :256].contiguous(), synth.V_CODEBOOK, 0)],
+                logits=[synth.logits_from_temperature(a[:, :4096].contiguous(), synth.V_CODEBOOK, 0)],
                 x_in=synth.activations(1, N, ms.C, 5, "cpu"))
 
 

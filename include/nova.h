@@ -27,6 +27,9 @@
  *  - bf16 tensors are row-major with the last dimension contiguous; device pointers to
  *    bf16/f32 tensors must be 16-byte aligned. Index tensors are int32.
  *  - Scales t and layers j are 1-based as in the paper.
+ *  - A context belongs to one CUDA device, which must be the caller's current device at every
+ *    call that enqueues work (else NOVA_ERR_INVALID_ARG; nothing is launched). nova_create and
+ *    nova_destroy leave the caller's current device as they found it.
  *  - Device-side waits are bounded. If one expires the kernel records
  *    NOVA_ERR_TIMEOUT in the context's device status word and returns; non-finite
  *    logits record NOVA_ERR_NONFINITE. nova_device_status() reads that word.
@@ -66,8 +69,9 @@ void        nova_destroy(nova_ctx* ctx);
 const char* nova_last_error(const nova_ctx* ctx);
 const char* nova_status_string(nova_status s);
 
-/* Synchronises `stream`, returns the device status word (NOVA_OK, NOVA_ERR_TIMEOUT or
- * NOVA_ERR_NONFINITE) and clears it. */
+/* Synchronises `stream`, returns the device status word (NOVA_OK, NOVA_ERR_TIMEOUT,
+ * NOVA_ERR_SHAPE for a K/V cache that would overflow, or NOVA_ERR_NONFINITE, in that order of
+ * precedence) and clears it. */
 nova_status nova_device_status(nova_ctx* ctx, void* stream);
 
 /* ---- measurement (no counterpart in the paper) --------------------------------- */
@@ -99,8 +103,8 @@ nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nova_dtype dt,
 
 /* ---- Eq. 4 and Eq. 7 from the hidden states: codebook head fused with the entropy -- */
 /*
- * The paper takes the predicted distributions "already produced during standard decoding"
- * (complexity paragraph after Table 8); a decoder that has the hidden states at hand can skip
+ * The paper's complexity analysis (paragraph after Table 8) assumes that decoding has the
+ * predicted distributions at hand anyway; a decoder that has the hidden states at hand can skip
  * writing the V-wide logits altogether. This call computes, per token,
  *   logits = x W_head^T + b_head (bf16 operands, fp32 accumulation, never rounded or stored),
  *   ent = -sum_v p(v) ln p(v), p = softmax(logits), and mean[s] = (1/N) sum_i ent[s, i].

@@ -61,8 +61,8 @@ void oracle_scale_entropy(const float* logits, int S, int N, int V,
 
 // ---------------------------------------------------------------------------
 // Eq. 4 / Eq. 7 taken one step earlier: the predicted distribution of a token is the
-// softmax of the codebook head applied to its hidden state (the paper takes the
-// distributions "already produced during standard decoding"), so
+// softmax of the codebook head applied to its hidden state (the paper's complexity
+// paragraph after Table 8 counts the distributions as a by-product of decoding), so
 //   logits[v] = sum_c x[c] * w[v, c] + b[v],   p = softmax(logits),   H = -sum p ln p.
 // x [S, N, C], w [V, C] ([out, in] row-major), b [V] or null. The logits are never
 // rounded: double accumulation in index order, entropy as in oracle_scale_entropy.

@@ -41,10 +41,15 @@ nova_status nova_create(nova_ctx** out, int device)
     ctx->launches = 0;
     ctx->profiling = false;
     ctx->events_used = 0;
+    // the allocation is made with `device` current; the caller's current device is put back
+    int prev = -1;
+    const bool have_prev = (cudaGetDevice(&prev) == cudaSuccess);
+    auto restore_device = [&]() { if (have_prev && prev != device) cudaSetDevice(prev); };
     if (cudaSetDevice(device) != cudaSuccess ||
         cudaMalloc(&ctx->dev_status, NOVA_STATUS_BYTES) != cudaSuccess ||
         cudaMemset(ctx->dev_status, 0, NOVA_STATUS_BYTES) != cudaSuccess) {
         delete ctx;
+        restore_device();
         return NOVA_ERR_CUDA;
     }
     cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device);
@@ -54,9 +59,11 @@ nova_status nova_create(nova_ctx** out, int device)
         qres != cudaDriverEntryPointSuccess || !fn) {
         cudaFree(ctx->dev_status);
         delete ctx;
+        restore_device();
         return NOVA_ERR_CUDA;
     }
     ctx->encode_tiled = fn;
+    restore_device();
     *out = ctx;
     return NOVA_OK;
 }
@@ -64,9 +71,12 @@ nova_status nova_create(nova_ctx** out, int device)
 void nova_destroy(nova_ctx* ctx)
 {
     if (!ctx) return;
+    int prev = -1;
+    const bool have_prev = (cudaGetDevice(&prev) == cudaSuccess);
     cudaSetDevice(ctx->device);
     for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
     cudaFree(ctx->dev_status);
+    if (have_prev && prev != ctx->device) cudaSetDevice(prev);
     delete ctx;
 }
 
@@ -113,6 +123,7 @@ const char* nova_last_error(const nova_ctx* ctx) { return ctx ? ctx->err : "null
 nova_status nova_device_status(nova_ctx* ctx, void* stream)
 {
     if (!ctx) return NOVA_ERR_INVALID_ARG;
+    NOVA_DEVICE_GUARD(ctx, "nova_device_status");
     cudaStream_t st = (cudaStream_t)stream;
     unsigned int word = 0;
     NOVA_CUDA_CHECK(ctx, cudaMemcpyAsync(&word, ctx->dev_status, sizeof(word), cudaMemcpyDeviceToHost, st));
@@ -253,6 +264,7 @@ nova_status nova_keep_ratios_device(nova_ctx* ctx, const nova_sched_params* p, i
     if (!hbar_scale || !keep) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_keep_ratios_device: null pointer");
     if (j >= 2 && !hbar_layer && p->force_keep_ratio < 0.0)
         return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_keep_ratios_device: layer history missing");
+    NOVA_DEVICE_GUARD(ctx, "nova_keep_ratios_device");
     cudaStream_t st = (cudaStream_t)stream;
     {
         nova_launch_scope scope(ctx, NOVA_K_KEEP_RATIOS, st);

@@ -257,6 +257,7 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
     Workspace ws = carve(ctx->workspace, s->M, s->C, s->F);
     if (!ctx->workspace || ctx->workspace_bytes < ws.bytes)
         return nova_fail(ctx, NOVA_ERR_WORKSPACE, "nova_pruned_block_forward: workspace missing or too small");
+    NOVA_DEVICE_GUARD(ctx, "nova_pruned_block_forward");
 
     cudaStream_t st = (cudaStream_t)stream;
     const int M = s->M, C = s->C, F = s->F;
@@ -381,8 +382,9 @@ extern "C" nova_status nova_pruned_block_forward_static(nova_ctx* ctx, const nov
     if (ctx->profiling)
         return nova_fail(ctx, NOVA_ERR_INVALID_ARG,
                          "nova_pruned_block_forward_static: not available inside a profiling window (event creation may allocate)");
+    if (!shape_ok(s)) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_pruned_block_forward_static: unsupported shape");
+    if (s->M == 0) return NOVA_OK;      // nothing kept: a no-op, as for the ordinary entry point
     const size_t need = nova_block_workspace_bytes(s);
-    if (need == 0) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_pruned_block_forward_static: unsupported shape");
     if (need > NOVA_STATIC_SCRATCH_BYTES) {
         snprintf(ctx->err, sizeof(ctx->err),
                  "nova_pruned_block_forward_static: shape needs %zu bytes of scratch, the built-in array holds %u",

@@ -107,6 +107,27 @@ static inline nova_status nova_cuda_fail(nova_ctx* ctx, cudaError_t e, const cha
 
 static inline bool nova_aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
 
+// Every launching entry point runs on the caller's current device with pointers (status word,
+// workspace) that live on the context's device: refuse the call when the two differ instead of
+// letting a kernel dereference another GPU's memory.
+static inline nova_status nova_check_device(nova_ctx* ctx, const char* who)
+{
+    int cur = -1;
+    const cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return nova_cuda_fail(ctx, e, "cudaGetDevice");
+    if (cur != ctx->device) {
+        snprintf(ctx->err, sizeof(ctx->err), "%s: the context belongs to device %d but device %d is current",
+                 who, ctx->device, cur);
+        return NOVA_ERR_INVALID_ARG;
+    }
+    return NOVA_OK;
+}
+#define NOVA_DEVICE_GUARD(ctx, who)                                           \
+    do {                                                                      \
+        const nova_status g__ = nova_check_device((ctx), (who));              \
+        if (g__ != NOVA_OK) return g__;                                       \
+    } while (0)
+
 // Kernel launchers implemented in the other translation units.
 
 enum nova_epilogue {

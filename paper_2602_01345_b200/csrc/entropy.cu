@@ -458,6 +458,7 @@ extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nov
     const int per = (dt == NOVA_BF16) ? 8 : 4;
     if (row_stride < V || (row_stride % per) != 0 || !nova_aligned16(logits))
         return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_scale_entropy: logits rows must start on 16-byte boundaries");
+    NOVA_DEVICE_GUARD(ctx, "nova_scale_entropy");
     cudaStream_t st = (cudaStream_t)stream;
     const int elt = (dt == NOVA_BF16) ? 2 : 4;
     const long row_bytes = (long)V * elt;
@@ -502,6 +503,7 @@ extern "C" nova_status nova_head_entropy(nova_ctx* ctx, const void* x, const voi
     if (C % 64 || V % 32) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_head_entropy: C must be a multiple of 64 and V of 32");
     if (!nova_aligned16(x) || !nova_aligned16(w_head) || !nova_aligned16(b_head))
         return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_head_entropy: tensors must be 16-byte aligned");
+    NOVA_DEVICE_GUARD(ctx, "nova_head_entropy");
     cudaStream_t st = (cudaStream_t)stream;
     nova_gemm_args g;
     memset(&g, 0, sizeof(g));

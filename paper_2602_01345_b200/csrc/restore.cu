@@ -148,6 +148,7 @@ static nova_status restore(nova_ctx* ctx, const void* x_in, const void* y_kept,
     if (!nova_aligned16(x_in) || !nova_aligned16(x_out) || !nova_aligned16(y_kept) ||
         !nova_aligned16(cache_prev) || !nova_aligned16(cache_out))
         return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_restore_from_cache: tensors must be 16-byte aligned");
+    NOVA_DEVICE_GUARD(ctx, "nova_restore_from_cache");
     const unsigned blocks = (unsigned)((total + kWarpsPerBlock - 1) / kWarpsPerBlock);
     nova_launch_scope scope(ctx, NOVA_K_RESTORE, (cudaStream_t)stream);
     restore_kernel<<<blocks, kWarpsPerBlock * 32, 0, (cudaStream_t)stream>>>(
@@ -173,6 +174,7 @@ extern "C" nova_status nova_restore_from_cache_device(nova_ctx* ctx, const void*
                                                       int hp, int wp, int h, int w, int C, int B,
                                                       void* x_out, void* cache_out, void* stream)
 {
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
     const long total = (long)B * h * w;
     if (total > 0x7fffffffL) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_restore_from_cache_device: too many rows");
     return restore(ctx, x_in, y_kept, keep_idx, prune_idx, cu_keep, cache_prev, hp, wp, h, w, C, B, (int)total, true,

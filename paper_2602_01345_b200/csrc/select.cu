@@ -171,6 +171,7 @@ extern "C" nova_status nova_select_topk(nova_ctx* ctx, const float* ent, int S, 
     if (S < 0 || N < 0) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_select_topk: negative size");
     if (N > 16384) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_select_topk: N > 16384");
     if (!cu_keep) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_select_topk: null cu_keep");
+    NOVA_DEVICE_GUARD(ctx, "nova_select_topk");
     cudaStream_t st = (cudaStream_t)stream;
     if (S == 0 || N == 0) {
         NOVA_CUDA_CHECK(ctx, cudaMemsetAsync(cu_keep, 0, sizeof(int32_t) * (size_t)(S + 1), st));
@@ -216,6 +217,7 @@ extern "C" nova_status nova_select_topk_device(nova_ctx* ctx, const float* ent, 
     if (N > 16384) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_select_topk_device: N > 16384");
     if (S > 65535) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_select_topk_device: S > 65535");
     if (!cu_keep) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_select_topk_device: null cu_keep");
+    NOVA_DEVICE_GUARD(ctx, "nova_select_topk_device");
     cudaStream_t st = (cudaStream_t)stream;
     if (S == 0 || N == 0) {
         NOVA_CUDA_CHECK(ctx, cudaMemsetAsync(cu_keep, 0, sizeof(int32_t) * (size_t)(S + 1), st));
