@@ -72,6 +72,9 @@ def parse_args():
     ap.add_argument("--keep", type=float, default=0.5)
     ap.add_argument("--scale", type=int, default=None, help="1-based scale index (default: last)")
     ap.add_argument("--layers", type=int, default=None, help="override the number of layers (small profiling cases)")
+    ap.add_argument("--two-call-layers", action="store_true",
+                    help="time nova_pruned_block_forward + nova_restore_from_cache per layer instead of the one "
+                         "nova_pruned_layer_forward call (the other form is timed after the timed region either way)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-next", action="store_true",
@@ -222,8 +225,10 @@ def run_ours(args):
 
     ctx = nova.Context(local)
     st = build_state(wd, dev)
+    fused = not args.two_call_layers
     runner = pipeline.PrunedScaleRunner(ctx, st["weights"], ms.heads, B, wd["h"], wd["w"], wd["Lmax"],
-                                        st["k_caches"], st["v_caches"], st["kv_len"], st["cache_prev"])
+                                        st["k_caches"], st["v_caches"], st["kv_len"], st["cache_prev"],
+                                        fused_restore=fused)
     sched = nova.SchedParams(force_act_scale=wd["t"], force_keep_ratio=wd["keep"])
     hbar_scale = torch.linspace(2.0, 7.0, wd["t"]).repeat(B, 1).contiguous()
     stream = torch.cuda.current_stream()
@@ -301,29 +306,53 @@ def run_ours(args):
     roofline = roof_attn if attn_ms >= gemm_ms else roof_gemm
     other_roofline = roof_gemm if attn_ms >= gemm_ms else roof_attn
     rows = B * N
-    ent_bytes = rows * (synth.V_CODEBOOK * 2 + 4)
-    if prof["entropy_rows"][1]:
-        kernels["entropy_rows"]["gbs"] = round(ent_bytes / (prof["entropy_rows"][0] / prof["entropy_rows"][1] * 1e-3) / 1e9, 1)
-    restore_bytes = (M * 4 + (rows - M) * 3) * ms.C * 2 + B * wd["hp"] * wd["wp"] * ms.C * 2
-    if prof["restore"][1]:
-        kernels["restore"]["gbs"] = round(restore_bytes / (prof["restore"][0] / prof["restore"][1] * 1e-3) / 1e9, 1)
-    # The per-launch events above put a launch latency of several microseconds inside the bracket of
-    # every kernel, which is a large part of a 30 microsecond kernel. The HBM-bound entropy pass is
-    # therefore also timed as it runs in a stream: the L layers' logits (each larger than L2) back
-    # to back between one pair of events, outside the timed region.
-    ent_buf = torch.empty((B, N), dtype=torch.float32, device=dev)
-    mean_buf = torch.empty((B,), dtype=torch.float32, device=dev)
+    # HBM-bound passes: algorithmic bytes of all launches of a step over their summed event time.
+    # entropy: per token V * 2 bytes read + 4 written; select: per token a 4-byte key read and a 4-byte
+    # index written; restore: kept row = y and x_in read, x_out and cache_out written (4 rows; when the
+    # block's last GEMM writes the kept rows itself, restore touches the pruned rows only), pruned row =
+    # x_in read, x_out and cache_out written (3 rows), plus the low-resolution cache once.
+    ent_bytes_step = ms.L * rows * (synth.V_CODEBOOK * 2 + 4)
+    sel_bytes_step = ms.L * rows * 8
+    kept_rows_in_restore = 0 if fused else M
+    restore_bytes = (kept_rows_in_restore * 4 + (rows - M) * 3) * ms.C * 2 + B * wd["hp"] * wd["wp"] * ms.C * 2
+    for key, step_bytes in (("entropy_rows", ent_bytes_step), ("select_topk", sel_bytes_step),
+                            ("restore", restore_bytes * ms.L)):
+        if prof.get(key, (0, 0))[1]:
+            kernels[key]["gbs"] = round(step_bytes * args.steps / (prof[key][0] * 1e-3) / 1e9, 1)
+            kernels[key]["bytes_per_launch"] = int(step_bytes * args.steps / prof[key][1])
+    # The entropy pass once more outside the timed region, back to back between one pair of events,
+    # with and without the per-image means.
+    ent_buf = torch.empty((ms.L, B, N), dtype=torch.float32, device=dev)
+    mean_buf = torch.empty((ms.L, B), dtype=torch.float32, device=dev)
     b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for with_mean in (True, False):
         torch.cuda.synchronize()
         b0.record(stream)
-        for lg in st["logits"]:
-            nova.nova_scale_entropy(ctx, lg, ent_buf, mean_buf if with_mean else None, stream=stream)
+        for _ in range(3):
+            nova.nova_scale_entropy_layers(ctx, st["logits"], ent_buf, mean_buf if with_mean else None, stream=stream)
         b1.record(stream)
         torch.cuda.synchronize()
-        us = b0.elapsed_time(b1) * 1e3 / len(st["logits"])
+        us = b0.elapsed_time(b1) * 1e3 / 3
         key = "gbs_back_to_back" if with_mean else "gbs_back_to_back_no_mean"
-        kernels["entropy_rows"][key] = round(ent_bytes / us / 1e3, 1)
+        kernels["entropy_rows"][key] = round(ent_bytes_step / us / 1e3, 1)
+    # the layers in the other form (two calls per layer, or one), same inputs, for the comparison
+    other = pipeline.PrunedScaleRunner(ctx, st["weights"], ms.heads, B, wd["h"], wd["w"], wd["Lmax"], st["k_caches"],
+                                       st["v_caches"], st["kv_len"], st["cache_prev"], fused_restore=not fused)
+    for it in range(2 + args.steps):
+        if it == 2:
+            torch.cuda.synchronize()
+            b0.record(stream)
+        st["kv_len"].copy_(st["kv_len0"])
+        x_other, _ = other.run_scale(st["x_in"], st["logits"], sched, wd["t"], hbar_scale, stream=stream)
+    b1.record(stream)
+    torch.cuda.synchronize()
+    other_ms = b0.elapsed_time(b1) / args.steps
+    layer_forms = {"timed": "one call per layer (nova_pruned_layer_forward)" if fused else
+                            "two calls per layer (nova_pruned_block_forward + nova_restore_from_cache)",
+                   "ms_per_step_one_call": round(ms_per_step if fused else other_ms, 4),
+                   "ms_per_step_two_calls": round(other_ms if fused else ms_per_step, 4),
+                   "same_result": bool(torch.equal(x_other, x_out))}
+    del other
     head_entropy = device_schedule = None
     if not args.no_next:
         # Entropy fused with the codebook head (the step before the path: hidden states -> entropy, the
@@ -350,7 +379,8 @@ def run_ours(args):
         hist_dev = hbar_scale.t().contiguous().to(dev)
         drun = pipeline.DeviceScaleRunner(ctx, st["weights"], ms.heads, B, wd["h"], wd["w"], wd["Lmax"], st["k_caches"],
                                           st["v_caches"], st["kv_len"], st["cache_prev"], sched, wd["t"], hist_dev,
-                                          synth.V_CODEBOOK, x_in=st["x_in"], layer_logits=st["logits"], scale_entropy=False)
+                                          synth.V_CODEBOOK, x_in=st["x_in"], layer_logits=st["logits"], scale_entropy=False,
+                                          fused_restore=fused)
         st["kv_len"].copy_(st["kv_len0"])
         l0 = pipeline.launch_count(ctx)
         drun.capture()
@@ -392,6 +422,7 @@ def run_ours(args):
         "config": config_json(wd, world), "clocks": clk, "gpu_launches": int(launches),
         "tokens_per_s": round(world * B * N / (ms_per_step / 1e3), 1),
         "roofline": roofline, "roofline_second": other_roofline, "kernels": kernels,
+        "layer_call_forms": layer_forms,
         "next_head_entropy": head_entropy, "next_device_schedule": device_schedule,
     }
 

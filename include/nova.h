@@ -101,6 +101,19 @@ nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nova_dtype dt,
                                int S, int N, int V, int64_t row_stride,
                                float* ent, float* mean, void* stream);
 
+/*
+ * The entropy maps of all layers of a scale in one call. The layers' logits are inputs of the scale
+ * (Eq. 12 takes one mean per layer), so nothing orders them behind the layers themselves: one launch
+ * streams the rows of all layers, which keeps HBM busy instead of ramping up and draining per layer.
+ * logits: HOST array of n_layers device pointers, each a [S, N, V] tensor as for nova_scale_entropy
+ *         (same dt, V and row_stride for all). n_layers * S <= 256 for the one-launch path.
+ * ent:    device f32 [n_layers, S, N].   mean: device f32 [n_layers, S] or NULL.
+ * Results and errors are those of n_layers calls of nova_scale_entropy.
+ */
+nova_status nova_scale_entropy_layers(nova_ctx* ctx, const void* const* logits, int n_layers, nova_dtype dt,
+                                      int S, int N, int V, int64_t row_stride,
+                                      float* ent, float* mean, void* stream);
+
 /* ---- Eq. 4 and Eq. 7 from the hidden states: codebook head fused with the entropy -- */
 /*
  * The paper's complexity analysis (paragraph after Table 8) assumes that decoding has the
@@ -152,6 +165,17 @@ nova_status nova_keep_ratios(const nova_sched_params* p, int B, int t, int j, in
                              int32_t* t_star, int32_t* act_scale,
                              double* ratio_scale, double* ratio_layer, int32_t* keep);
 
+/*
+ * Eq. 8-13 for all L layers of scale t at once (host arithmetic, double), given the L layer means
+ * of the scale: layer j's ratio uses the means of layers 1..j exactly as nova_keep_ratios(.., j, ..).
+ * hbar_scale host [B, t]; hbar_layer host [B, L]; t_star, act_scale host int32 [B]; ratio_scale
+ * host double [B]; ratio_layer host double [L, B]; keep host int32 [L, B]. Errors as nova_keep_ratios.
+ */
+nova_status nova_keep_ratios_layers(const nova_sched_params* p, int B, int t, int L, int N_t,
+                                    const float* hbar_scale, const float* hbar_layer,
+                                    int32_t* t_star, int32_t* act_scale,
+                                    double* ratio_scale, double* ratio_layer, int32_t* keep);
+
 /* ---- keep the highest-entropy tokens ------------------------------------------- */
 /*
  * ent:  device f32 [S, N] (finite).   k: HOST int32 [S], 0 <= k[s] <= N.
@@ -166,6 +190,22 @@ nova_status nova_keep_ratios(const nova_sched_params* p, int B, int t, int j, in
 nova_status nova_select_topk(nova_ctx* ctx, const float* ent, int S, int N, const int32_t* k,
                              int32_t* keep_idx, int32_t* prune_idx, int32_t* cu_keep,
                              int32_t* pos, void* stream);
+
+/*
+ * The selection of all layers of a scale in one launch (the pruning sentence after Eq. 13 applies
+ * per layer with that layer's ratio): G lists (layers) of S segments (images) each. List g is what
+ * nova_select_topk(ent + g*S*N, S, N, k + g*S, ...) gives, written to
+ *   keep_idx + g*S*N, prune_idx + g*S*N (each list has room for S*N entries), cu_keep + g*(S+1),
+ *   pos + g*S*N (or pos == NULL).
+ * k: HOST int32 [G, S]. S <= 256. Errors as nova_select_topk. The _device form takes k from device
+ * memory (clamped to [0, N]) as nova_select_topk_device does.
+ */
+nova_status nova_select_topk_grouped(nova_ctx* ctx, const float* ent, int G, int S, int N, const int32_t* k,
+                                     int32_t* keep_idx, int32_t* prune_idx, int32_t* cu_keep,
+                                     int32_t* pos, void* stream);
+nova_status nova_select_topk_grouped_device(nova_ctx* ctx, const float* ent, int G, int S, int N,
+                                            const int32_t* k_dev, int32_t* keep_idx, int32_t* prune_idx,
+                                            int32_t* cu_keep, int32_t* pos, void* stream);
 
 /* ---- Eq. 14: the layer on the kept tokens -------------------------------------- */
 typedef struct nova_block_weights {  /* device bf16; matrices are [out, in] row-major */
@@ -295,6 +335,24 @@ nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, const void*
                                     int hp, int wp, int h, int w, int C, int B, int M,
                                     void* x_out, void* cache_out, void* stream);
 
+/* ---- Eq. 14 and Eq. 15-16 of one layer in one call ------------------------------------------ */
+/*
+ * nova_pruned_block_forward[_adaln] followed by nova_restore_from_cache, without the compacted
+ * y_kept in between: the block's last GEMM writes each kept row straight to its place in x_out
+ * (Eq. 16, kept rows) and its difference to the layer input to cache_out (Eq. 15), and the restore
+ * pass then touches the pruned rows only. x_out and cache_out are bit-identical to the two calls.
+ * Arguments as for those calls (mod may be NULL; cache_out may be NULL; the token map is h rows by
+ * w_tokens columns, h * w_tokens == s->N;
+ * m_on_device != 0: s->M is an upper bound and the kept count is cu_keep[B] on the device, and
+ * cache_prev is then always required). Errors as for the two calls.
+ */
+nova_status nova_pruned_layer_forward(nova_ctx* ctx, const nova_block_weights* w,
+                                      const nova_block_modulation* mod, const nova_block_shape* s,
+                                      const void* x_in, const int32_t* keep_idx, const int32_t* prune_idx,
+                                      const int32_t* cu_keep, void* k_cache, void* v_cache, int32_t* kv_len,
+                                      int append_kv, const void* cache_prev, int hp, int wp, int h, int w_tokens,
+                                      void* x_out, void* cache_out, int m_on_device, void* stream);
+
 /* ---- the same steps driven from the device: no host value between the calls of a layer ----- */
 /*
  * (The paper fixes what is computed, not where the keep counts live; these calls exist so that a
@@ -323,6 +381,11 @@ nova_status nova_restore_from_cache(nova_ctx* ctx, const void* x_in, const void*
 nova_status nova_keep_ratios_device(nova_ctx* ctx, const nova_sched_params* p, int B, int t, int j, int N_t,
                                     const float* hbar_scale, const float* hbar_layer,
                                     int32_t* t_star, int32_t* act_scale, int32_t* keep, void* stream);
+/* All L layers of scale t in one launch: hbar_layer device f32 [L, B] (all layers' means), keep device
+ * int32 [L, B]; row j equals what nova_keep_ratios_device(.., j + 1, ..) writes. */
+nova_status nova_keep_ratios_layers_device(nova_ctx* ctx, const nova_sched_params* p, int B, int t, int L, int N_t,
+                                           const float* hbar_scale, const float* hbar_layer,
+                                           int32_t* t_star, int32_t* act_scale, int32_t* keep, void* stream);
 nova_status nova_select_topk_device(nova_ctx* ctx, const float* ent, int S, int N, const int32_t* k_dev,
                                     int32_t* keep_idx, int32_t* prune_idx, int32_t* cu_keep,
                                     int32_t* pos, void* stream);

@@ -210,6 +210,27 @@ def nova_scale_entropy(ctx: Context, logits, ent, mean=None, stream=None):
                                       logits.stride(1), _ptr(ent), _ptr(mean), _stream(stream)))
 
 
+_lib.nova_scale_entropy_layers.argtypes = [_vp, C.POINTER(_vp), _i, _i, _i, _i, _i, _i64, _vp, _vp, _vp]
+_lib.nova_scale_entropy_layers.restype = _i
+
+
+def nova_scale_entropy_layers(ctx: Context, layer_logits, ent, mean=None, stream=None):
+    """The entropy maps of several layers in one call: layer_logits is a sequence of L tensors
+    [S, N, V] (same dtype, shape and row stride) -> ent [L, S, N] f32, mean [L, S] f32."""
+    L = len(layer_logits)
+    S, N, V = layer_logits[0].shape
+    dt = {torch.bfloat16: NOVA_BF16, torch.float32: NOVA_F32}[layer_logits[0].dtype]
+    stride = layer_logits[0].stride(1)
+    for t in layer_logits:
+        assert t.shape == (S, N, V) and t.dtype == layer_logits[0].dtype
+        assert t.stride(2) == 1 and t.stride(1) == stride and t.stride(0) == N * stride
+    assert ent.dtype == torch.float32 and ent.is_contiguous() and ent.numel() == L * S * N
+    assert mean is None or (mean.dtype == torch.float32 and mean.is_contiguous() and mean.numel() == L * S)
+    table = (_vp * L)(*[t.data_ptr() if t.numel() else None for t in layer_logits])
+    ctx.check(_lib.nova_scale_entropy_layers(ctx.handle, table, L, dt, S, N, V, stride, _ptr(ent), _ptr(mean),
+                                             _stream(stream)))
+
+
 _lib.nova_head_entropy.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]
 _lib.nova_head_entropy.restype = _i
 
@@ -248,6 +269,55 @@ def nova_keep_ratios(p: SchedParams, t: int, j: int, N_t: int, hbar_scale, hbar_
     if st != 0:
         raise NovaError(st, "nova_keep_ratios")
     return out
+
+
+_lib.nova_keep_ratios_layers.argtypes = _lib.nova_keep_ratios.argtypes
+_lib.nova_keep_ratios_layers.restype = _i
+
+
+def nova_keep_ratios_layers(p: SchedParams, t: int, N_t: int, hbar_scale, hbar_layer):
+    """Eq. 8-13 for all layers of scale t. hbar_scale CPU f32 [B, t]; hbar_layer CPU f32 [B, L] (the
+    means of all L layers). Returns dict: t_star, act_scale int32 [B]; ratio_scale f64 [B];
+    ratio_layer f64 [L, B]; keep int32 [L, B]."""
+    hs = hbar_scale.to("cpu", torch.float32).contiguous()
+    hl = hbar_layer.to("cpu", torch.float32).contiguous()
+    B, L = hl.shape
+    assert hs.shape == (B, t)
+    out = dict(t_star=torch.zeros(B, dtype=torch.int32), act_scale=torch.zeros(B, dtype=torch.int32),
+               ratio_scale=torch.zeros(B, dtype=torch.float64), ratio_layer=torch.zeros((L, B), dtype=torch.float64),
+               keep=torch.zeros((L, B), dtype=torch.int32))
+    c = p._c()
+    st = _lib.nova_keep_ratios_layers(C.byref(c), B, t, L, N_t, _ptr(hs), _ptr(hl), _ptr(out["t_star"]),
+                                      _ptr(out["act_scale"]), _ptr(out["ratio_scale"]), _ptr(out["ratio_layer"]),
+                                      _ptr(out["keep"]))
+    if st != 0:
+        raise NovaError(st, "nova_keep_ratios_layers")
+    return out
+
+
+_lib.nova_select_topk_grouped.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.nova_select_topk_grouped.restype = _i
+_lib.nova_select_topk_grouped_device.argtypes = _lib.nova_select_topk_grouped.argtypes
+_lib.nova_select_topk_grouped_device.restype = _i
+
+
+def nova_select_topk_grouped(ctx: Context, ent, k, keep_idx, prune_idx, cu_keep, pos=None, stream=None):
+    """Selection for G lists (layers) of S segments each in one launch. ent [G, S, N] f32 device;
+    k: int32 [G, S], a CPU tensor (host counts) or a device tensor (counts left on the device);
+    keep_idx, prune_idx device int32 [G, S*N]; cu_keep device int32 [G, S+1]; pos [G, S, N] or None."""
+    G, S, N = ent.shape
+    assert ent.dtype == torch.float32 and ent.is_contiguous()
+    assert keep_idx.is_contiguous() and prune_idx.is_contiguous() and cu_keep.is_contiguous()
+    assert keep_idx.numel() >= G * S * N and prune_idx.numel() >= G * S * N and cu_keep.numel() >= G * (S + 1)
+    if k.is_cuda:
+        assert k.dtype == torch.int32 and k.numel() == G * S and k.is_contiguous()
+        ctx.check(_lib.nova_select_topk_grouped_device(ctx.handle, _ptr(ent), G, S, N, _ptr(k), _ptr(keep_idx),
+                                                       _ptr(prune_idx), _ptr(cu_keep), _ptr(pos), _stream(stream)))
+        return
+    kk = k.to("cpu", torch.int32).contiguous()
+    assert kk.numel() == G * S
+    ctx.check(_lib.nova_select_topk_grouped(ctx.handle, _ptr(ent), G, S, N, _ptr(kk), _ptr(keep_idx), _ptr(prune_idx),
+                                            _ptr(cu_keep), _ptr(pos), _stream(stream)))
 
 
 def nova_select_topk(ctx: Context, ent, k, keep_idx, prune_idx, cu_keep, pos=None, stream=None):
@@ -329,6 +399,24 @@ def nova_keep_ratios_device(ctx: Context, p: SchedParams, t: int, j: int, N_t: i
                                            _ptr(t_star), _ptr(act_scale), _ptr(keep), _stream(stream)))
 
 
+_lib.nova_keep_ratios_layers_device.argtypes = _lib.nova_keep_ratios_device.argtypes
+_lib.nova_keep_ratios_layers_device.restype = _i
+
+
+def nova_keep_ratios_layers_device(ctx: Context, p: SchedParams, t: int, N_t: int, hbar_scale, hbar_layer, keep,
+                                   t_star=None, act_scale=None, stream=None):
+    """Eq. 8-13 for all L layers on the device. hbar_scale device f32 [t, B]; hbar_layer device f32
+    [L, B]; keep device int32 [L, B]."""
+    L, B = keep.shape
+    assert hbar_scale.dtype == torch.float32 and hbar_scale.shape == (t, B)
+    assert hbar_layer.dtype == torch.float32 and hbar_layer.shape == (L, B) and hbar_layer.is_contiguous()
+    assert keep.dtype == torch.int32 and keep.is_contiguous()
+    c = p._c()
+    ctx.check(_lib.nova_keep_ratios_layers_device(ctx.handle, C.byref(c), B, t, L, N_t, _ptr(hbar_scale),
+                                                  _ptr(hbar_layer), _ptr(t_star), _ptr(act_scale), _ptr(keep),
+                                                  _stream(stream)))
+
+
 def nova_select_topk_device(ctx: Context, ent, k_dev, keep_idx, prune_idx, cu_keep, pos=None, stream=None):
     """nova_select_topk with the keep counts in a device int32 tensor [S]; keep_idx and prune_idx
     must each have room for S*N entries."""
@@ -390,3 +478,32 @@ def nova_pruned_block_forward_adaln(ctx: Context, w: BlockWeights, modulation: d
     ctx.check(_lib.nova_pruned_block_forward_adaln(
         ctx.handle, C.byref(w.c), C.byref(cm), C.byref(c), _ptr(x_in), _ptr(keep_idx), _ptr(cu_keep), _ptr(k_cache),
         _ptr(v_cache), _ptr(kv_len), int(bool(append_kv)), _ptr(y_kept), int(bool(m_on_device)), _stream(stream)))
+
+
+# ---- Eq. 14 + Eq. 15-16 of one layer in one call ---------------------------------------------------
+_lib.nova_pruned_layer_forward.argtypes = [_vp, C.POINTER(_BlockWeights), C.POINTER(_BlockModulation),
+                                           C.POINTER(_BlockShape), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp,
+                                           _i, _i, _i, _i, _vp, _vp, _i, _vp]
+_lib.nova_pruned_layer_forward.restype = _i
+
+
+def nova_pruned_layer_forward(ctx: Context, w: BlockWeights, modulation, shape: BlockShape, x_in, keep_idx, prune_idx,
+                              cu_keep, k_cache, v_cache, kv_len, append_kv, cache_prev, h, w_tokens, x_out,
+                              cache_out=None, m_on_device: bool = False, stream=None):
+    """The block on the kept rows and the restore of the pruned rows in one call: the block's last GEMM
+    writes the kept rows of x_out / cache_out directly (no compacted y_kept); results are bit-identical
+    to nova_pruned_block_forward[_adaln] followed by nova_restore_from_cache."""
+    ptrs = []
+    for n in MODULATION_NAMES:
+        t = modulation.get(n) if modulation else None
+        if t is not None:
+            assert t.dtype == torch.bfloat16 and t.shape == (shape.B, shape.C)
+        ptrs.append(_ptr(t))
+    cm = _BlockModulation(*ptrs)
+    c = shape._c()
+    assert x_in.shape == (shape.B, shape.N, shape.C) and h * w_tokens == shape.N
+    hp, wp = (cache_prev.shape[1], cache_prev.shape[2]) if cache_prev is not None else (0, 0)
+    ctx.check(_lib.nova_pruned_layer_forward(
+        ctx.handle, C.byref(w.c), C.byref(cm) if modulation else None, C.byref(c), _ptr(x_in), _ptr(keep_idx),
+        _ptr(prune_idx), _ptr(cu_keep), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len), int(bool(append_kv)),
+        _ptr(cache_prev), hp, wp, h, w_tokens, _ptr(x_out), _ptr(cache_out), int(bool(m_on_device)), _stream(stream)))

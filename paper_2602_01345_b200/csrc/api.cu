@@ -237,6 +237,62 @@ __global__ void keep_ratios_kernel(const nova_sched_params p, int B, int t, int 
     keep[b] = kp;
 }
 
+// All L layers of a scale at once; thread (j, b) evaluates layer j + 1 of image b on the means of
+// layers 1..j+1 (every layer's mean is known once the scale's entropy maps are taken).
+__global__ void keep_ratios_layers_kernel(const nova_sched_params p, int B, int t, int L, int n_tokens,
+                                          const float* __restrict__ hs, const float* __restrict__ hl,
+                                          int32_t* __restrict__ t_star, int32_t* __restrict__ act_scale,
+                                          int32_t* __restrict__ keep)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= L * B) return;
+    const int j = i / B, b = i - j * B;
+    int32_t ts, as, kp;
+    double rs, rl;
+    schedule_one(p, t, j + 1, n_tokens, hs + b, B, hl + b, B, &ts, &as, &rs, &rl, &kp);
+    if (j == 0) {
+        if (t_star) t_star[b] = ts;
+        if (act_scale) act_scale[b] = as;
+    }
+    keep[i] = kp;
+}
+
+nova_status nova_keep_ratios_layers(const nova_sched_params* p, int B, int t, int L, int N_t,
+                                    const float* hbar_scale, const float* hbar_layer,
+                                    int32_t* t_star, int32_t* act_scale,
+                                    double* ratio_scale, double* ratio_layer, int32_t* keep)
+{
+    if (!p || B < 0 || t < 1 || L < 1 || N_t < 1 || p->t_est < 2 || !(p->tau > 0.0)) return NOVA_ERR_INVALID_ARG;
+    if (B == 0) return NOVA_OK;
+    if (!hbar_scale || !hbar_layer || !t_star || !act_scale || !ratio_scale || !ratio_layer || !keep) return NOVA_ERR_INVALID_ARG;
+    for (int j = 0; j < L; ++j)
+        for (int b = 0; b < B; ++b)
+            schedule_one(*p, t, j + 1, N_t, hbar_scale + (size_t)b * t, 1, hbar_layer + (size_t)b * L, 1,
+                         t_star + b, act_scale + b, ratio_scale + b, ratio_layer + (size_t)j * B + b, keep + (size_t)j * B + b);
+    return NOVA_OK;
+}
+
+nova_status nova_keep_ratios_layers_device(nova_ctx* ctx, const nova_sched_params* p, int B, int t, int L, int N_t,
+                                           const float* hbar_scale, const float* hbar_layer,
+                                           int32_t* t_star, int32_t* act_scale, int32_t* keep, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if (!p || B < 0 || t < 1 || L < 1 || N_t < 1 || p->t_est < 2 || !(p->tau > 0.0))
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_keep_ratios_layers_device: bad argument");
+    if (B == 0) return NOVA_OK;
+    if (!hbar_scale || !hbar_layer || !keep)
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_keep_ratios_layers_device: null pointer");
+    NOVA_DEVICE_GUARD(ctx, "nova_keep_ratios_layers_device");
+    cudaStream_t st = (cudaStream_t)stream;
+    {
+        nova_launch_scope scope(ctx, NOVA_K_KEEP_RATIOS, st);
+        keep_ratios_layers_kernel<<<(L * B + 127) / 128, 128, 0, st>>>(*p, B, t, L, N_t, hbar_scale, hbar_layer, t_star,
+                                                                     act_scale, keep);
+    }
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    return NOVA_OK;
+}
+
 nova_status nova_keep_ratios(const nova_sched_params* p, int B, int t, int j, int N_t,
                              const float* hbar_scale, const float* hbar_layer,
                              int32_t* t_star, int32_t* act_scale,

@@ -232,19 +232,27 @@ extern "C" size_t nova_block_workspace_bytes(const nova_block_shape* s)
     return carve(nullptr, s->M, s->C, s->F).bytes;
 }
 
+// Where the block's output goes when the last GEMM scatters it straight into the token map (Eq. 15-16
+// on the kept rows) instead of writing the compacted y_kept.
+struct ScatterOut {
+    void* x_out;        // [B, N, C]: kept rows receive the layer output
+    void* cache_out;    // [B, N, C] or NULL: kept rows receive output - input
+};
+
 // m_on_device: s->M is only an upper bound of the kept rows (it sizes grids, tensor maps and the
 // workspace); every kernel takes the true count from cu_keep[B] on the device.
 static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, const nova_block_modulation* mod,
                                  const nova_block_shape* s, const void* x_in,
                                  const int32_t* keep_idx, const int32_t* cu_keep,
                                  void* k_cache, void* v_cache, int32_t* kv_len,
-                                 int append_kv, void* y_kept, void* stream, bool m_on_device)
+                                 int append_kv, void* y_kept, void* stream, bool m_on_device,
+                                 const ScatterOut* scatter = nullptr)
 {
     if (!ctx) return NOVA_ERR_INVALID_ARG;
     if (!w || !s) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward: null weights or shape");
     if (!shape_ok(s)) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_pruned_block_forward: unsupported shape");
     if (s->M == 0) return NOVA_OK;
-    if (!x_in || !keep_idx || !cu_keep || !k_cache || !v_cache || !kv_len || !y_kept)
+    if (!x_in || !keep_idx || !cu_keep || !k_cache || !v_cache || !kv_len || (!y_kept && !scatter))
         return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward: null tensor");
     const void* wp[] = {w->ln1_g, w->ln1_b, w->w_qkv, w->b_qkv, w->w_o, w->b_o,
                         w->ln2_g, w->ln2_b, w->w_fc1, w->b_fc1, w->w_fc2, w->b_fc2};
@@ -318,6 +326,11 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
     g.A = ws.f; g.W = (cbf)w->w_fc2; g.bias = (cbf)w->b_fc2; g.M = M; g.m_dev = m_dev; g.N = C; g.K = F;
     g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_FC2; g.out = (bf)y_kept; g.res = ws.x1; g.res_row = nullptr;
     g.gate = (cbf)md.gate2; g.img_row = ws.img_row;
+    if (scatter) {
+        // kept row r is token src_row[r] of the map: x_out[token] = y, cache_out[token] = y - x_in[token]
+        g.out = (bf)scatter->x_out; g.out_row = ws.src_row;
+        g.diff_in = (cbf)x_in; g.diff_out = (bf)scatter->cache_out;
+    }
     if (append_kv) {
         // the last kernel of the block also advances kv_len: every reader of the old lengths (row
         // maps, attention) ran in an earlier kernel of this call
@@ -355,6 +368,36 @@ extern "C" nova_status nova_pruned_block_forward_adaln(nova_ctx* ctx, const nova
 {
     return block_forward(ctx, w, mod, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream,
                          m_on_device != 0);
+}
+
+// Eq. 14 followed by Eq. 15-16 for one layer: the block on the kept rows with its last GEMM writing
+// the kept rows of x_out / cache_out directly, then the pruned rows from the upsampled cache.
+extern "C" nova_status nova_pruned_layer_forward(nova_ctx* ctx, const nova_block_weights* w,
+                                                 const nova_block_modulation* mod, const nova_block_shape* s,
+                                                 const void* x_in, const int32_t* keep_idx, const int32_t* prune_idx,
+                                                 const int32_t* cu_keep, void* k_cache, void* v_cache, int32_t* kv_len,
+                                                 int append_kv, const void* cache_prev, int hp, int wp, int h, int w_,
+                                                 void* x_out, void* cache_out, int m_on_device, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if (!s) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_layer_forward: null shape");
+    if (!shape_ok(s)) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_pruned_layer_forward: unsupported shape");
+    if ((long)h * w_ != (long)s->N) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_layer_forward: h * w must equal N");
+    if (!x_in || !x_out || !cu_keep) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_layer_forward: null tensor");
+    if (x_out == x_in) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_layer_forward: x_out aliases x_in");
+    if (!nova_aligned16(x_out) || !nova_aligned16(cache_out))
+        return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_pruned_layer_forward: tensors must be 16-byte aligned");
+    const long total = (long)s->B * s->N;
+    if (total > 0x7fffffffL) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_pruned_layer_forward: too many rows");
+    const bool on_dev = m_on_device != 0;
+    if ((s->M < total || on_dev) && (!prune_idx || !cache_prev || hp < 1 || wp < 1))
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_layer_forward: pruned rows need prune_idx and cache_prev");
+    ScatterOut sc = {x_out, cache_out};
+    nova_status rc = block_forward(ctx, w, mod, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, nullptr,
+                                   stream, on_dev, &sc);
+    if (rc != NOVA_OK) return rc;
+    return nova_restore_pruned_rows(ctx, x_in, prune_idx, cu_keep, cache_prev, hp, wp, h, w_, s->C, s->B, s->M, on_dev,
+                                    x_out, cache_out, stream);
 }
 
 // ---- block forward for callers that cannot allocate device memory --------------------------

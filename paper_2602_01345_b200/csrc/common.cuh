@@ -151,6 +151,11 @@ struct nova_gemm_args {
     const int32_t* res_row;     // row map into res, or NULL for identity
     const __nv_bfloat16* gate;  // NULL, or [images, N]: out = res + gate[img_row[r]] * (acc + bias)
     const int32_t* img_row;     // [M] image of each row (needed with gate)
+    // scattered output (residual epilogue only): row r goes to row out_row[r] of `out`, and, with
+    // diff_out, diff_out[out_row[r]] = out value - diff_in[out_row[r]] (Eq. 15 on the kept rows)
+    const int32_t* out_row;
+    const __nv_bfloat16* diff_in;
+    __nv_bfloat16* diff_out;
     // QKV epilogue
     int C;
     __nv_bfloat16* k_cache;
@@ -178,3 +183,9 @@ struct nova_attn_args {
 };
 
 nova_status nova_launch_attention(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st);
+
+// Eq. 16 for the pruned rows only (restore.cu); the kept rows were written by the block's last epilogue.
+nova_status nova_restore_pruned_rows(nova_ctx* ctx, const void* x_in, const int32_t* prune_idx,
+                                     const int32_t* cu_keep, const void* cache_prev,
+                                     int hp, int wp, int h, int w, int C, int B, int M, bool m_on_device,
+                                     void* x_out, void* cache_out, void* stream);

@@ -257,12 +257,23 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                  ::"r"(tc::smem_u32(dst)), "l"(src), "r"(bytes), "r"(tc::smem_u32(bar)) : "memory");
 }
 
+// Logits of several layers in one launch: layer l's [S, N, V] tensor starts at p[l]; row r of the
+// launch is row r % rows_per_layer of layer r / rows_per_layer.
+constexpr int kMaxEntropyLayers = 64;
+struct LayerPtrs {
+    const char* p[kMaxEntropyLayers];
+};
+
 template <int VEC, bool BF16>
 __global__ void __launch_bounds__(kRingThreads, 1)
-entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_stride_bytes,
+entropy_rows_ring(const LayerPtrs layers, long rows_per_layer, long rows, int V, long row_stride_bytes,
                   float* __restrict__ ent, float* __restrict__ mean, int seg_rows, int n_seg,
                   unsigned int* status, unsigned long long* __restrict__ accum, int fix_shift)
 {
+    auto row_ptr = [&](long row) -> const char* {
+        const long l = row / rows_per_layer;
+        return layers.p[l] + (row - l * rows_per_layer) * row_stride_bytes;
+    };
     using namespace tc;
     constexpr int kRowBytes = VEC * 512;
     constexpr int kSlots = kRingBytes / kRowBytes;
@@ -299,7 +310,7 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
                 if (i >= kSlots && !mbar_wait(&empty_bar[slot], (uint32_t)((i / kSlots) - 1) & 1, abort_flag, status)) break;
                 const long row = blockIdx.x + i * G;
                 mbar_arrive_expect_tx(&full_bar[slot], kRowBytes);
-                bulk_load(ring + slot * kRowBytes, logits + row * row_stride_bytes, kRowBytes, &full_bar[slot]);
+                bulk_load(ring + slot * kRowBytes, row_ptr(row), kRowBytes, &full_bar[slot]);
                 issued = i + 1;
             }
             if (*abort_flag)
@@ -321,7 +332,7 @@ entropy_rows_ring(const char* __restrict__ logits, long rows, int V, long row_st
             if (lane == 0) mbar_arrive(&empty_bar[slot]);       // the row now lives in registers
             const long row = blockIdx.x + i * G;
             float m, s_sum, u;
-            entropy_row_from_regs<VEC, BF16>(reg, logits + row * row_stride_bytes, V, lane, m, s_sum, u);
+            entropy_row_from_regs<VEC, BF16>(reg, row_ptr(row), V, lane, m, s_sum, u);
             if (lane == 0) {
                 const float h = finish_row(m, s_sum, u, ent, row, status);
                 if (mean) {
@@ -420,8 +431,8 @@ void launch_rows(const void* logits, long rows, int V, long row_stride, float* e
 }
 
 template <int VEC, bool BF16>
-nova_status launch_ring(nova_ctx* ctx, const void* logits, long rows, int V, long stride_bytes, float* ent,
-                        float* mean, int N, int S, cudaStream_t st)
+nova_status launch_ring(nova_ctx* ctx, const LayerPtrs& layers, long rows_per_layer, long rows, int V, long stride_bytes,
+                        float* ent, float* mean, int N, int S, cudaStream_t st)
 {
     constexpr int kSlots = kRingBytes / (VEC * 512);
     const size_t smem = kRingBytes + 128 + 2 * sizeof(uint64_t) * kSlots + sizeof(float) * kRingConsumers * kMaxMeanSegments;
@@ -437,7 +448,7 @@ nova_status launch_ring(nova_ctx* ctx, const void* logits, long rows, int V, lon
     int fix_shift = 30;
     while (fix_shift > 0 && 24.0 * (double)N * exp2((double)fix_shift) >= 70368744177664.0 /* 2^46 */) --fix_shift;
     entropy_rows_ring<VEC, BF16><<<grid, kRingThreads, smem, st>>>(
-        (const char*)logits, rows, V, stride_bytes, ent, mean, N, S, ctx->dev_status,
+        layers, rows_per_layer, rows, V, stride_bytes, ent, mean, N, S, ctx->dev_status,
         (unsigned long long*)(ctx->dev_status + NOVA_STATUS_WORDS), fix_shift);
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
@@ -445,40 +456,62 @@ nova_status launch_ring(nova_ctx* ctx, const void* logits, long rows, int V, lon
 
 }  // namespace
 
-extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nova_dtype dt,
-                                          int S, int N, int V, int64_t row_stride,
-                                          float* ent, float* mean, void* stream)
+// Entropy of n_layers tensors [S, N, V] (one per layer of a scale; `layers` holds their device
+// addresses) into ent [n_layers, S, N] and mean [n_layers, S]: one launch of the persistent ring
+// kernel over all n_layers * S * N rows where the shape allows it, else one launch per layer.
+static nova_status entropy_layers(nova_ctx* ctx, const void* const* layers, int n_layers, nova_dtype dt,
+                                  int S, int N, int V, int64_t row_stride, float* ent, float* mean, void* stream,
+                                  const char* who)
 {
     if (!ctx) return NOVA_ERR_INVALID_ARG;
-    if (S < 0 || N < 0 || V < 1 || (dt != NOVA_BF16 && dt != NOVA_F32))
-        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_scale_entropy: bad S, N, V or dtype");
-    const long rows = (long)S * N;
+    if (n_layers < 0 || S < 0 || N < 0 || V < 1 || (dt != NOVA_BF16 && dt != NOVA_F32))
+        return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_scale_entropy: bad layer count, S, N, V or dtype");
+    const long rows_per_layer = (long)S * N;
+    const long rows = rows_per_layer * n_layers;
     if (rows == 0) return NOVA_OK;
-    if (!logits || !ent) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_scale_entropy: null pointer");
+    if (!layers || !ent) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_scale_entropy: null pointer");
     const int per = (dt == NOVA_BF16) ? 8 : 4;
-    if (row_stride < V || (row_stride % per) != 0 || !nova_aligned16(logits))
-        return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_scale_entropy: logits rows must start on 16-byte boundaries");
-    NOVA_DEVICE_GUARD(ctx, "nova_scale_entropy");
+    for (int l = 0; l < n_layers; ++l) {
+        if (!layers[l]) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_scale_entropy: null pointer");
+        if (row_stride < V || (row_stride % per) != 0 || !nova_aligned16(layers[l]))
+            return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_scale_entropy: logits rows must start on 16-byte boundaries");
+    }
+    NOVA_DEVICE_GUARD(ctx, who);
     cudaStream_t st = (cudaStream_t)stream;
     const int elt = (dt == NOVA_BF16) ? 2 : 4;
     const long row_bytes = (long)V * elt;
+    const long segs = (long)n_layers * S;
     if ((row_bytes == 2048 || row_bytes == 4096 || row_bytes == 8192) && rows >= 64 && rows <= 0x7fffffffL &&
-        (!mean || (S <= NOVA_MEAN_MAX_SEGMENTS && ctx->num_sms <= NOVA_MEAN_MAX_CTAS))) {
-        // persistent ring kernel; the second word of the status allocation is its completion counter
+        n_layers <= kMaxEntropyLayers &&
+        (!mean || (segs <= NOVA_MEAN_MAX_SEGMENTS && ctx->num_sms <= NOVA_MEAN_MAX_CTAS))) {
+        // persistent ring kernel over the rows of all layers
+        LayerPtrs lp;
+        memset(&lp, 0, sizeof(lp));
+        for (int l = 0; l < n_layers; ++l) lp.p[l] = (const char*)layers[l];
         const long stride_bytes = (long)row_stride * elt;
         nova_launch_scope scope(ctx, NOVA_K_ENTROPY, st);
         const bool bf = (dt == NOVA_BF16);
-        if (row_bytes == 2048) return bf ? launch_ring<4, true>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st)
-                                         : launch_ring<4, false>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st);
-        if (row_bytes == 4096) return bf ? launch_ring<8, true>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st)
-                                         : launch_ring<8, false>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st);
-        return bf ? launch_ring<16, true>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st)
-                  : launch_ring<16, false>(ctx, logits, rows, V, stride_bytes, ent, mean, N, S, st);
+        const int sg = (int)segs;
+        if (row_bytes == 2048) return bf ? launch_ring<4, true>(ctx, lp, rows_per_layer, rows, V, stride_bytes, ent, mean, N, sg, st)
+                                         : launch_ring<4, false>(ctx, lp, rows_per_layer, rows, V, stride_bytes, ent, mean, N, sg, st);
+        if (row_bytes == 4096) return bf ? launch_ring<8, true>(ctx, lp, rows_per_layer, rows, V, stride_bytes, ent, mean, N, sg, st)
+                                         : launch_ring<8, false>(ctx, lp, rows_per_layer, rows, V, stride_bytes, ent, mean, N, sg, st);
+        return bf ? launch_ring<16, true>(ctx, lp, rows_per_layer, rows, V, stride_bytes, ent, mean, N, sg, st)
+                  : launch_ring<16, false>(ctx, lp, rows_per_layer, rows, V, stride_bytes, ent, mean, N, sg, st);
+    }
+    if (n_layers > 1) {
+        // shapes the ring kernel does not take: layer by layer
+        for (int l = 0; l < n_layers; ++l) {
+            const nova_status rc = entropy_layers(ctx, layers + l, 1, dt, S, N, V, row_stride, ent + (long)l * rows_per_layer,
+                                                  mean ? mean + (long)l * S : nullptr, stream, who);
+            if (rc != NOVA_OK) return rc;
+        }
+        return NOVA_OK;
     }
     {
         nova_launch_scope scope(ctx, NOVA_K_ENTROPY, st);
-        if (dt == NOVA_BF16) launch_rows<true>(logits, rows, V, row_stride, ent, ctx->dev_status, st);
-        else launch_rows<false>(logits, rows, V, row_stride, ent, ctx->dev_status, st);
+        if (dt == NOVA_BF16) launch_rows<true>(layers[0], rows, V, row_stride, ent, ctx->dev_status, st);
+        else launch_rows<false>(layers[0], rows, V, row_stride, ent, ctx->dev_status, st);
     }
     if (mean) {
         nova_launch_scope scope(ctx, NOVA_K_ENTROPY_MEAN, st);
@@ -486,6 +519,22 @@ extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nov
     }
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
+}
+
+extern "C" nova_status nova_scale_entropy(nova_ctx* ctx, const void* logits, nova_dtype dt,
+                                          int S, int N, int V, int64_t row_stride,
+                                          float* ent, float* mean, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    if ((long)S * N != 0 && !logits) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_scale_entropy: null pointer");
+    return entropy_layers(ctx, &logits, 1, dt, S, N, V, row_stride, ent, mean, stream, "nova_scale_entropy");
+}
+
+extern "C" nova_status nova_scale_entropy_layers(nova_ctx* ctx, const void* const* logits, int n_layers, nova_dtype dt,
+                                                 int S, int N, int V, int64_t row_stride,
+                                                 float* ent, float* mean, void* stream)
+{
+    return entropy_layers(ctx, logits, n_layers, dt, S, N, V, row_stride, ent, mean, stream, "nova_scale_entropy_layers");
 }
 
 // Eq. 4 / Eq. 7 one step earlier: entropy of softmax(x W^T + b) without the logits ever reaching

@@ -70,6 +70,9 @@ struct GemmParams {
     const int32_t* m_dev;
     const __nv_bfloat16* gate;
     const int32_t* img_row;
+    const int32_t* out_row;
+    const __nv_bfloat16* diff_in;
+    __nv_bfloat16* diff_out;
 };
 
 // Rows of this launch: p.M, or the device-side count when the host only knows an upper bound.
@@ -137,7 +140,27 @@ __device__ __forceinline__ void epilogue_chunk(const GemmParams& p, int row, int
                 v[i * 8 + j * 2 + 1] += __uint_as_float(rw[j] & 0xffff0000u);
             }
         }
-        dst = p.out + (long)row * p.N + col0;
+        const long orow = p.out_row ? (long)p.out_row[row] : (long)row;
+        dst = p.out + orow * p.N + col0;
+        if (p.diff_out) {
+            // second output: the stored (bf16-rounded) value minus diff_in's row, i.e. what a separate
+            // pass over the stored output would compute
+            const uint4* x4 = (const uint4*)(p.diff_in + orow * p.N + col0);
+            uint4* c4 = (uint4*)(p.diff_out + orow * p.N + col0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 x = x4[i];
+                const uint32_t xw[4] = {x.x, x.y, x.z, x.w};
+                uint32_t o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t yb = pack_bf16(v[i * 8 + j * 2], v[i * 8 + j * 2 + 1]);
+                    o[j] = pack_bf16(__uint_as_float(yb << 16) - __uint_as_float(xw[j] << 16),
+                                     __uint_as_float(yb & 0xffff0000u) - __uint_as_float(xw[j] & 0xffff0000u));
+                }
+                c4[i] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
     } else {
         // QKV routing: this 32-column chunk lies entirely in q, k or v (C % 32 == 0)
         const int which = col0 / p.C, cc = col0 - which * p.C;
@@ -273,6 +296,7 @@ GemmParams make_params(nova_ctx* ctx, const nova_gemm_args& a)
     p.kv_row = a.kv_row; p.status = ctx->dev_status;
     p.adv_cu_keep = a.adv_cu_keep; p.adv_kv_len = a.adv_kv_len; p.adv_B = a.adv_B; p.adv_Lmax = a.adv_Lmax;
     p.ent = a.ent; p.m_dev = a.m_dev; p.gate = a.gate; p.img_row = a.img_row;
+    p.out_row = a.out_row; p.diff_in = a.diff_in; p.diff_out = a.diff_out;
     return p;
 }
 

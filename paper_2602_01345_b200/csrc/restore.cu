@@ -38,12 +38,14 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 restore_kernel(const uint4* __restrict__ x_in, const uint4* __restrict__ y_kept,
                const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ prune_idx,
                const int32_t* __restrict__ cu_keep, const uint4* __restrict__ cache_prev,
-               int hp, int wp, int h, int w, int vec_per_row, int B, int M, bool m_on_device,
+               int hp, int wp, int h, int w, int vec_per_row, int B, int M, bool m_on_device, bool pruned_only,
                uint4* __restrict__ x_out, uint4* __restrict__ cache_out)
 {
     if (m_on_device) M = cu_keep[B];    // the kept count lives on the device
     const int lane = threadIdx.x & 31;
-    const long r = (long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    // pruned_only: the kept rows were already written (by the block's last epilogue); work items
+    // start at the first pruned entry
+    const long r = (long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5) + (pruned_only ? M : 0);
     const int N = h * w;
     const long total = (long)B * N;
     if (r >= total) return;
@@ -132,7 +134,7 @@ static nova_status restore(nova_ctx* ctx, const void* x_in, const void* y_kept,
                            const int32_t* keep_idx, const int32_t* prune_idx,
                            const int32_t* cu_keep, const void* cache_prev,
                            int hp, int wp, int h, int w, int C, int B, int M, bool m_on_device,
-                           void* x_out, void* cache_out, void* stream)
+                           void* x_out, void* cache_out, void* stream, bool pruned_only = false)
 {
     if (!ctx) return NOVA_ERR_INVALID_ARG;
     if (B < 0 || h < 0 || w < 0 || C < 1 || M < 0 || (long)M > (long)B * h * w)
@@ -140,7 +142,7 @@ static nova_status restore(nova_ctx* ctx, const void* x_in, const void* y_kept,
     const long total = (long)B * h * w;
     if (total == 0) return NOVA_OK;
     if (C % 8) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_restore_from_cache: C must be a multiple of 8");
-    if (!x_in || !x_out || !cu_keep || (M > 0 && (!y_kept || !keep_idx)))
+    if (!x_in || !x_out || !cu_keep || (M > 0 && !pruned_only && (!y_kept || !keep_idx)))
         return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_restore_from_cache: null pointer");
     if ((M < total || m_on_device) && (!prune_idx || !cache_prev || hp < 1 || wp < 1))
         return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_restore_from_cache: pruned rows need prune_idx and cache_prev");
@@ -149,11 +151,14 @@ static nova_status restore(nova_ctx* ctx, const void* x_in, const void* y_kept,
         !nova_aligned16(cache_prev) || !nova_aligned16(cache_out))
         return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_restore_from_cache: tensors must be 16-byte aligned");
     NOVA_DEVICE_GUARD(ctx, "nova_restore_from_cache");
-    const unsigned blocks = (unsigned)((total + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    // rows this launch may have to visit: all of them, or only the pruned ones (when the host knows M)
+    const long items = (pruned_only && !m_on_device) ? total - M : total;
+    if (items == 0) return NOVA_OK;
+    const unsigned blocks = (unsigned)((items + kWarpsPerBlock - 1) / kWarpsPerBlock);
     nova_launch_scope scope(ctx, NOVA_K_RESTORE, (cudaStream_t)stream);
     restore_kernel<<<blocks, kWarpsPerBlock * 32, 0, (cudaStream_t)stream>>>(
         (const uint4*)x_in, (const uint4*)y_kept, keep_idx, prune_idx, cu_keep, (const uint4*)cache_prev,
-        hp, wp, h, w, C / 8, B, M, m_on_device, (uint4*)x_out, (uint4*)cache_out);
+        hp, wp, h, w, C / 8, B, M, m_on_device, pruned_only, (uint4*)x_out, (uint4*)cache_out);
     NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }
@@ -179,4 +184,16 @@ extern "C" nova_status nova_restore_from_cache_device(nova_ctx* ctx, const void*
     if (total > 0x7fffffffL) return nova_fail(ctx, NOVA_ERR_SHAPE, "nova_restore_from_cache_device: too many rows");
     return restore(ctx, x_in, y_kept, keep_idx, prune_idx, cu_keep, cache_prev, hp, wp, h, w, C, B, (int)total, true,
                    x_out, cache_out, stream);
+}
+
+
+// Eq. 16 for the pruned rows only: used by nova_pruned_layer_forward, whose last GEMM epilogue has
+// already written the kept rows of x_out and cache_out.
+nova_status nova_restore_pruned_rows(nova_ctx* ctx, const void* x_in, const int32_t* prune_idx,
+                                     const int32_t* cu_keep, const void* cache_prev,
+                                     int hp, int wp, int h, int w, int C, int B, int M, bool m_on_device,
+                                     void* x_out, void* cache_out, void* stream)
+{
+    return restore(ctx, x_in, nullptr, nullptr, prune_idx, cu_keep, cache_prev, hp, wp, h, w, C, B, M, m_on_device,
+                   x_out, cache_out, stream, true);
 }

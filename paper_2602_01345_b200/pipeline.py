@@ -1,9 +1,10 @@
 """One accelerated scale through all layers: the call sequence a user of the library makes.
 
-Entropy of every layer's logits -> (all means to the host in one copy) -> then for every layer j:
-keep counts from the trigger/ratio functions -> top-k selection -> block on the kept rows
--> restore of the pruned rows from the residual cache. This module only owns buffers and
-issues the five C-ABI calls in order; it computes nothing itself.
+The layers' logits are inputs of the scale, so the steps that depend only on them run once for all
+layers: entropy maps of every layer (one launch) -> all means to the host in one copy -> keep counts
+of every layer from the trigger/ratio functions -> top-k selection of every layer (one launch).
+Then for every layer j: block on the kept rows -> restore of the pruned rows from the residual
+cache. This module only owns buffers and issues the C-ABI calls in order; it computes nothing itself.
 """
 from __future__ import annotations
 
@@ -24,10 +25,14 @@ class PrunedScaleRunner:
 
     def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, h: int, w: int, Lmax: int,
                  k_caches, v_caches, kv_len, cache_prev, eps: float = 1e-6, keep_cache_out: bool = True,
-                 modulation=None):
+                 modulation=None, fused_restore: bool = False):
         """modulation: optional list of L dicts of per-image [B, C] bf16 tensors (adaptive LayerNorm
-        of the class-conditional backbones, see nova_pruned_block_forward_adaln)."""
+        of the class-conditional backbones, see nova_pruned_block_forward_adaln).
+        fused_restore: run each layer as one nova_pruned_layer_forward call (the block's last GEMM
+        scatters the kept rows into x_out / cache_out, the restore pass touches pruned rows only)
+        instead of nova_pruned_block_forward + nova_restore_from_cache; same results."""
         self.ctx = ctx
+        self.fused_restore = fused_restore
         self.modulation = modulation
         self.L = len(weights)
         self.B, self.h, self.w, self.N = B, h, w, h * w
@@ -43,9 +48,9 @@ class PrunedScaleRunner:
         self.ent = torch.empty((self.L, B, N), dtype=torch.float32, device=dev)
         self.mean = torch.empty((self.L, B), dtype=torch.float32, device=dev)
         self.mean_host = torch.empty((self.L, B), dtype=torch.float32).pin_memory()
-        self.keep_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
-        self.prune_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
-        self.cu_keep = torch.empty((B + 1,), dtype=torch.int32, device=dev)
+        self.keep_idx = torch.empty((self.L, B * N), dtype=torch.int32, device=dev)      # one list per layer
+        self.prune_idx = torch.empty((self.L, B * N), dtype=torch.int32, device=dev)
+        self.cu_keep = torch.empty((self.L, B + 1), dtype=torch.int32, device=dev)
         self.y_kept = torch.empty((B * N, Cc), dtype=torch.bfloat16, device=dev)
         self.x_buf = [torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev) for _ in range(2)]
         self.cache_out = ([torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev) for _ in range(self.L)]
@@ -67,44 +72,56 @@ class PrunedScaleRunner:
         ctx, B, N = self.ctx, self.B, self.N
         st = stream if stream is not None else torch.cuda.current_stream()
         # The layers' logits are inputs of the scale, not results of its layers, so the entropy maps
-        # of a whole group of layers are taken first and their means cross to the host in one copy:
-        # one synchronisation per group decides the keep counts of all its layers. With resident
-        # logits the group is the whole scale; while logits are still being uploaded a small group
-        # lets the blocks of the first layers run under the uploads of the later ones.
+        # of a whole group of layers are taken first, in one launch, and their means cross to the host
+        # in one copy: one synchronisation per group decides the keep counts of all its layers, and one
+        # more launch selects for all of them. With resident logits the group is the whole scale; while
+        # logits are still being uploaded a small group lets the blocks of the first layers run under
+        # the uploads of the later ones.
         group = self.L if logits_ready is None else min(self.L, 4)
-        hbar_layer = torch.empty((B, self.L), dtype=torch.float32)
+        hbar_layer = torch.zeros((B, self.L), dtype=torch.float32)
         keeps = []
         x = x_in
         for g0 in range(0, self.L, group):
             g1 = min(self.L, g0 + group)
-            for j in range(g0, g1):
-                if logits_ready is not None:
+            if logits_ready is not None:
+                for j in range(g0, g1):
                     st.wait_event(logits_ready[j])
-                nv.nova_scale_entropy(ctx, layer_logits[j], self.ent[j], self.mean[j], stream=st)
+            nv.nova_scale_entropy_layers(ctx, layer_logits[g0:g1], self.ent[g0:g1], self.mean[g0:g1], stream=st)
             self.mean_host[g0:g1].copy_(self.mean[g0:g1], non_blocking=True)
             st.synchronize()
             hbar_layer[:, g0:g1] = self.mean_host[g0:g1].t()
+            keep_all = nv.nova_keep_ratios_layers(sched, t, N, hbar_scale, hbar_layer[:, :g1])["keep"]
+            if select_ent is None:
+                nv.nova_select_topk_grouped(ctx, self.ent[g0:g1], keep_all[g0:g1], self.keep_idx[g0:g1],
+                                            self.prune_idx[g0:g1], self.cu_keep[g0:g1], None, stream=st)
             for j in range(g0, g1):
-                r = nv.nova_keep_ratios(sched, t, j + 1, N, hbar_scale, hbar_layer[:, : j + 1].contiguous())
-                keep = r["keep"]
+                keep = keep_all[j]
                 M = int(keep.sum())
                 keeps.append(keep)
-                nv.nova_select_topk(ctx, self.ent[j] if select_ent is None else select_ent, keep, self.keep_idx[:M],
-                                    self.prune_idx[: B * N - M], self.cu_keep, None, stream=st)
+                keep_idx, prune_idx, cu_keep = self.keep_idx[j, :M], self.prune_idx[j, : B * N - M], self.cu_keep[j]
+                if select_ent is not None:
+                    nv.nova_select_topk(ctx, select_ent, keep, keep_idx, prune_idx, cu_keep, None, stream=st)
                 shape = nv.BlockShape(B, N, self.C, self.n_heads, self.F, self.Lmax, M)
+                x_out = self.x_buf[j & 1] if x is not self.x_buf[j & 1] else self.x_buf[(j + 1) & 1]
+                cache_out = self.cache_out[j] if self.cache_out is not None else None
+                if self.fused_restore:
+                    nv.nova_pruned_layer_forward(ctx, self.weights[j], self.modulation[j] if self.modulation else None,
+                                                 shape, x, keep_idx, prune_idx, cu_keep, self.k_caches[j],
+                                                 self.v_caches[j], self.kv_len[j], append_kv, self.cache_prev[j],
+                                                 self.h, self.w, x_out, cache_out, stream=st)
+                    x = x_out
+                    continue
                 if self.modulation is None:
-                    nv.nova_pruned_block_forward(ctx, self.weights[j], shape, x, self.keep_idx[:M], self.cu_keep,
+                    nv.nova_pruned_block_forward(ctx, self.weights[j], shape, x, keep_idx, cu_keep,
                                                  self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
                                                  self.y_kept[:M], stream=st)
                 else:
                     nv.nova_pruned_block_forward_adaln(ctx, self.weights[j], self.modulation[j], shape, x,
-                                                       self.keep_idx[:M], self.cu_keep, self.k_caches[j],
+                                                       keep_idx, cu_keep, self.k_caches[j],
                                                        self.v_caches[j], self.kv_len[j], append_kv, self.y_kept[:M],
                                                        stream=st)
-                x_out = self.x_buf[j & 1] if x is not self.x_buf[j & 1] else self.x_buf[(j + 1) & 1]
-                nv.nova_restore_from_cache(ctx, x, self.y_kept[:M], self.keep_idx[:M], self.prune_idx[: B * N - M],
-                                           self.cu_keep, self.cache_prev[j], self.h, self.w, x_out,
-                                           self.cache_out[j] if self.cache_out is not None else None, stream=st)
+                nv.nova_restore_from_cache(ctx, x, self.y_kept[:M], keep_idx, prune_idx,
+                                           cu_keep, self.cache_prev[j], self.h, self.w, x_out, cache_out, stream=st)
                 x = x_out
         self.last_keep = keeps
         return x, keeps
@@ -175,8 +192,9 @@ class MultiScaleRunner:
 class DeviceScaleRunner:
     """One scale through all layers with every decision left on the device.
 
-    Per layer: entropy map and mean -> Eq. 8-13 in a one-thread-per-image kernel -> selection with
-    the keep counts read from device memory -> the block and the restore sized by an upper bound
+    For all layers at once: entropy maps and means -> Eq. 8-13 in a one-thread-per-(layer, image)
+    kernel -> selection with the keep counts read from device memory. Then per layer the block and
+    the restore sized by an upper bound
     (all B*N rows), the kept count read from cu_keep[B]. Nothing crosses to the host, so the whole
     scale is one uninterrupted run of launches that can be recorded in a CUDA graph once and
     replayed for every new batch of the same shape. Inputs live in fixed buffers:
@@ -188,10 +206,11 @@ class DeviceScaleRunner:
     def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, h: int, w: int, Lmax: int,
                  k_caches, v_caches, kv_len, cache_prev, sched: nv.SchedParams, t: int, hist, V: int,
                  eps: float = 1e-6, logits_dtype=torch.bfloat16, x_in=None, layer_logits=None,
-                 scale_entropy: bool = True, modulation=None):
+                 scale_entropy: bool = True, modulation=None, fused_restore: bool = False):
         """x_in / layer_logits: existing tensors to use as the fixed input buffers instead of new
         ones. scale_entropy=False: hist row t-1 is already filled by the caller (no scale_logits)."""
         self.ctx, self.sched, self.t = ctx, sched, t
+        self.fused_restore = fused_restore    # one nova_pruned_layer_forward call per layer
         self.modulation = modulation          # optional list of L dicts of [B, C] bf16 tensors (fixed buffers)
         self.L = len(weights)
         self.B, self.h, self.w, self.N = B, h, w, h * w
@@ -216,9 +235,9 @@ class DeviceScaleRunner:
         self.keep = torch.zeros((L, B), dtype=torch.int32, device=dev)
         self.t_star = torch.zeros((B,), dtype=torch.int32, device=dev)
         self.act_scale = torch.zeros((B,), dtype=torch.int32, device=dev)
-        self.keep_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
-        self.prune_idx = torch.empty((B * N,), dtype=torch.int32, device=dev)
-        self.cu_keep = torch.zeros((B + 1,), dtype=torch.int32, device=dev)
+        self.keep_idx = torch.empty((L, B * N), dtype=torch.int32, device=dev)       # one list per layer
+        self.prune_idx = torch.empty((L, B * N), dtype=torch.int32, device=dev)
+        self.cu_keep = torch.zeros((L, B + 1), dtype=torch.int32, device=dev)
         self.y_kept = torch.empty((B * N, Cc), dtype=torch.bfloat16, device=dev)
         self.x_buf = [torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev) for _ in range(2)]
         self.cache_out = [torch.empty((B, N, Cc), dtype=torch.bfloat16, device=dev) for _ in range(L)]
@@ -234,23 +253,33 @@ class DeviceScaleRunner:
         hist_t = self.hist[:t]
         if self.scale_logits is not None:
             nv.nova_scale_entropy(ctx, self.scale_logits, self.ent_scale, hist_t[t - 1], stream=st)
+        # everything that depends only on the scale's logits, for all layers at once: three launches
+        nv.nova_scale_entropy_layers(ctx, self.layer_logits, self.ent, self.mean, stream=st)
+        nv.nova_keep_ratios_layers_device(ctx, self.sched, t, N, hist_t, self.mean, self.keep, self.t_star,
+                                          self.act_scale, stream=st)
+        nv.nova_select_topk_grouped(ctx, self.ent, self.keep, self.keep_idx, self.prune_idx, self.cu_keep, None,
+                                    stream=st)
         x = self.x_in
         for j in range(self.L):
-            nv.nova_scale_entropy(ctx, self.layer_logits[j], self.ent[j], self.mean[j], stream=st)
-            nv.nova_keep_ratios_device(ctx, self.sched, t, j + 1, N, hist_t, self.mean[: j + 1], self.keep[j],
-                                       self.t_star, self.act_scale, stream=st)
-            nv.nova_select_topk_device(ctx, self.ent[j], self.keep[j], self.keep_idx, self.prune_idx, self.cu_keep,
-                                       None, stream=st)
+            keep_idx, prune_idx, cu_keep = self.keep_idx[j], self.prune_idx[j], self.cu_keep[j]
+            if self.fused_restore:
+                x_out = self.x_buf[j & 1]
+                nv.nova_pruned_layer_forward(ctx, self.weights[j], self.modulation[j] if self.modulation else None,
+                                             self.shape, x, keep_idx, prune_idx, cu_keep, self.k_caches[j],
+                                             self.v_caches[j], self.kv_len[j], append_kv, self.cache_prev[j],
+                                             self.h, self.w, x_out, self.cache_out[j], m_on_device=True, stream=st)
+                x = x_out
+                continue
             if self.modulation is None:
-                nv.nova_pruned_block_forward_device(ctx, self.weights[j], self.shape, x, self.keep_idx, self.cu_keep,
+                nv.nova_pruned_block_forward_device(ctx, self.weights[j], self.shape, x, keep_idx, cu_keep,
                                                     self.k_caches[j], self.v_caches[j], self.kv_len[j], append_kv,
                                                     self.y_kept, stream=st)
             else:
                 nv.nova_pruned_block_forward_adaln(ctx, self.weights[j], self.modulation[j], self.shape, x,
-                                                   self.keep_idx, self.cu_keep, self.k_caches[j], self.v_caches[j],
+                                                   keep_idx, cu_keep, self.k_caches[j], self.v_caches[j],
                                                    self.kv_len[j], append_kv, self.y_kept, m_on_device=True, stream=st)
             x_out = self.x_buf[j & 1]
-            nv.nova_restore_from_cache_device(ctx, x, self.y_kept, self.keep_idx, self.prune_idx, self.cu_keep,
+            nv.nova_restore_from_cache_device(ctx, x, self.y_kept, keep_idx, prune_idx, cu_keep,
                                               self.cache_prev[j], self.h, self.w, x_out, self.cache_out[j], stream=st)
             x = x_out
         return x

@@ -84,6 +84,34 @@ def test_keep_ratios_bit_exact_against_oracle_random_histories():
         _compare(oracle.SchedParams(**kw), nova.SchedParams(**kw), T, j, N, hs, hl)
 
 
+def test_keep_ratios_all_layers_equals_layer_by_layer_and_oracle():
+    """The all-layers call gives, for every layer j, what the per-layer call and the oracle give on
+    the means of layers 1..j (Eq. 12-13), bit for bit."""
+    rng = np.random.default_rng(3)
+    for trial in range(40):
+        B, T, L = int(rng.integers(1, 9)), int(rng.integers(6, 14)), int(rng.integers(1, 33))
+        N = int(rng.choice([256, 1024, 4096]))
+        t_axis = np.arange(1, T + 1)
+        hs = (2 + 6 / (1 + np.exp(-(t_axis[None] - rng.uniform(1, 6, (B, 1))) / rng.uniform(0.4, 2, (B, 1)))) +
+              0.05 * rng.standard_normal((B, T))).astype(np.float32)
+        hl = (hs[:, -1:] * rng.uniform(0.7, 1.3, (B, L))).astype(np.float32)
+        kw = dict(lam=float(rng.uniform(0, 0.3)), tau=float(rng.uniform(0.3, 2.0)))
+        if trial % 4 == 0:
+            kw["force_act_scale"] = T - 1
+        got = nova.nova_keep_ratios_layers(nova.SchedParams(**kw), T, N, torch.from_numpy(hs), torch.from_numpy(hl))
+        pruned = 0
+        for j in range(1, L + 1):
+            want = oracle.keep_ratios(oracle.SchedParams(**kw), T, j, N, hs, hl[:, :j].copy())
+            assert np.array_equal(got["keep"][j - 1].numpy(), want["keep"]), (trial, j)
+            assert np.array_equal(got["ratio_layer"][j - 1].numpy(), want["ratio_layer"]), (trial, j)
+            pruned += int((want["keep"] < N).sum())
+        assert np.array_equal(got["t_star"].numpy(), want["t_star"])
+        assert np.array_equal(got["act_scale"].numpy(), want["act_scale"])
+        assert np.array_equal(got["ratio_scale"].numpy(), want["ratio_scale"])
+        if trial % 4 == 0:
+            assert pruned > 0
+
+
 def test_keep_ratios_worked_example_and_errors():
     hs = np.array([[1, 2, 3, 4, 5, 6, 6, 6, 6, 6]], np.float32)
     got = nova.nova_keep_ratios(nova.SchedParams(), 8, 1, 256, torch.from_numpy(hs[:, :8]))

@@ -164,6 +164,33 @@ def test_entropy_empty_and_bad_args(ctx):
     assert ei.value.status == 3
 
 
+@pytest.mark.parametrize("L,S,N,V", [
+    (3, 2, 700, 4096),      # the persistent kernel over three layers' rows: one launch
+    (5, 4, 64, 2048),       # fewer rows per layer than CTAs: rows of several layers inside every CTA
+    (2, 2, 9, 1000),        # a shape the persistent kernel does not take: layer by layer
+])
+def test_entropy_all_layers_in_one_call(ctx, L, S, N, V):
+    """The entropy maps of all layers of a scale from separate logits tensors: equal, bit for bit,
+    to one nova_scale_entropy call per layer, within tolerance of the oracle, in a single launch
+    where the persistent kernel applies."""
+    from paper_2602_01345_b200 import pipeline
+    a = synth.smooth_temperature_field(S, 1, N, seed=3, device=DEV)
+    logits = [synth.logits_from_temperature(a * (0.8 + 0.2 * l), V, seed=40 + l) for l in range(L)]
+    ent = torch.full((L, S, N), float("nan"), dtype=torch.float32, device=DEV)
+    mean = torch.full((L, S), float("nan"), dtype=torch.float32, device=DEV)
+    n0 = pipeline.launch_count(ctx)
+    nova.nova_scale_entropy_layers(ctx, logits, ent, mean)
+    launches = pipeline.launch_count(ctx) - n0
+    assert launches == (1 if V in (2048, 4096) else 2 * L)
+    for l in range(L):
+        e1, m1 = gpu_entropy(ctx, logits[l])
+        assert torch.equal(ent[l], e1) and torch.equal(mean[l], m1)
+        want_ent, want_mean = oracle.scale_entropy(f32(logits[l]))
+        assert np.abs(ent[l].cpu().numpy() - want_ent).max() <= ENT_TOL
+        assert np.abs(mean[l].cpu().numpy() - want_mean).max() <= ENT_TOL
+    assert ctx.device_status() == 0
+
+
 # ------------------------------------------------------- entropy fused with the codebook head
 def _head_case(ctx, S, N, C, V, seed, bias=True, sample=None):
     x = synth.activations(S, N, C, seed, DEV)
@@ -255,6 +282,38 @@ def test_select_edge_counts_and_many_segments(ctx):
     assert np.array_equal(cu.cpu().numpy(), w_cu)
     assert np.array_equal(keep_idx.cpu().numpy(), w_keep)
     assert np.array_equal(prune_idx.cpu().numpy(), w_prune)
+
+
+@pytest.mark.parametrize("G,S,N", [(3, 4, 1000), (32, 4, 4096), (70, 4, 300), (2, 1, 16384)])
+@pytest.mark.parametrize("counts_on_device", [False, True])
+def test_select_all_layers_in_one_call(ctx, G, S, N, counts_on_device):
+    """The selection of G layers x S images in one call: every layer's index lists, cumulative
+    counts and positions equal the oracle's for that layer, with host and with device keep counts.
+    (32, 4, 4096) is the benchmark's launch; (70, 4, 300) needs more than 256 segments."""
+    from paper_2602_01345_b200 import pipeline
+    g = torch.Generator(device="cpu").manual_seed(G * 1009 + N)
+    ent = torch.rand((G, S, N), generator=g) * 8.0
+    ent[:, :, ::7] = ent[:, :, 1:2]                    # exact ties
+    k = torch.randint(0, N + 1, (G, S), generator=g).to(torch.int32)
+    k[0, 0], k[-1, -1] = N // 2, N
+    if S > 1:
+        k[0, 1] = 0
+    keep_idx = torch.full((G, S * N), -7, dtype=torch.int32, device=DEV)
+    prune_idx = torch.full((G, S * N), -7, dtype=torch.int32, device=DEV)
+    cu = torch.full((G, S + 1), -7, dtype=torch.int32, device=DEV)
+    pos = torch.full((G, S, N), -7, dtype=torch.int32, device=DEV)
+    n0 = pipeline.launch_count(ctx)
+    nova.nova_select_topk_grouped(ctx, ent.to(DEV), k.to(DEV) if counts_on_device else k, keep_idx, prune_idx, cu, pos)
+    launches = pipeline.launch_count(ctx) - n0
+    assert launches == (1 if counts_on_device or G * S <= 256 else 2)
+    kk, pp, cc, ps = keep_idx.cpu().numpy(), prune_idx.cpu().numpy(), cu.cpu().numpy(), pos.cpu().numpy()
+    for l in range(G):
+        w_keep, w_prune, w_cu, w_pos = oracle.select_topk(ent[l].numpy(), k[l].numpy())
+        M = int(w_cu[-1])
+        assert np.array_equal(cc[l], w_cu), l
+        assert np.array_equal(kk[l, :M], w_keep) and np.array_equal(pp[l, : S * N - M], w_prune), l
+        assert np.array_equal(ps[l], w_pos), l
+        assert (kk[l, M:] == -7).all() and (pp[l, S * N - M:] == -7).all()      # nothing written past the lists
 
 
 def test_select_teacher_forced_on_gpu_entropy(ctx):
@@ -652,6 +711,86 @@ def test_block_bad_args(ctx):
     assert ei.value.status == 4
 
 
+# ------------------------------------------------- block + restore in one call (scattered last epilogue)
+@pytest.mark.parametrize("case", ["config1", "ragged_small", "keep_all", "keep_none", "device_count", "modulated",
+                                  "no_cache_out", "full_size_1024"])
+def test_layer_forward_equals_block_then_restore(ctx, case):
+    """nova_pruned_layer_forward (the block's last GEMM scatters the kept rows into x_out and writes
+    their residual to cache_out; the restore pass touches pruned rows only) gives bit for bit what
+    nova_pruned_block_forward + nova_restore_from_cache give, and both match the oracle's block
+    followed by its restore."""
+    md = None
+    if case == "full_size_1024":
+        B, h, w, hp, wp, C, heads, F, Lmax = 4, 64, 64, 48, 48, 2048, 16, 8192, 10521
+        ks, kv_lens = [2048, 1901, 2048, 2100], [6425] * 4
+    elif case == "config1" or case == "modulated":
+        B, h, w, hp, wp, C, heads, F, Lmax = 2, 16, 16, 13, 13, 1024, 16, 4096, 680
+        ks, kv_lens = [128, 101], [424, 424]
+        if case == "modulated":
+            md = _modulation(B, C, 77)
+    else:
+        B, h, w, hp, wp, C, heads, F, Lmax = 3, 10, 15, 7, 9, 128, 2, 256, 512
+        ks = {"keep_all": [150] * 3, "keep_none": [0] * 3}.get(case, [150, 37, 0])
+        kv_lens = [0, 130, 17]
+    N, M = h * w, sum(ks)
+    wt = synth.block_weights(C, F, 31, DEV)
+    bw = nova.BlockWeights(wt, 1e-6)
+    x = synth.activations(B, N, C, 32, DEV)
+    k_cache, v_cache, _ = synth.kv_cache(B, Lmax, max(kv_lens), C, 33, DEV)
+    cache_prev = synth.residual_cache(B, hp, wp, C, 34, DEV)
+    ent = torch.rand((B, N), generator=torch.Generator(device="cpu").manual_seed(31))
+    on_device = case == "device_count"
+    cap = B * N if on_device else M
+    keep_idx = torch.zeros(max(cap, 1), dtype=torch.int32, device=DEV)
+    prune_idx = torch.zeros(B * N, dtype=torch.int32, device=DEV)
+    cu = torch.empty(B + 1, dtype=torch.int32, device=DEV)
+    nova.nova_select_topk(ctx, ent.to(DEV), torch.tensor(ks, dtype=torch.int32), keep_idx[:M], prune_idx[: B * N - M], cu, None)
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, cap)
+    ctx.ensure_workspace(shape)
+    want_cache = case != "no_cache_out"
+    # two calls
+    ka, va, la = k_cache.clone(), v_cache.clone(), torch.tensor(kv_lens, dtype=torch.int32, device=DEV)
+    y = torch.full((max(cap, 1), C), float("nan"), dtype=torch.bfloat16, device=DEV)
+    xa = torch.full_like(x, float("nan"))
+    ca = torch.full_like(x, float("nan")) if want_cache else None
+    if M > 0:
+        nova.nova_pruned_block_forward_adaln(ctx, bw, md, shape, x, keep_idx[:cap], cu, ka, va, la, True, y[:cap],
+                                             m_on_device=on_device)
+    if on_device:
+        nova.nova_restore_from_cache_device(ctx, x, y, keep_idx, prune_idx, cu, cache_prev, h, w, xa, ca)
+    else:
+        nova.nova_restore_from_cache(ctx, x, y[:M], keep_idx[:M], prune_idx[: B * N - M], cu, cache_prev, h, w, xa, ca)
+    # one call
+    kb, vb, lb = k_cache.clone(), v_cache.clone(), torch.tensor(kv_lens, dtype=torch.int32, device=DEV)
+    xb = torch.full_like(x, float("nan"))
+    cb = torch.full_like(x, float("nan")) if want_cache else None
+    nova.nova_pruned_layer_forward(ctx, bw, md, shape, x, keep_idx[:cap], prune_idx if on_device else prune_idx[: B * N - M],
+                                   cu, kb, vb, lb, True, cache_prev, h, w, xb, cb, m_on_device=on_device)
+    assert ctx.device_status() == 0
+    assert torch.equal(xa, xb) and torch.equal(ka, kb) and torch.equal(va, vb) and torch.equal(la, lb)
+    if want_cache:
+        assert torch.equal(ca, cb)
+    assert torch.isfinite(xb.float()).all()
+    # against the oracle (sampled kept rows at the full size; every pruned row in any case)
+    ki, pi, cuu = keep_idx[:M].cpu().numpy(), prune_idx[: B * N - M].cpu().numpy(), cu.cpu().numpy()
+    rows = None
+    if case == "full_size_1024":
+        rows = np.array([0, 127, 2047, 2048, 2048 + 1900, M - 2100, M - 1], np.int32)
+    mod_np = {n: f32(t) for n, t in md.items()} if md else None
+    wy, _, _ = oracle.pruned_block_forward({n: f32(t) for n, t in wt.items()}, 1e-6, heads, f32(x), ki, cuu, f32(k_cache),
+                                           f32(v_cache), np.array(kv_lens, np.int32), rows=rows, modulation=mod_np)
+    gx = f32(xb)
+    rr = np.arange(M) if rows is None else rows
+    if M > 0:
+        img = np.searchsorted(cuu, rr, side="right") - 1
+        assert _rel_err(gx[img, ki[rr]], wy) <= BLOCK_TOL
+    y_for_restore = f32(y[:M])                      # teacher-forced: the restore step on the GPU's block output
+    wx, wc = oracle.restore_from_cache(f32(x), y_for_restore, ki, pi, cuu, f32(cache_prev), h, w)
+    assert _bf16_ulp_ok(gx, wx)
+    if want_cache:
+        assert _bf16_ulp_ok(f32(cb), wc)
+
+
 # ------------------------------------------------------------------------ whole step
 def test_whole_pruned_step_config1(ctx):
     """entropy -> keep ratios -> top-k -> block on kept rows -> restore, config-1 shapes, each
@@ -848,6 +987,30 @@ def test_keep_ratios_device_against_oracle(ctx):
             fired += int((want["keep"] < N).sum())
     assert fired > 0
     assert ctx.device_status() == 0
+
+
+def test_keep_ratios_all_layers_device_against_oracle(ctx):
+    """Eq. 8-13 for all layers of a scale in one launch: row j of the keep counts equals the oracle's
+    for layer j + 1 on the means of layers 1..j + 1."""
+    B, T, L, N = 16, 10, 16, 4096
+    _, hbar = synth.scale_envelope_temperatures(B, T, seed=11)
+    hist = hbar.t().contiguous().to(DEV)
+    rng = np.random.default_rng(5)
+    layer = torch.from_numpy((hbar[:, -1:].numpy() * (1 + 0.2 * rng.standard_normal((B, L)))).astype(np.float32))
+    layer_dev = layer.t().contiguous().to(DEV)
+    keep = torch.zeros((L, B), dtype=torch.int32, device=DEV)
+    ts = torch.zeros(B, dtype=torch.int32, device=DEV)
+    act = torch.zeros(B, dtype=torch.int32, device=DEV)
+    fired = 0
+    for t in (5, 7, 8, 10):
+        nova.nova_keep_ratios_layers_device(ctx, nova.SchedParams(), t, N, hist[:t], layer_dev, keep, ts, act)
+        got = keep.cpu().numpy()
+        for j in range(1, L + 1):
+            want = oracle.keep_ratios(oracle.SchedParams(), t, j, N, hbar[:, :t].numpy().copy(), layer[:, :j].numpy().copy())
+            assert np.array_equal(got[j - 1], want["keep"]), (t, j)
+            fired += int((want["keep"] < N).sum())
+        assert np.array_equal(ts.cpu().numpy(), want["t_star"]) and np.array_equal(act.cpu().numpy(), want["act_scale"])
+    assert fired > 0
 
 
 def test_select_topk_device_counts(ctx):
