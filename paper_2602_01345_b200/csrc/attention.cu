@@ -13,9 +13,11 @@
 //   (tile B)      back into tensor memory over the S columns, from where the next MMA takes them
 //                 as its A operand. While one tile's softmax runs, the tensor core works on the
 //                 other tile.
-// The running maximum m is only raised (and O, l rescaled, in tensor memory) when the row maximum
-// grows by more than 2^8 in the exponent; until then probabilities are taken against the stale
-// maximum, which cancels in the final division by l. K tiles are K-major operands; V tiles are
+// Probabilities are taken against a reference maximum m fixed at the row's first key tile: bf16
+// and fp32 share their exponent range, so a reference that is not the running maximum costs no
+// precision, and it cancels in the final division by l. Only a score about 2^40 above the
+// reference (seen as a huge row sum) raises it, with O and l rescaled in tensor memory; the row
+// maximum is therefore not computed on the way. K tiles are K-major operands; V tiles are
 // the MN-major B operand, i.e. V is consumed exactly as it lies in the cache ([keys, dh]).
 // MMAs issued by one thread execute in issue order, which orders "P_A read by O_A += P_A V" before
 // "S_A overwritten by the next Q_A K^T" and "O complete" before the next S of the same tile.
@@ -37,7 +39,10 @@ constexpr int kThreads = 384;     // warpgroup 0: producer + MMA issuer (+2 idle
 constexpr int kRegsLow = 64, kRegsHigh = 216;
 static_assert(128 * kRegsLow + 256 * kRegsHigh <= 65536 - 2048, "keep slack for setmaxnreg.inc");
 constexpr int kSlabBytes = 128 * 128;   // [128 rows][64 bf16]
-constexpr float kRescaleThreshold = 8.f;   // in log2 units
+// A row's sum of probabilities over one key tile at or above this (or NaN) means a score about
+// 2^40 above the row's reference maximum: the reference is raised and O, l rescaled. Far below
+// anything that could overflow fp32 in l or O, far above anything ordinary data reaches.
+constexpr float kHugeSum = 1.0995116e12f;   // 2^40
 
 template <int DH>
 struct AttnSmem {
@@ -213,7 +218,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint64_t* v_full = k_empty + kKStages;            // kVStages
     uint64_t* v_empty = v_full + kVStages;            // kVStages
     uint64_t* s_full = v_empty + kVStages;            // 2 (tile A, tile B)
-    uint64_t* p_full = s_full + 2;                    // 2, 128 arrivals each
+    uint64_t* p_full = s_full + 2;                    // 2, one arrival per softmax warp
     uint64_t* o_done = p_full + 2;                    // 1
     uint32_t* tmem_slot = (uint32_t*)(o_done + 1);
     __shared__ int abort_flag_s;
@@ -235,7 +240,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&s_full[t], 1);
-            mbar_init(&p_full[t], 128);
+            mbar_init(&p_full[t], 4);
         }
         mbar_init(o_done, 1);
         fence_barrier_init();
@@ -398,7 +403,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             const uint32_t s_addr = tmem_base + lane_off + 128u * t;
             const uint32_t o_addr = tmem_base + lane_off + 256u + 128u * t;
             const float c = p.scale_log2e;
-            float m_ref = -INFINITY, l_run = 0.f;
+            // Polynomial share of the exponentials (pairs out of every four pairs of scores): the
+            // special-function unit delivers one exponential per 8 clocks and scheduler, the polynomial
+            // costs about as much in issue slots, so the two pipes share the work.
+            constexpr int kPolyPairs = (DH == 64) ? 1 : 2;
+            // The reference maximum starts at a finite floor, not -inf: (-inf) - (-inf) must not appear.
+            float m_ref = -1e30f, l_run = 0.f;
             bool ok = true;
             for (int j = 0; j < n_tiles && ok; ++j) {
                 ok = mbar_wait_warp(&s_full[t], j & 1, abort_flag, p.status);
@@ -416,69 +426,80 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     for (int i = 0; i < 128; ++i)
                         if (i >= cols_valid) sv[i] = 0xff800000u;   // -inf: key past the end
                 }
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                auto row_max = [&]() {
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int i = 0; i < 128; i += 8) {
+                    for (int i = 0; i < 128; i += 8) {
 #pragma unroll
-                    for (int a = 0; a < 4; ++a)
-                        mx4[a] = fmax3(mx4[a], __uint_as_float(sv[i + 2 * a]), __uint_as_float(sv[i + 2 * a + 1]));
-                }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                // raise the reference maximum only when it would change the exponent by > 2^8
-                const bool need = (mx - m_ref) * c > kRescaleThreshold;     // true on the first tile
-                if (__any_sync(0xffffffffu, need)) {
-                    const float m_new = fmaxf(m_ref, mx);
-                    const float alpha = ex2((m_ref - m_new) * c);             // 0 on the first tile
-                    if (j > 0) {
+                        for (int a = 0; a < 4; ++a)
+                            mx4[a] = fmax3(mx4[a], __uint_as_float(sv[i + 2 * a]), __uint_as_float(sv[i + 2 * a + 1]));
+                    }
+                    return fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                };
+                if (j == 0) m_ref = fmaxf(m_ref, row_max());      // the row's reference: its maximum over the first key tile
+                // p = 2^(s*c - m*c), 32 scores at a time: 16 registers of bf16 pairs each, written over the
+                // first columns of S as they are ready. Returns the sum of the 128 probabilities.
+                auto exponentials = [&](bool store) {
+                    const uint64_t c2 = pack_f32x2(c, c);
+                    const uint64_t nm2 = pack_f32x2(-m_ref * c, -m_ref * c);
+                    uint64_t lsum_a = pack_f32x2(0.f, 0.f), lsum_b = lsum_a;
 #pragma unroll
-                        for (int cch = 0; cch < DH / 32; ++cch) {
-                            uint32_t ov[32];
-                            tmem_ld32(o_addr + cch * 32, ov);
-                            tmem_ld_wait();
+                    for (int cch = 0; cch < 4; ++cch) {
+                        uint32_t pk[16];
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                            tmem_st32(o_addr + cch * 32, ov);
+                        for (int g = 0; g < 4; ++g) {
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int i = cch * 32 + 8 * g + 2 * q;
+                                const uint64_t y = fma_f32x2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2, nm2);
+                                float p0, p1;
+                                if (q < kPolyPairs) {
+                                    exp2_poly_x2(y, p0, p1);
+                                } else {
+                                    float y0, y1;
+                                    unpack_f32x2(y, y0, y1);
+                                    p0 = ex2(y0);
+                                    p1 = ex2(y1);
+                                }
+                                if (q & 1) lsum_b = add_f32x2(lsum_b, pack_f32x2(p0, p1));
+                                else lsum_a = add_f32x2(lsum_a, pack_f32x2(p0, p1));
+                                pk[4 * g + q] = pack_bf16(p0, p1);
+                            }
                         }
+                        if (store) tmem_st16(s_addr + cch * 16, pk);
+                    }
+                    float s0, s1, s2, s3;
+                    unpack_f32x2(lsum_a, s0, s1);
+                    unpack_f32x2(lsum_b, s2, s3);
+                    return (s0 + s2) + (s1 + s3);
+                };
+                float lsum = exponentials(true);
+                if (j > 0 && __any_sync(0xffffffffu, !(lsum < kHugeSum))) {
+                    // a score far above the reference: raise it, rescale what has been accumulated
+                    // (the tile's previous O += P V is complete: its S could not have been written
+                    // otherwise) and take the tile's probabilities again
+                    const float m_new = fmaxf(m_ref, row_max());
+                    const float alpha = ex2((m_ref - m_new) * c);
+                    tmem_st_wait();
+#pragma unroll
+                    for (int cch = 0; cch < DH / 32; ++cch) {
+                        uint32_t ov[32];
+                        tmem_ld32(o_addr + cch * 32, ov);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+                        tmem_st32(o_addr + cch * 32, ov);
                     }
                     l_run *= alpha;
                     m_ref = m_new;
+                    lsum = exponentials(true);
                 }
-                // p = 2^(s*c - m*c). Of every four scores, two go through the special-function unit
-                // and two through the polynomial, which balances the two pipes. Each 32 scores
-                // become 16 registers of bf16 pairs, written over the first columns of S.
-                const uint64_t c2 = pack_f32x2(c, c);
-                const uint64_t nm2 = pack_f32x2(-m_ref * c, -m_ref * c);
-                uint64_t lsum_a = pack_f32x2(0.f, 0.f), lsum_b = lsum_a;
-#pragma unroll
-                for (int cch = 0; cch < 4; ++cch) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        const int i = cch * 32 + 4 * g;
-                        const uint64_t ya = fma_f32x2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2, nm2);
-                        const uint64_t yb = fma_f32x2(pack_f32x2(__uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3])), c2, nm2);
-                        float ya0, ya1, p0, p1, p2, p3;
-                        unpack_f32x2(ya, ya0, ya1);
-                        p0 = ex2(ya0);
-                        p1 = ex2(ya1);
-                        exp2_poly_x2(yb, p2, p3);
-                        lsum_a = add_f32x2(lsum_a, pack_f32x2(p0, p1));
-                        lsum_b = add_f32x2(lsum_b, pack_f32x2(p2, p3));
-                        pk[2 * g] = pack_bf16(p0, p1);
-                        pk[2 * g + 1] = pack_bf16(p2, p3);
-                    }
-                    tmem_st16(s_addr + cch * 16, pk);
-                }
-                float lsum0, lsum1, lsum2, lsum3;
-                unpack_f32x2(lsum_a, lsum0, lsum1);
-                unpack_f32x2(lsum_b, lsum2, lsum3);
-                lsum0 += lsum2;
-                lsum1 += lsum3;
-                l_run += lsum0 + lsum1;
+                l_run += lsum;
                 tmem_st_wait();
                 if (t == 0 && cols_valid < BKV) {
                     // ragged last tile: rows of V past the last key may hold anything (even NaN);
-                    // zero them so that 0 * garbage cannot poison the accumulator
+                    // zero them so that 0 * garbage cannot poison the accumulator (tile A's O += P V
+                    // is issued before tile B's, so tile A's softmax warps do it for both)
                     const int s = j % kVStages;
                     ok = mbar_wait_warp(&v_full[s], (j / kVStages) & 1, abort_flag, p.status);
                     if (!ok) break;
@@ -492,7 +513,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     fence_proxy_async_smem();
                 }
                 tc_fence_before();
-                mbar_arrive(&p_full[t]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_full[t]);
             }
             if (ok) ok = mbar_wait_warp(o_done, 0, abort_flag, p.status);
             const int grow = t * BQ + row;

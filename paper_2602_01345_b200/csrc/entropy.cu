@@ -270,9 +270,11 @@ entropy_rows_ring(const LayerPtrs layers, long rows_per_layer, long rows, int V,
                   float* __restrict__ ent, float* __restrict__ mean, int seg_rows, int n_seg,
                   unsigned int* status, unsigned long long* __restrict__ accum, int fix_shift)
 {
+    // row counts fit 31 bits (checked by the launcher): 32-bit division, not the much slower 64-bit one
+    const unsigned int rpl = (unsigned int)rows_per_layer;
     auto row_ptr = [&](long row) -> const char* {
-        const long l = row / rows_per_layer;
-        return layers.p[l] + (row - l * rows_per_layer) * row_stride_bytes;
+        const unsigned int l = (unsigned int)row / rpl;
+        return layers.p[l] + (long)((unsigned int)row - l * rpl) * row_stride_bytes;
     };
     using namespace tc;
     constexpr int kRowBytes = VEC * 512;

@@ -235,13 +235,17 @@ def _step_profile(n, lo=0.25, hi=4.0, at=None):
 
 
 @pytest.mark.parametrize("C,heads", [(256, 2), (128, 2)])
-def test_attention_running_maximum_rises_across_key_tiles(ctx, C, heads):
-    """The prior keys' magnitude steps from 0.25 to 4 half way through, so each row's largest score
-    rises by roughly 9 nats (13 in log2 units) between key tiles: the stale reference maximum of the
-    streaming softmax must be raised and the accumulated output rescaled in tensor memory. 1500 prior
+@pytest.mark.parametrize("hi", [4.0, 8.0])
+def test_attention_running_maximum_rises_across_key_tiles(ctx, C, heads, hi):
+    """The prior keys' magnitude steps from 0.25 to `hi` half way through, so each row's largest
+    score rises between key tiles: by roughly 9 nats (13 in log2 units) at 4, which the streaming
+    softmax must carry against the reference maximum of the first key tile, and by 20 to 30 nats
+    (about 2^30 to 2^45) at 8, which for some rows of every warp exceeds what is carried (2^40): the
+    reference is raised and the accumulated output and row sum are rescaled in tensor memory, by
+    nearly zero for those rows and by moderate factors for the other rows of the warp. 1500 prior
     keys = 12 key tiles per item, whole items (B such that the wave is not split)."""
     attention_case(ctx, B=2, N=300, C=C, heads=heads, F=256, Lmax=2000, ks=[300, 129], kv_lens=[1500, 1500], seed=83,
-                   k_profile=_step_profile(1500), label=f"rising maximum, head size {C // heads}")
+                   k_profile=_step_profile(1500, hi=hi), label=f"rising maximum to x{hi}, head size {C // heads}")
 
 
 def test_attention_rising_maximum_in_key_split_items(ctx):
@@ -249,7 +253,7 @@ def test_attention_rising_maximum_in_key_split_items(ctx):
     magnitude step at the middle, the two halves finish with reference maxima many units apart, so
     the merge weights of the low half underflow towards zero."""
     attention_case(ctx, B=1, N=600, C=256, heads=2, F=2048, Lmax=1024, ks=[300], kv_lens=[517], seed=53,
-                   k_profile=_step_profile(517, at=384), label="rising maximum, key-split items")
+                   k_profile=_step_profile(517, at=384, hi=8.0), label="rising maximum, key-split items")
 
 
 @pytest.mark.parametrize("C,heads", [(256, 2), (128, 2)])
