@@ -246,6 +246,7 @@ entropy_rows_reg(const void* __restrict__ logits, long rows, int V, long row_str
 // order (a copy that misses the TLB can trail later ones by microseconds), so a warp must never
 // poll a slot whose previous use some other warp has yet to see.
 constexpr int kRingConsumers = 16;
+constexpr int kRingProducers = 4;
 constexpr int kRingThreads = (kRingConsumers + 1) * 32;
 constexpr int kMaxMeanSegments = NOVA_MEAN_MAX_SEGMENTS;
 constexpr int kRingBytes = 128 * 1024;
@@ -280,6 +281,7 @@ entropy_rows_ring(const LayerPtrs layers, long rows_per_layer, long rows, int V,
     constexpr int kRowBytes = VEC * 512;
     constexpr int kSlots = kRingBytes / kRowBytes;
     static_assert(kSlots % kRingConsumers == 0, "each slot must belong to one consumer warp");
+    static_assert(kSlots % kRingProducers == 0, "each slot must belong to one producer lane");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* ring = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     uint64_t* full_bar = (uint64_t*)(ring + kSlots * kRowBytes);
@@ -305,18 +307,22 @@ entropy_rows_ring(const LayerPtrs layers, long rows_per_layer, long rows, int V,
     __syncthreads();
 
     if (warp == kRingConsumers) {
-        if (lane == 0) {
-            long issued = 0;
-            for (long i = 0; i < n_my; ++i) {
+        // kRingProducers lanes issue the copies, lane p those of rows p, p + kRingProducers, ... of the
+        // CTA (slots p, p + kRingProducers, ... : kSlots is a multiple of kRingProducers). A row must
+        // be issued every ~190 clocks to keep up with HBM, and one thread's wait on the slot, its
+        // expect_tx and the copy instruction take about that long.
+        if (lane < kRingProducers) {
+            long issued = -1;          // last row index this lane issued
+            for (long i = lane; i < n_my; i += kRingProducers) {
                 const int slot = (int)(i % kSlots);
                 if (i >= kSlots && !mbar_wait(&empty_bar[slot], (uint32_t)((i / kSlots) - 1) & 1, abort_flag, status)) break;
                 const long row = blockIdx.x + i * G;
                 mbar_arrive_expect_tx(&full_bar[slot], kRowBytes);
                 bulk_load(ring + slot * kRowBytes, row_ptr(row), kRowBytes, &full_bar[slot]);
-                issued = i + 1;
+                issued = i;
             }
             if (*abort_flag)
-                for (long i = (issued > kSlots ? issued - kSlots : 0); i < issued; ++i)
+                for (long i = issued; i >= 0 && i > issued - kSlots; i -= kRingProducers)
                     mbar_drain(&full_bar[i % kSlots], (uint32_t)(i / kSlots) & 1);
         }
     } else {
