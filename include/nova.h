@@ -74,6 +74,17 @@ const char* nova_status_string(nova_status s);
  * precedence) and clears it. */
 nova_status nova_device_status(nova_ctx* ctx, void* stream);
 
+/* ---- bounded device-side waits (no counterpart in the paper) -------------------- */
+/* Every wait inside a kernel (on a copy in flight, on another warp, on the tensor core) gives up
+ * after a limit, records NOVA_ERR_TIMEOUT in the device status word and lets the kernel return, so
+ * that a lost signal can never hang the GPU. nova_set_wait_limit_ns sets that limit for the
+ * context's later launches (0 = the default, one second); it synchronises the device.
+ * nova_debug_wait_probe launches a one-block diagnostic kernel whose only warp waits for a signal
+ * that never comes: it must return after the limit with NOVA_ERR_TIMEOUT in the status word and
+ * leave the context usable. It reads and writes no caller memory. */
+nova_status nova_set_wait_limit_ns(nova_ctx* ctx, unsigned long long ns);
+nova_status nova_debug_wait_probe(nova_ctx* ctx, void* stream);
+
 /* ---- measurement (no counterpart in the paper) --------------------------------- */
 /* Kernels launched by this context since nova_create. */
 unsigned long long nova_launch_count(const nova_ctx* ctx);

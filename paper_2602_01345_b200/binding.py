@@ -190,6 +190,17 @@ class Context:
         if self._workspace is None or self._workspace.numel() < need:
             self.set_workspace(torch.empty(need + 256, dtype=torch.uint8, device=f"cuda:{self.device}"))
 
+    def set_wait_limit_ns(self, ns: int):
+        """Limit of every device-side wait of this context's later launches (0 = default, 1 s)."""
+        _lib.nova_set_wait_limit_ns.argtypes = [_vp, C.c_ulonglong]
+        with torch.cuda.device(self.device):
+            self.check(_lib.nova_set_wait_limit_ns(self.handle, int(ns)))
+
+    def debug_wait_probe(self, stream=None):
+        """Launches the diagnostic kernel whose wait can only end by running into the limit."""
+        _lib.nova_debug_wait_probe.argtypes = [_vp, _vp]
+        self.check(_lib.nova_debug_wait_probe(self.handle, _stream(stream)))
+
     def device_status(self, stream=None) -> int:
         """Synchronises the stream and returns (and clears) the device status word as a status code."""
         return int(_lib.nova_device_status(self.handle, _stream(stream)))

@@ -1,5 +1,5 @@
 // Context management and the host-side schedule arithmetic (Eq. 8-13).
-#include "common.cuh"
+#include "tc_common.cuh"
 
 #include <math.h>
 #include <new>
@@ -41,6 +41,7 @@ nova_status nova_create(nova_ctx** out, int device)
     ctx->launches = 0;
     ctx->profiling = false;
     ctx->events_used = 0;
+    ctx->wait_limit_ns = 0;
     // the allocation is made with `device` current; the caller's current device is put back
     int prev = -1;
     const bool have_prev = (cudaGetDevice(&prev) == cudaSuccess);
@@ -129,10 +130,53 @@ nova_status nova_device_status(nova_ctx* ctx, void* stream)
     NOVA_CUDA_CHECK(ctx, cudaMemcpyAsync(&word, ctx->dev_status, sizeof(word), cudaMemcpyDeviceToHost, st));
     NOVA_CUDA_CHECK(ctx, cudaStreamSynchronize(st));
     // an aborted kernel may leave the entropy accumulators or attention tickets half way: clear everything
-    if (word) NOVA_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->dev_status, 0, NOVA_STATUS_BYTES, st));
+    if (word) {
+        NOVA_CUDA_CHECK(ctx, cudaMemsetAsync(ctx->dev_status, 0, NOVA_STATUS_BYTES, st));
+        if (ctx->wait_limit_ns)     // the wait limit lives in the same block: put it back
+            NOVA_CUDA_CHECK(ctx, cudaMemcpyAsync(ctx->dev_status + NOVA_WAIT_LIMIT_WORD, &ctx->wait_limit_ns,
+                                                 sizeof(ctx->wait_limit_ns), cudaMemcpyHostToDevice, st));
+        NOVA_CUDA_CHECK(ctx, cudaStreamSynchronize(st));
+    }
     if (word & NOVA_DEV_TIMEOUT) return nova_fail(ctx, NOVA_ERR_TIMEOUT, "a device-side wait expired");
     if (word & NOVA_DEV_SHAPE) return nova_fail(ctx, NOVA_ERR_SHAPE, "K/V cache overflow on the device");
     if (word & NOVA_DEV_NONFINITE) return nova_fail(ctx, NOVA_ERR_NONFINITE, "non-finite logit");
+    return NOVA_OK;
+}
+
+nova_status nova_set_wait_limit_ns(nova_ctx* ctx, unsigned long long ns)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    NOVA_DEVICE_GUARD(ctx, "nova_set_wait_limit_ns");
+    ctx->wait_limit_ns = ns;
+    // ordered after everything enqueued so far on any stream: a synchronous copy
+    NOVA_CUDA_CHECK(ctx, cudaDeviceSynchronize());
+    NOVA_CUDA_CHECK(ctx, cudaMemcpy(ctx->dev_status + NOVA_WAIT_LIMIT_WORD, &ctx->wait_limit_ns, sizeof(ns), cudaMemcpyHostToDevice));
+    return NOVA_OK;
+}
+
+// One CTA whose consumer warp waits on a barrier that no producer ever arrives on: the wait runs
+// into the context's limit, records the time-out and the kernel returns normally.
+__global__ void wait_probe_kernel(unsigned int* status)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag_s;
+    volatile int* abort_flag = &abort_flag_s;
+    if (threadIdx.x == 0) {
+        abort_flag_s = 0;
+        tc::mbar_init(&bar, 1);
+        tc::fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) tc::mbar_wait_warp(&bar, 0, abort_flag, status);
+    __syncthreads();
+}
+
+nova_status nova_debug_wait_probe(nova_ctx* ctx, void* stream)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    NOVA_DEVICE_GUARD(ctx, "nova_debug_wait_probe");
+    wait_probe_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(ctx->dev_status);
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
     return NOVA_OK;
 }
 

@@ -20,6 +20,7 @@
 // flags, a block of tickets for key-split attention items), then one 64-bit accumulator per segment
 // for the entropy means (NOVA_MEAN_MAX_SEGMENTS of them). All of it is zero between launches.
 #define NOVA_STATUS_WORDS 128
+#define NOVA_WAIT_LIMIT_WORD 2        // words 2-3: limit of a device-side wait in ns (0 = the default of one second)
 #define NOVA_ATTN_TICKET_WORD0 16     // words 16 .. 16 + NOVA_ATTN_TICKETS - 1: tickets of key-split attention items
 #define NOVA_ATTN_TICKETS 96
 #define NOVA_MEAN_MAX_CTAS 192        // the accumulator's arrival count has 8 bits
@@ -46,6 +47,7 @@ struct nova_ctx {
     void* encode_tiled;         // cuTensorMapEncodeTiled, resolved through the runtime
     int num_sms;
     bool attr_select, attr_gemm, attr_attn;   // dynamic shared memory opt-in done on this device
+    unsigned long long wait_limit_ns;   // mirrored in the status block (0 = default)
     char err[256];
     // measurement: launches since creation, and event pairs around each launch while profiling
     unsigned long long launches;

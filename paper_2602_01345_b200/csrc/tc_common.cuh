@@ -7,7 +7,8 @@
 
 namespace tc {
 
-// A wait that has not completed after this long records NOVA_DEV_TIMEOUT and gives up.
+// A wait that has not completed after this long records NOVA_DEV_TIMEOUT and gives up: the context's
+// limit if one is set (nova_set_wait_limit_ns; kept next to the status word), else one second.
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -78,7 +79,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            unsigned long long limit = *(volatile const unsigned long long*)(status + NOVA_WAIT_LIMIT_WORD);
+            if (limit == 0) limit = kWaitLimitNs;
+            if (global_ns() - t0 > limit) {
                 *abort_flag = 1;
                 atomicOr(status, NOVA_DEV_TIMEOUT);
                 return false;

@@ -59,7 +59,7 @@ class PrunedScaleRunner:
         self.last_keep = None
 
     def run_scale(self, x_in, layer_logits, sched: nv.SchedParams, t: int, hbar_scale, append_kv: bool = True,
-                  stream=None, logits_ready=None, select_ent=None):
+                  stream=None, logits_ready=None, select_ent=None, layer_hook=None):
         """x_in [B, N, C] bf16; layer_logits: sequence of L tensors [B, N, V]; hbar_scale: CPU
         float32 [B, t] with the mean entropies of scales 1..t. Returns (x_out, keeps) where keeps
         is the list of per-layer keep-count tensors. `logits_ready`, if given, is a list of
@@ -68,6 +68,8 @@ class PrunedScaleRunner:
         on this one map (the layers' kept sets are then nested: a smaller keep count keeps a subset)
         and the layers' own logits only provide the means of Eq. 12-13; by default layer j selects
         on the entropy map of its own logits.
+        layer_hook: optional callable(stage, j, info) called with stage "before" / "after" around layer
+        j's launches (info: dict of the tensors involved); for tests that compare layer by layer.
         """
         ctx, B, N = self.ctx, self.B, self.N
         st = stream if stream is not None else torch.cuda.current_stream()
@@ -104,11 +106,18 @@ class PrunedScaleRunner:
                 shape = nv.BlockShape(B, N, self.C, self.n_heads, self.F, self.Lmax, M)
                 x_out = self.x_buf[j & 1] if x is not self.x_buf[j & 1] else self.x_buf[(j + 1) & 1]
                 cache_out = self.cache_out[j] if self.cache_out is not None else None
+                if layer_hook is not None:
+                    info = dict(x_in=x, x_out=x_out, cache_out=cache_out, keep=keep, keep_idx=keep_idx, prune_idx=prune_idx,
+                                cu_keep=cu_keep, k_cache=self.k_caches[j], v_cache=self.v_caches[j], kv_len=self.kv_len[j],
+                                cache_prev=self.cache_prev[j], ent=self.ent[j], stream=st)
+                    layer_hook("before", j, info)
                 if self.fused_restore:
                     nv.nova_pruned_layer_forward(ctx, self.weights[j], self.modulation[j] if self.modulation else None,
                                                  shape, x, keep_idx, prune_idx, cu_keep, self.k_caches[j],
                                                  self.v_caches[j], self.kv_len[j], append_kv, self.cache_prev[j],
                                                  self.h, self.w, x_out, cache_out, stream=st)
+                    if layer_hook is not None:
+                        layer_hook("after", j, info)
                     x = x_out
                     continue
                 if self.modulation is None:
@@ -122,6 +131,8 @@ class PrunedScaleRunner:
                                                        stream=st)
                 nv.nova_restore_from_cache(ctx, x, self.y_kept[:M], keep_idx, prune_idx,
                                            cu_keep, self.cache_prev[j], self.h, self.w, x_out, cache_out, stream=st)
+                if layer_hook is not None:
+                    layer_hook("after", j, info)
                 x = x_out
         self.last_keep = keeps
         return x, keeps
@@ -139,11 +150,12 @@ class MultiScaleRunner:
     """
 
     def __init__(self, ctx: nv.Context, weights, n_heads: int, B: int, scales, eps: float = 1e-6,
-                 on_device: bool = False):
+                 on_device: bool = False, fused_restore: bool = False):
         """on_device: keep the entropy history and every keep count in device memory and run each
         scale through DeviceScaleRunner (no host synchronisation inside a scale)."""
         self.ctx, self.weights, self.n_heads, self.B, self.eps = ctx, weights, n_heads, B, eps
         self.on_device = on_device
+        self.fused_restore = fused_restore
         self.scales = tuple(scales)
         self.L = len(weights)
         self.C = weights[0]["w_o"].shape[0]
@@ -157,7 +169,7 @@ class MultiScaleRunner:
         self.hist_dev = torch.zeros((len(self.scales), B), dtype=torch.float32, device=dev) if on_device else None
         self.t_done = 0
 
-    def run_scale(self, t: int, x_in, scale_logits, layer_logits, sched: nv.SchedParams, stream=None):
+    def run_scale(self, t: int, x_in, scale_logits, layer_logits, sched: nv.SchedParams, stream=None, layer_hook=None):
         """Scale t (1-based, in order). scale_logits [B, N_t, V] give the scale's mean entropy
         (Eq. 7) that extends the history; layer_logits: L tensors [B, N_t, V]. Returns
         (x_out, keeps, runner) where runner is the PrunedScaleRunner that ran the layers."""
@@ -169,7 +181,8 @@ class MultiScaleRunner:
         if self.on_device:
             runner = DeviceScaleRunner(self.ctx, self.weights, self.n_heads, B, side, side, self.Lmax, self.k_caches,
                                        self.v_caches, self.kv_len, self.res_cache, sched, t, self.hist_dev,
-                                       scale_logits.shape[-1], eps=self.eps, logits_dtype=scale_logits.dtype)
+                                       scale_logits.shape[-1], eps=self.eps, logits_dtype=scale_logits.dtype,
+                                       fused_restore=self.fused_restore)
             with torch.cuda.stream(st):
                 runner.x_in.copy_(x_in)
                 runner.scale_logits.copy_(scale_logits)
@@ -183,8 +196,10 @@ class MultiScaleRunner:
         nv.nova_scale_entropy(self.ctx, scale_logits, ent, mean, stream=st)
         self.hbar_scale = torch.cat([self.hbar_scale, mean.cpu().view(B, 1)], dim=1)
         runner = PrunedScaleRunner(self.ctx, self.weights, self.n_heads, B, side, side, self.Lmax, self.k_caches,
-                                   self.v_caches, self.kv_len, self.res_cache, eps=self.eps)
-        x_out, keeps = runner.run_scale(x_in, layer_logits, sched, t, self.hbar_scale.contiguous(), stream=st)
+                                   self.v_caches, self.kv_len, self.res_cache, eps=self.eps,
+                                   fused_restore=self.fused_restore)
+        x_out, keeps = runner.run_scale(x_in, layer_logits, sched, t, self.hbar_scale.contiguous(), stream=st,
+                                        layer_hook=layer_hook)
         self.res_cache = [c.view(B, side, side, self.C) for c in runner.cache_out]
         return x_out, keeps, runner
 

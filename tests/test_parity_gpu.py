@@ -1225,3 +1225,35 @@ def test_selection_on_one_scale_map_gives_nested_sets(ctx):
         order = sorted(range(L), key=lambda j: int(counts[j, b]))
         for lo, hi in zip(order, order[1:]):
             assert kept[lo][b] <= kept[hi][b]
+
+
+# ------------------------------------------------------------------ bounded device-side waits
+def test_device_wait_runs_into_its_limit_and_context_stays_usable():
+    """A wait that nothing will ever satisfy (a diagnostic kernel waits on a barrier without a producer)
+    ends at the context's wait limit, here 1 ms: the kernel returns, the status word says
+    NOVA_ERR_TIMEOUT, and the next ordinary call on the same context is correct. Nothing faults, traps
+    or waits without a bound."""
+    import time
+    c = nova.Context(0)
+    try:
+        c.set_wait_limit_ns(1_000_000)
+        t0 = time.perf_counter()
+        c.debug_wait_probe()
+        assert c.device_status() == 6                         # NOVA_ERR_TIMEOUT, then cleared
+        assert time.perf_counter() - t0 < 0.5                 # milliseconds, not the default second
+        assert c.device_status() == 0
+        # the limit survives the clearing of the status block: a second probe ends as quickly
+        t0 = time.perf_counter()
+        c.debug_wait_probe()
+        assert c.device_status() == 6 and time.perf_counter() - t0 < 0.5
+        # ordinary work on the same context (default limit again), through kernels that wait on barriers themselves
+        c.set_wait_limit_ns(0)
+        z = synth.randn_bf16((2, 300, 4096), 77, DEV, std=2.0)
+        ent, mean = gpu_entropy(c, z)
+        want, want_mean = oracle.scale_entropy(f32(z))
+        assert np.abs(ent.cpu().numpy() - want).max() <= ENT_TOL
+        assert np.abs(mean.cpu().numpy() - want_mean).max() <= ENT_TOL
+        _block_case(c, B=1, N=256, C=128, heads=2, F=256, Lmax=512, ks=[200], kv_lens=[100], seed=7)
+        assert c.device_status() == 0
+    finally:
+        c.close()
