@@ -56,8 +56,8 @@ def _generation(cfg, B, seed, spatial, fused, value_scales, value_layers, n_rows
         side = ms.scales[t - 1]
         N = side * side
         x_in = synth.activations(B, N, C, 200 * seed + t, DEV)
-        if spatial:
-            # a seeded smooth field per scale, scaled so that its mean follows the image's envelope
+        if spatial and side >= 3:
+            # a seeded smooth field per scale (from 3 x 3 tokens up), scaled by the image's envelope
             field = synth.smooth_temperature_field(B, side, side, seed * 31 + t, a_lo=0.6, a_hi=1.4, device=DEV)
             a = field * a_env[:, t - 1].view(B, 1).to(DEV)
         else:
