@@ -75,6 +75,9 @@ def parse_args():
     ap.add_argument("--two-call-layers", action="store_true",
                     help="time nova_pruned_block_forward + nova_restore_from_cache per layer instead of the one "
                          "nova_pruned_layer_forward call (the other form is timed after the timed region either way)")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="one JSON line per stated configuration (the five workloads; the 1024 shape at keep ratios "
+                         "0.25 / 0.5 / 0.75 and batch 1 / 4), device-resident timing only")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-next", action="store_true",
@@ -242,6 +245,7 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    torch.cuda.reset_peak_memory_stats()
     for _ in range(args.warmup):
         one_step()
     barrier()
@@ -263,6 +267,9 @@ def run_ours(args):
     launches = pipeline.launch_count(ctx) - launches0
     clk = clocks.stop()
     total_ms = max_over_ranks(total_ms, dist, dev)
+    # device memory in use at its peak up to here: weights, K/V and residual caches, logits, activations
+    # and the library's workspace (a torch tensor), i.e. everything the step needs resident
+    peak_hbm_bytes = int(torch.cuda.max_memory_allocated())
     ms_per_step = total_ms / args.steps
     value = replica_throughput(world, B, ms_per_step)
     status = ctx.device_status()
@@ -425,7 +432,7 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": config_json(wd, world), "clocks": clk, "gpu_launches": int(launches),
-        "tokens_per_s": round(world * B * N / (ms_per_step / 1e3), 1),
+        "tokens_per_s": round(world * B * N / (ms_per_step / 1e3), 1), "peak_hbm_bytes": peak_hbm_bytes,
         "roofline": roofline, "roofline_second": other_roofline, "kernels": kernels,
         "layer_call_forms": layer_forms,
         "next_head_entropy": head_entropy, "next_device_schedule": device_schedule,
@@ -436,10 +443,30 @@ def run_ours(args):
         out["e2e"] = run_e2e(args, wd, st, runner, sched, hbar_scale, barrier, dist, dev, world)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wd, st, keeps)
-    if rank == 0:
-        print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
+    return out if rank == 0 else None
+
+
+ALL_CONFIGS = (
+    [("c1_single_step", None, 0.5), ("c2_var_d16_256", None, 0.5), ("c3_var_d30_512", None, 0.5)] +
+    [("c4_1024", b, k) for b in (1, 4) for k in (0.25, 0.5, 0.75)] + [("c5_2048", None, 0.2)])
+
+
+def run_all_configs(args):
+    """The stated configurations one after the other in this process, device-resident timing only."""
+    import copy
+    import gc
+    for wl, batch, keep in ALL_CONFIGS:
+        a = copy.copy(args)
+        a.workload, a.batch, a.keep = wl, batch, keep
+        a.no_e2e = a.no_cpu_baseline = True
+        out = run_ours(a)
+        if out is not None:
+            print(json.dumps(out), flush=True)
+        del out
+        gc.collect()
+        torch.cuda.empty_cache()
 
 
 def run_e2e(args, wd, st, runner, sched, hbar_scale, barrier, dist, dev, world):
@@ -614,5 +641,9 @@ if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.all_configs:
+        run_all_configs(a)
     else:
-        run_ours(a)
+        res = run_ours(a)
+        if res is not None:
+            print(json.dumps(res))

@@ -227,3 +227,32 @@ def restore_from_cache(x_in, y_kept, keep_idx, prune_idx, cu_keep, cache_prev, h
     _load().oracle_restore_from_cache(_p(x), _p(y), _p(ki), _p(pi), _p(cu), _p(cp),
                                       hp, wp, h, w, C, B, _p(x_out), _p(cache_out))
     return x_out, cache_out
+
+
+def score_mse(x, ref_prev, h: int, w: int):
+    """MSE selection score (reading of the paper's selection-metric ablation): mean squared distance
+    between a token and the bilinear resize of the previous scale's map to its position.
+    x [B, h*w, C], ref_prev [B, hp, wp, C] -> score [B, h*w] f32."""
+    xx, rr = _f32(x), _f32(ref_prev)
+    B, N, C = xx.shape
+    assert N == h * w and rr.shape[0] == B and rr.shape[3] == C
+    score = np.empty((B, N), np.float32)
+    _load().oracle_score_mse(_p(xx), _p(rr), B, rr.shape[1], rr.shape[2], h, w, C, _p(score))
+    return score
+
+
+def score_attention_mass(q, k, k_cache, kv_len, n_heads: int):
+    """Attention-mass selection score: the share of the scale's attention (all N tokens as queries,
+    keys = prior cache rows followed by the N tokens' own keys) that lands on each token's key,
+    averaged over heads and queries. q, k [B, N, C]; k_cache [B, Lmax, C] or None; kv_len [B] or None
+    -> score [B, N] f32."""
+    qq, kk = _f32(q), _f32(k)
+    B, N, C = qq.shape
+    kc = _f32(k_cache) if k_cache is not None else None
+    kl = _i32(kv_len) if kv_len is not None else np.zeros(B, np.int32)
+    Lmax = kc.shape[1] if kc is not None else 0
+    assert kc is not None or (kl == 0).all()
+    score = np.empty((B, N), np.float32)
+    _load().oracle_score_attention_mass(_p(qq), _p(kk), _p(kc) if kc is not None else None, _p(kl), B, N, C, n_heads,
+                                        Lmax, _p(score))
+    return score

@@ -476,6 +476,98 @@ void oracle_restore_from_cache(const float* x_in, const float* y_kept,
     }
 }
 
+// ---------------------------------------------------------------------------
+// Alternative selection scores of the paper's selection-metric ablation (the table comparing
+// entropy with an attention-based and an MSE-based criterion). The paper names the two criteria
+// and says only that the MSE one stands for the magnitude of the frequency signal; the definitions
+// below are this build's readings. Both give one score per token, and the tokens with the highest
+// scores are kept by the same top-k rule as for the entropy.
+//
+// MSE score: how far a token's representation is from what the previous, coarser scale predicts
+// for its position, i.e. the energy of the detail the coarser scale cannot carry:
+//   score[b, i] = (1/C) sum_c ( x[b, i, c] - U(ref_prev)[b, i, c] )^2
+// with U the bilinear resize of Eq. 16 (half-pixel centres, edge clamp) from (hp, wp) to (h, w).
+// ---------------------------------------------------------------------------
+void oracle_score_mse(const float* x, const float* ref_prev, int B, int hp, int wp, int h, int w, int C,
+                      float* score)
+{
+    const int N = h * w;
+    for (int b = 0; b < B; ++b) {
+#pragma omp parallel for schedule(static)
+        for (int i = 0; i < N; ++i) {
+            const int oy = i / w, ox = i % w;
+            double sy = ((double)oy + 0.5) * ((double)hp / (double)h) - 0.5;
+            double sx = ((double)ox + 0.5) * ((double)wp / (double)w) - 0.5;
+            if (sy < 0.0) sy = 0.0;
+            if (sx < 0.0) sx = 0.0;
+            int y0 = (int)std::floor(sy), x0 = (int)std::floor(sx);
+            if (y0 > hp - 1) y0 = hp - 1;
+            if (x0 > wp - 1) x0 = wp - 1;
+            const int y1 = std::min(y0 + 1, hp - 1), x1 = std::min(x0 + 1, wp - 1);
+            const double fy = sy - (double)y0, fx = sx - (double)x0;
+            const float* c00 = ref_prev + (((long)b * hp + y0) * wp + x0) * C;
+            const float* c01 = ref_prev + (((long)b * hp + y0) * wp + x1) * C;
+            const float* c10 = ref_prev + (((long)b * hp + y1) * wp + x0) * C;
+            const float* c11 = ref_prev + (((long)b * hp + y1) * wp + x1) * C;
+            const float* xr = x + ((long)b * N + i) * C;
+            double acc = 0.0;
+            for (int c = 0; c < C; ++c) {
+                const double top = (1.0 - fx) * (double)c00[c] + fx * (double)c01[c];
+                const double bot = (1.0 - fx) * (double)c10[c] + fx * (double)c11[c];
+                const double d = (double)xr[c] - ((1.0 - fy) * top + fy * bot);
+                acc += d * d;
+            }
+            score[(long)b * N + i] = (float)(acc / (double)C);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Attention-mass score: the share of the scale's attention that lands on a token's key. With the
+// scale's N tokens as queries (q) and, as keys, the kv_len[b] prior-scale keys of the cache followed
+// by the N tokens' own keys (k), all tokens present (nothing pruned yet), per head
+//   P_h = softmax_rows( q_h K_h^T / sqrt(dh) ),        K_h = [cache rows ; k]_h
+//   score[b, j] = (1 / (n_heads * N)) sum_h sum_q P_h[q, kv_len[b] + j]
+// so the scores of an image sum to at most 1 (exactly 1 without prior keys).
+// q, k [B, N, C]; k_cache [B, Lmax, C] (may be NULL when every kv_len is 0); score [B, N].
+// ---------------------------------------------------------------------------
+void oracle_score_attention_mass(const float* q, const float* k, const float* k_cache, const int32_t* kv_len,
+                                 int B, int N, int C, int n_heads, int Lmax, float* score)
+{
+    const int dh = C / n_heads;
+    for (int b = 0; b < B; ++b) {
+        const int n_old = kv_len ? kv_len[b] : 0;
+        const int n_keys = n_old + N;
+        std::vector<double> mass((size_t)N, 0.0);
+#pragma omp parallel
+        {
+            std::vector<double> local((size_t)N, 0.0), sc((size_t)n_keys);
+#pragma omp for schedule(static) collapse(2)
+            for (int hd = 0; hd < n_heads; ++hd) {
+                for (int qi = 0; qi < N; ++qi) {
+                    const int c0 = hd * dh;
+                    const float* qr = q + ((long)b * N + qi) * C + c0;
+                    double smax = -INFINITY;
+                    for (int jx = 0; jx < n_keys; ++jx) {
+                        const float* kr = (jx < n_old) ? k_cache + ((long)b * Lmax + jx) * C + c0
+                                                       : k + ((long)b * N + (jx - n_old)) * C + c0;
+                        double acc = 0.0;
+                        for (int d = 0; d < dh; ++d) acc += (double)qr[d] * (double)kr[d];
+                        sc[jx] = acc / std::sqrt((double)dh);
+                        smax = std::max(smax, sc[jx]);
+                    }
+                    double denom = 0.0;
+                    for (int jx = 0; jx < n_keys; ++jx) { sc[jx] = std::exp(sc[jx] - smax); denom += sc[jx]; }
+                    for (int j = 0; j < N; ++j) local[j] += sc[n_old + j] / denom;
+                }
+            }
+#pragma omp critical
+            for (int j = 0; j < N; ++j) mass[j] += local[j];
+        }
+        for (int j = 0; j < N; ++j) score[(long)b * N + j] = (float)(mass[j] / ((double)n_heads * (double)N));
+    }
+}
+
 int oracle_num_threads(void)
 {
     int n = 1;

@@ -638,3 +638,65 @@ def test_whole_step_keep_all_reproduces_dense_layer():
         wy, _, _ = _torch_block(w, 1e-6, 2, x[b], kc[b, :kv_len[b]], vc[b, :kv_len[b]])
         assert np.allclose(x_out[b], wy, atol=2e-5, rtol=1e-5)
         assert np.allclose(cache_out[b], wy - x[b], atol=3e-5)
+
+
+# ------------------------------------------------------------------ alternative selection scores
+def test_score_mse_pins():
+    """Closed forms and a library composition: same-size reference -> plain mean squared difference;
+    constant reference -> mean (x - const)^2; torch's bilinear interpolation (fp64) for a real resize;
+    a token equal to the resized reference scores 0."""
+    import torch.nn.functional as F
+    rng = np.random.default_rng(0)
+    B, h, w, C = 2, 6, 9, 16
+    x = rng.standard_normal((B, h * w, C)).astype(np.float32)
+    same = rng.standard_normal((B, h, w, C)).astype(np.float32)
+    got = oracle.score_mse(x, same, h, w)
+    assert np.allclose(got, ((x - same.reshape(B, h * w, C)).astype(np.float64) ** 2).mean(-1), rtol=1e-6)
+    const = np.full((B, 3, 4, C), 0.75, np.float32)
+    assert np.allclose(oracle.score_mse(x, const, h, w), ((x.astype(np.float64) - 0.75) ** 2).mean(-1), rtol=1e-6)
+    ref = rng.standard_normal((B, 4, 5, C)).astype(np.float32)
+    up = F.interpolate(torch.from_numpy(ref).double().permute(0, 3, 1, 2), size=(h, w), mode="bilinear",
+                       align_corners=False).permute(0, 2, 3, 1).reshape(B, h * w, C).numpy()
+    assert np.allclose(oracle.score_mse(x, ref, h, w), ((x - up) ** 2).mean(-1), rtol=1e-5)
+    assert np.abs(oracle.score_mse(up.astype(np.float32), ref, h, w)).max() < 1e-12
+    # a token moved away from the prediction scores higher: the criterion ranks by detail energy
+    x2 = up.astype(np.float32).copy()
+    x2[0, 7] += 0.5
+    s = oracle.score_mse(x2, ref, h, w)
+    assert s[0].argmax() == 7 and abs(s[0, 7] - 0.25) < 1e-6
+
+
+def test_score_attention_mass_pins():
+    """Zero queries -> every key gets 1 / (prior + N) of every row; the scores of an image sum to the
+    share of attention that stays inside the scale (1 without prior keys); a key every query is
+    aligned with collects almost everything; torch softmax (fp64) on random inputs with ragged prior
+    lengths; per-head layout (head h uses channels [h*dh, (h+1)*dh))."""
+    rng = np.random.default_rng(1)
+    B, N, heads, dh, Lmax = 2, 12, 3, 8, 20
+    C = heads * dh
+    q = rng.standard_normal((B, N, C)).astype(np.float32)
+    k = rng.standard_normal((B, N, C)).astype(np.float32)
+    kc = rng.standard_normal((B, Lmax, C)).astype(np.float32)
+    lens = np.array([7, 0], np.int32)
+    got = oracle.score_attention_mass(np.zeros_like(q), k, kc, lens, heads)
+    assert np.allclose(got[0], 1.0 / (7 + N)) and np.allclose(got[1], 1.0 / N)
+    got = oracle.score_attention_mass(q, k, kc, lens, heads)
+    want = np.zeros((B, N))
+    for b in range(B):
+        keys = np.concatenate([kc[b, :lens[b]], k[b]], 0).astype(np.float64)
+        for hd in range(heads):
+            sl = slice(hd * dh, (hd + 1) * dh)
+            p = torch.softmax(torch.from_numpy(q[b, :, sl].astype(np.float64) @ keys[:, sl].T / np.sqrt(dh)), dim=-1).numpy()
+            want[b] += p[:, lens[b]:].sum(0)
+    want /= heads * N
+    assert np.allclose(got, want, rtol=1e-6, atol=1e-9)
+    assert abs(got[1].sum() - 1.0) < 1e-6 and got[0].sum() < 1.0
+    # one key aligned with every query in every head
+    q2 = np.tile(rng.standard_normal((1, 1, C)).astype(np.float32), (1, N, 1)) * 3
+    k2 = 0.01 * rng.standard_normal((1, N, C)).astype(np.float32)
+    k2[0, 5] = q2[0, 0] * 3
+    s = oracle.score_attention_mass(q2, k2, None, None, heads)
+    assert s[0].argmax() == 5 and s[0, 5] > 0.99
+    # swapping two heads' channel blocks in q and k alike leaves the scores unchanged
+    perm = np.r_[np.arange(dh, 2 * dh), np.arange(0, dh), np.arange(2 * dh, C)]
+    assert np.allclose(oracle.score_attention_mass(q[..., perm], k[..., perm], kc[..., perm], lens, heads), got, rtol=1e-6)
