@@ -218,6 +218,32 @@ nova_status nova_select_topk_grouped_device(nova_ctx* ctx, const float* ent, int
                                             const int32_t* k_dev, int32_t* keep_idx, int32_t* prune_idx,
                                             int32_t* cu_keep, int32_t* pos, void* stream);
 
+/* ---- alternative selection scores (the paper's selection-metric ablation) ------------------ */
+/*
+ * The ablation table on token selection metrics compares the entropy with an attention-based and an
+ * MSE-based criterion; the paper names them and says only that the MSE one stands for the magnitude
+ * of the frequency signal. The two calls below are this library's readings; each writes one score
+ * per token, and nova_select_topk keeps the highest scores exactly as it does for entropies.
+ *
+ * nova_score_mse: score[b, i] = (1/C) sum_c (x[b, i, c] - U(ref_prev)[b, i, c])^2, U the bilinear
+ *   resize of Eq. 16 (half-pixel centres, edge clamp) from (hp, wp) to (h, w): the energy of the
+ *   detail that the previous scale's map cannot carry. x device bf16 [B, h*w, C]; ref_prev device bf16
+ *   [B, hp, wp, C]; score device f32 [B, h*w]. C a multiple of 8.
+ * nova_score_attention_mass: with the scale's N tokens as queries and, as keys, the kv_len[b] rows of
+ *   k_cache followed by the N tokens' own keys (all tokens, nothing pruned), per head
+ *   P = softmax_rows(q K^T / sqrt(dh)); score[b, j] = (1 / (n_heads * N)) sum_heads sum_queries
+ *   P[query, kv_len[b] + j]: the share of the scale's attention that lands on token j's key.
+ *   q, k device bf16 [B, N, C]; k_cache device bf16 [B, Lmax, C] and kv_len device int32 [B], or both
+ *   NULL (no prior keys); lse_scratch device f32 [B, n_heads, N] (scratch); score device f32 [B, N].
+ *   Head size 64 or 128. Sums run in a fixed order: results are reproducible bit for bit.
+ * Errors: bad sizes -> INVALID_ARG / SHAPE; misaligned pointers -> ALIGNMENT. Empty inputs are no-ops.
+ */
+nova_status nova_score_mse(nova_ctx* ctx, const void* x, const void* ref_prev, int B, int hp, int wp,
+                           int h, int w, int C, float* score, void* stream);
+nova_status nova_score_attention_mass(nova_ctx* ctx, const void* q, const void* k, const void* k_cache,
+                                      const int32_t* kv_len, int B, int N, int C, int n_heads, int Lmax,
+                                      float* lse_scratch, float* score, void* stream);
+
 /* ---- Eq. 14: the layer on the kept tokens -------------------------------------- */
 typedef struct nova_block_weights {  /* device bf16; matrices are [out, in] row-major */
     const void *ln1_g, *ln1_b;       /* [C]            */

@@ -209,6 +209,60 @@ def pruned_block_forward(weights: dict, eps: float, n_heads: int, x_in, keep_idx
     return y, k_new, v_new
 
 
+EXT_NAMES = ("rope_cos", "rope_sin", "qk_gain_q", "qk_gain_k", "lnc_g", "lnc_b", "w_q2", "b_q2", "w_o2", "b_o2", "ck", "cv")
+
+
+class _BlockExt(ctypes.Structure):
+    _fields_ = [("rope_cos", ctypes.c_void_p), ("rope_sin", ctypes.c_void_p), ("qk_gain_q", ctypes.c_void_p),
+                ("qk_gain_k", ctypes.c_void_p), ("qk_eps", ctypes.c_float)] + \
+               [(n, ctypes.c_void_p) for n in ("lnc_g", "lnc_b", "w_q2", "b_q2", "w_o2", "b_o2", "ck", "cv", "cond_len")] + \
+               [("Lc_max", ctypes.c_int)]
+
+
+def pruned_block_forward_ext(weights: dict, eps: float, n_heads: int, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len,
+                             ext: dict, rows=None, modulation=None, qk_eps: float = 1e-12):
+    """pruned_block_forward with the optional parts of the text-conditioned backbones. ext maps names
+    from EXT_NAMES to arrays (missing = absent): rope_cos / rope_sin [N, dh/2]; qk_gain_q / qk_gain_k [C];
+    lnc_g, lnc_b [C], w_q2, w_o2 [C, C], b_q2, b_o2 [C], ck, cv [B, Lc_max, C] together with
+    ext["cond_len"] int32 [B] for the cross-attention. Returns (y, k_new, v_new); k_new holds the
+    transformed keys."""
+    x = _f32(x_in)
+    B, N, C = x.shape
+    w = {n: _f32(weights[n]) for n in WEIGHT_NAMES}
+    F = w["w_fc1"].shape[0]
+    ki, cu = _i32(keep_idx), _i32(cu_keep)
+    M = int(cu[B])
+    kc, vc = _f32(k_cache), _f32(v_cache)
+    Lmax = kc.shape[1]
+    kl = _i32(kv_len)
+    rr = _i32(rows) if rows is not None else None
+    R = len(rr) if rr is not None else M
+    y = np.empty((R, C), np.float32)
+    k_new = np.empty((M, C), np.float32)
+    v_new = np.empty((M, C), np.float32)
+    cw = _BlockWeights(*[_p(w[n]) for n in WEIGHT_NAMES], eps)
+    e = {n: _f32(ext[n]) for n in EXT_NAMES if ext.get(n) is not None}
+    dh = C // n_heads
+    if "rope_cos" in e:
+        assert e["rope_cos"].shape == (N, dh // 2) and e["rope_sin"].shape == (N, dh // 2)
+    cl = _i32(ext["cond_len"]) if ext.get("cond_len") is not None else None
+    Lc = e["ck"].shape[1] if "ck" in e else 0
+    if "w_q2" in e:
+        assert cl is not None and e["ck"].shape == (B, Lc, C) and e["cv"].shape == (B, Lc, C)
+    g = lambda n: _p(e[n]) if n in e else None
+    ce = _BlockExt(g("rope_cos"), g("rope_sin"), g("qk_gain_q"), g("qk_gain_k"), qk_eps, g("lnc_g"), g("lnc_b"),
+                   g("w_q2"), g("b_q2"), g("w_o2"), g("b_o2"), g("ck"), g("cv"), _p(cl) if cl is not None else None, Lc)
+    cm = None
+    md = {}
+    if modulation is not None:
+        md = {n: _f32(modulation[n]) for n in MODULATION_NAMES if modulation.get(n) is not None}
+        cm = _BlockModulation(*[_p(md[n]) if n in md else None for n in MODULATION_NAMES])
+    _load().oracle_pruned_block_forward_ext(
+        ctypes.byref(cw), ctypes.byref(cm) if cm is not None else None, ctypes.byref(ce), B, N, C, n_heads, F, Lmax,
+        _p(x), _p(ki), _p(cu), _p(kc), _p(vc), _p(kl), _p(rr), R, _p(y), _p(k_new), _p(v_new))
+    return y, k_new, v_new
+
+
 def restore_from_cache(x_in, y_kept, keep_idx, prune_idx, cu_keep, cache_prev, h, w,
                        want_cache=True):
     """Eq. 15-16. x_in [B, h*w, C]; y_kept [M, C]; cache_prev [B, hp, wp, C].

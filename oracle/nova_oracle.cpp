@@ -308,7 +308,30 @@ static void modulate_row(float* h, const float* scale, const float* shift, int b
     }
 }
 
-void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle_block_modulation* mod,
+// Block variants of the text-conditioned backbones the paper accelerates (the Infinity models use
+// rotary position embedding, query/key normalisation and cross-attention to the text tokens; the
+// paper itself names only the layer's parts). Every group is optional (NULL pointers = absent):
+//  * QK normalisation: per head, q and k are scaled to unit L2 norm, x / max(||x||, qk_eps), and
+//    multiplied by a per-channel gain (qk_gain_q / qk_gain_k, [C]); applied first.
+//  * Rotary embedding: within every head, channel pairs (2i, 2i+1) of q and k are rotated by the
+//    angle whose cosine and sine are rope_cos / rope_sin [N, dh/2] at the token's index in the scale:
+//    (a, b) -> (a cos - b sin, a sin + b cos). Cached keys of earlier scales were rotated when they
+//    were appended; the keys returned in k_new are the transformed ones.
+//  * Cross-attention after the self-attention residual: q2 = LN(x1; lnc) W_q2^T + b_q2 attends (per
+//    head, softmax(q2 K^T / sqrt(dh)) V, no mask) to the cond_len[b] rows of the image's condition
+//    keys / values ck, cv [B, Lc_max, C]; x1 <- x1 + o2 W_o2^T + b_o2. No normalisation or rotation there.
+struct oracle_block_ext {
+    const float *rope_cos, *rope_sin;
+    const float *qk_gain_q, *qk_gain_k;
+    float qk_eps;
+    const float *lnc_g, *lnc_b, *w_q2, *b_q2, *w_o2, *b_o2;
+    const float *ck, *cv;
+    const int32_t* cond_len;
+    int Lc_max;
+};
+
+void oracle_pruned_block_forward_ext(const oracle_block_weights* w, const oracle_block_modulation* mod,
+                                     const oracle_block_ext* ext,
                                      int B, int N, int C, int n_heads, int F, int Lmax,
                                      const float* x_in, const int32_t* keep_idx,
                                      const int32_t* cu_keep,
@@ -316,6 +339,42 @@ void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle
                                      const int32_t* kv_len,
                                      const int32_t* rows, int n_rows,
                                      float* y, float* k_new, float* v_new);
+
+void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle_block_modulation* mod,
+                                     int B, int N, int C, int n_heads, int F, int Lmax,
+                                     const float* x_in, const int32_t* keep_idx,
+                                     const int32_t* cu_keep,
+                                     const float* k_cache, const float* v_cache,
+                                     const int32_t* kv_len,
+                                     const int32_t* rows, int n_rows,
+                                     float* y, float* k_new, float* v_new)
+{
+    oracle_pruned_block_forward_ext(w, mod, nullptr, B, N, C, n_heads, F, Lmax, x_in, keep_idx, cu_keep, k_cache,
+                                    v_cache, kv_len, rows, n_rows, y, k_new, v_new);
+}
+
+// q or k of one token, all heads, in place: QK normalisation, then the rotation for position `pos`
+static void qk_transform_row(float* v, const float* gain, float eps, const float* rope_cos, const float* rope_sin,
+                             int pos, int n_heads, int dh)
+{
+    for (int hd = 0; hd < n_heads; ++hd) {
+        float* h = v + hd * dh;
+        if (gain) {
+            double ss = 0.0;
+            for (int d = 0; d < dh; ++d) ss += (double)h[d] * (double)h[d];
+            const double nrm = std::max(std::sqrt(ss), (double)eps);
+            for (int d = 0; d < dh; ++d) h[d] = (float)((double)h[d] / nrm * (double)gain[hd * dh + d]);
+        }
+        if (rope_cos) {
+            for (int i = 0; i < dh / 2; ++i) {
+                const double c = rope_cos[(long)pos * (dh / 2) + i], sn = rope_sin[(long)pos * (dh / 2) + i];
+                const double a = h[2 * i], b = h[2 * i + 1];
+                h[2 * i] = (float)(a * c - b * sn);
+                h[2 * i + 1] = (float)(a * sn + b * c);
+            }
+        }
+    }
+}
 
 void oracle_pruned_block_forward(const oracle_block_weights* w,
                                  int B, int N, int C, int n_heads, int F, int Lmax,
@@ -330,7 +389,8 @@ void oracle_pruned_block_forward(const oracle_block_weights* w,
                                     v_cache, kv_len, rows, n_rows, y, k_new, v_new);
 }
 
-void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle_block_modulation* mod,
+void oracle_pruned_block_forward_ext(const oracle_block_weights* w, const oracle_block_modulation* mod,
+                                 const oracle_block_ext* ext,
                                  int B, int N, int C, int n_heads, int F, int Lmax,
                                  const float* x_in, const int32_t* keep_idx,
                                  const int32_t* cu_keep,
@@ -357,6 +417,8 @@ void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle
                    k_new + (long)m * C);
         linear_row(&h1[(size_t)m * C], w->w_qkv + 2L * C * C, w->b_qkv + 2 * C, C, C,
                    v_new + (long)m * C);
+        if (ext) qk_transform_row(k_new + (long)m * C, ext->qk_gain_k, ext->qk_eps, ext->rope_cos, ext->rope_sin,
+                                  keep_idx[m], n_heads, dh);
     }
 
     const int R = rows ? n_rows : M;
@@ -367,6 +429,8 @@ void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle
         const float* x = x_in + ((long)b * N + keep_idx[m]) * C;
         std::vector<float> q(C), o(C), x1(C), h2(C), f1(F), f2(C);
         linear_row(&h1[(size_t)m * C], w->w_qkv, w->b_qkv, C, C, q.data());
+        if (ext) qk_transform_row(q.data(), ext->qk_gain_q, ext->qk_eps, ext->rope_cos, ext->rope_sin, keep_idx[m],
+                                  n_heads, dh);
 
         // attention over [cache rows 0..kv_len[b]) ++ [kept rows of image b]
         const int n_old = kv_len[b];
@@ -403,6 +467,36 @@ void oracle_pruned_block_forward_mod(const oracle_block_weights* w, const oracle
         for (int c = 0; c < C; ++c) {
             const double g1 = (mod && mod->gate1) ? (double)mod->gate1[(long)b * C + c] : 1.0;
             x1[c] = (float)((double)x[c] + g1 * (double)x1[c]);
+        }
+
+        if (ext && ext->w_q2) {
+            // cross-attention to the image's condition tokens
+            std::vector<float> hc(C), q2(C), o2(C), xo(C);
+            layer_norm_row(x1.data(), ext->lnc_g, ext->lnc_b, w->eps, C, hc.data());
+            linear_row(hc.data(), ext->w_q2, ext->b_q2, C, C, q2.data());
+            const int n_c = ext->cond_len[b];
+            std::vector<double> sc2(std::max(n_c, 1));
+            for (int hd = 0; hd < n_heads; ++hd) {
+                const int c0 = hd * dh;
+                double smax = -INFINITY;
+                for (int jx = 0; jx < n_c; ++jx) {
+                    const float* kr = ext->ck + ((long)b * ext->Lc_max + jx) * C + c0;
+                    double acc = 0.0;
+                    for (int d = 0; d < dh; ++d) acc += (double)q2[c0 + d] * (double)kr[d];
+                    sc2[jx] = acc / std::sqrt((double)dh);
+                    smax = std::max(smax, sc2[jx]);
+                }
+                double denom = 0.0;
+                for (int jx = 0; jx < n_c; ++jx) { sc2[jx] = std::exp(sc2[jx] - smax); denom += sc2[jx]; }
+                for (int d = 0; d < dh; ++d) {
+                    double acc = 0.0;
+                    for (int jx = 0; jx < n_c; ++jx)
+                        acc += (sc2[jx] / denom) * (double)ext->cv[((long)b * ext->Lc_max + jx) * C + c0 + d];
+                    o2[c0 + d] = (float)acc;       // no condition tokens: the branch adds only its bias
+                }
+            }
+            linear_row(o2.data(), ext->w_o2, ext->b_o2, C, C, xo.data());
+            for (int c = 0; c < C; ++c) x1[c] = (float)((double)x1[c] + (double)xo[c]);
         }
 
         layer_norm_row(x1.data(), w->ln2_g, w->ln2_b, w->eps, C, h2.data());

@@ -518,3 +518,32 @@ def nova_pruned_layer_forward(ctx: Context, w: BlockWeights, modulation, shape: 
         ctx.handle, C.byref(w.c), C.byref(cm) if modulation else None, C.byref(c), _ptr(x_in), _ptr(keep_idx),
         _ptr(prune_idx), _ptr(cu_keep), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len), int(bool(append_kv)),
         _ptr(cache_prev), hp, wp, h, w_tokens, _ptr(x_out), _ptr(cache_out), int(bool(m_on_device)), _stream(stream)))
+
+
+# ---- alternative selection scores ------------------------------------------------------------------
+_lib.nova_score_mse.argtypes = [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.nova_score_mse.restype = _i
+_lib.nova_score_attention_mass.argtypes = [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp]
+_lib.nova_score_attention_mass.restype = _i
+
+
+def nova_score_mse(ctx: Context, x, ref_prev, h, w, score, stream=None):
+    """x [B, h*w, C] bf16, ref_prev [B, hp, wp, C] bf16 -> score [B, h*w] f32: mean squared distance to
+    the bilinear resize of the previous scale's map."""
+    B, N, Cc = x.shape
+    assert N == h * w and ref_prev.shape[0] == B and ref_prev.shape[3] == Cc
+    assert x.dtype == torch.bfloat16 and ref_prev.dtype == torch.bfloat16 and score.dtype == torch.float32
+    ctx.check(_lib.nova_score_mse(ctx.handle, _ptr(x), _ptr(ref_prev), B, ref_prev.shape[1], ref_prev.shape[2], h, w,
+                                  Cc, _ptr(score), _stream(stream)))
+
+
+def nova_score_attention_mass(ctx: Context, q, k, k_cache, kv_len, n_heads, score, stream=None):
+    """q, k [B, N, C] bf16; k_cache [B, Lmax, C] bf16 and kv_len int32 [B] (device) or None, None ->
+    score [B, N] f32: share of the scale's attention landing on each token's key."""
+    B, N, Cc = q.shape
+    assert k.shape == q.shape and q.dtype == torch.bfloat16 and k.dtype == torch.bfloat16
+    assert score.dtype == torch.float32 and score.numel() == B * N
+    Lmax = k_cache.shape[1] if k_cache is not None else 0
+    lse = torch.empty((B, n_heads, N), dtype=torch.float32, device=q.device)
+    ctx.check(_lib.nova_score_attention_mass(ctx.handle, _ptr(q), _ptr(k), _ptr(k_cache), _ptr(kv_len), B, N, Cc,
+                                             n_heads, Lmax, _ptr(lse), _ptr(score), _stream(stream)))

@@ -89,7 +89,7 @@ const char* nova_profile_category_name(int cat)
 {
     static const char* names[NOVA_K_COUNT] = {
         "entropy_rows", "entropy_mean", "select_topk", "layernorm", "gemm_qkv",
-        "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "restore", "keep_ratios"};
+        "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "restore", "keep_ratios", "selection_score"};
     return (cat >= 0 && cat < NOVA_K_COUNT) ? names[cat] : "?";
 }
 

@@ -31,7 +31,7 @@
 enum nova_kernel_cat {
     NOVA_K_ENTROPY = 0, NOVA_K_ENTROPY_MEAN, NOVA_K_SELECT, NOVA_K_LAYERNORM,
     NOVA_K_GEMM_QKV, NOVA_K_ATTENTION, NOVA_K_GEMM_PROJ, NOVA_K_GEMM_FC1, NOVA_K_GEMM_FC2,
-    NOVA_K_RESTORE, NOVA_K_KEEP_RATIOS, NOVA_K_COUNT
+    NOVA_K_RESTORE, NOVA_K_KEEP_RATIOS, NOVA_K_SCORE, NOVA_K_COUNT
 };
 
 struct nova_prof_rec {

@@ -700,3 +700,149 @@ def test_score_attention_mass_pins():
     # swapping two heads' channel blocks in q and k alike leaves the scores unchanged
     perm = np.r_[np.arange(dh, 2 * dh), np.arange(0, dh), np.arange(2 * dh, C)]
     assert np.allclose(oracle.score_attention_mass(q[..., perm], k[..., perm], kc[..., perm], lens, heads), got, rtol=1e-6)
+
+
+# ------------------------------------------------- block variants: rotary embedding, QK norm, cross-attention
+def _ext_case(rng, B=2, N=10, heads=2, dh=8, F=24, Lmax=14, Lc=5):
+    C = heads * dh
+    names = {"ln1_g": (C,), "ln1_b": (C,), "w_qkv": (3 * C, C), "b_qkv": (3 * C,), "w_o": (C, C), "b_o": (C,),
+             "ln2_g": (C,), "ln2_b": (C,), "w_fc1": (F, C), "b_fc1": (F,), "w_fc2": (C, F), "b_fc2": (C,)}
+    w = {n: (0.3 * rng.standard_normal(sh)).astype(np.float32) for n, sh in names.items()}
+    w["ln1_g"] += 1
+    w["ln2_g"] += 1
+    x = rng.standard_normal((B, N, C)).astype(np.float32)
+    kc = rng.standard_normal((B, Lmax, C)).astype(np.float32)
+    vc = rng.standard_normal((B, Lmax, C)).astype(np.float32)
+    lens = np.array([4, 0], np.int32)[:B]
+    keep = [np.sort(rng.choice(N, size=k, replace=False)).astype(np.int32) for k in (7, 3)[:B]]
+    keep_idx = np.concatenate(keep)
+    cu = np.r_[0, np.cumsum([len(k) for k in keep])].astype(np.int32)
+    ang = rng.uniform(0, 2 * np.pi, (N, dh // 2))
+    ext = dict(rope_cos=np.cos(ang).astype(np.float32), rope_sin=np.sin(ang).astype(np.float32),
+               qk_gain_q=(1 + 0.2 * rng.standard_normal(C)).astype(np.float32),
+               qk_gain_k=(1 + 0.2 * rng.standard_normal(C)).astype(np.float32),
+               lnc_g=(1 + 0.1 * rng.standard_normal(C)).astype(np.float32), lnc_b=(0.1 * rng.standard_normal(C)).astype(np.float32),
+               w_q2=(0.3 * rng.standard_normal((C, C))).astype(np.float32), b_q2=(0.1 * rng.standard_normal(C)).astype(np.float32),
+               w_o2=(0.3 * rng.standard_normal((C, C))).astype(np.float32), b_o2=(0.1 * rng.standard_normal(C)).astype(np.float32),
+               ck=rng.standard_normal((B, Lc, C)).astype(np.float32), cv=rng.standard_normal((B, Lc, C)).astype(np.float32),
+               cond_len=np.array([Lc, 2], np.int32)[:B])
+    return dict(w=w, x=x, kc=kc, vc=vc, lens=lens, keep_idx=keep_idx, cu=cu, heads=heads, dh=dh, C=C, F=F, ext=ext, N=N, B=B)
+
+
+def _ext_torch(c, ext):
+    """The extended block as a composition of torch library ops in float64 (independent of the
+    oracle's loops): F.layer_norm, F.linear, F.normalize, complex multiplication for the rotation,
+    F.scaled_dot_product_attention, F.gelu(tanh)."""
+    import torch.nn.functional as Fn
+    t = lambda a: torch.from_numpy(np.asarray(a)).double()
+    w = {n: t(v) for n, v in c["w"].items()}
+    heads, dh, C, B = c["heads"], c["dh"], c["C"], c["B"]
+    ys, ks = [], []
+
+    def transform(v, gain, pos):                       # v [n, C]
+        v = v.view(-1, heads, dh)
+        if gain is not None:
+            v = Fn.normalize(v, dim=-1, eps=1e-12) * t(gain).view(heads, dh)
+        if ext.get("rope_cos") is not None:
+            rot = torch.complex(t(ext["rope_cos"])[pos], t(ext["rope_sin"])[pos]).unsqueeze(1)        # [n, 1, dh/2]
+            v = torch.view_as_real(torch.view_as_complex(v.reshape(-1, heads, dh // 2, 2).contiguous()) * rot).reshape(-1, heads, dh)
+        return v.reshape(-1, C)
+
+    for b in range(B):
+        idx = c["keep_idx"][c["cu"][b]:c["cu"][b + 1]]
+        xb = t(c["x"][b, idx])
+        h = Fn.layer_norm(xb, (C,), w["ln1_g"], w["ln1_b"], 1e-6)
+        qkv = Fn.linear(h, w["w_qkv"], w["b_qkv"])
+        q, k, v = qkv[:, :C], qkv[:, C:2 * C], qkv[:, 2 * C:]
+        q = transform(q.contiguous(), ext.get("qk_gain_q"), idx)
+        k = transform(k.contiguous(), ext.get("qk_gain_k"), idx)
+        n0 = c["lens"][b]
+        K = torch.cat([t(c["kc"][b, :n0]), k], 0).view(-1, heads, dh).transpose(0, 1)
+        V = torch.cat([t(c["vc"][b, :n0]), v], 0).view(-1, heads, dh).transpose(0, 1)
+        o = Fn.scaled_dot_product_attention(q.view(-1, heads, dh).transpose(0, 1), K, V).transpose(0, 1).reshape(-1, C)
+        x1 = xb + Fn.linear(o, w["w_o"], w["b_o"])
+        if ext.get("w_q2") is not None:
+            hc = Fn.layer_norm(x1, (C,), t(ext["lnc_g"]), t(ext["lnc_b"]), 1e-6)
+            q2 = Fn.linear(hc, t(ext["w_q2"]), t(ext["b_q2"])).view(-1, heads, dh).transpose(0, 1)
+            n_c = int(ext["cond_len"][b])
+            Kc = t(ext["ck"][b, :n_c]).view(-1, heads, dh).transpose(0, 1)
+            Vc = t(ext["cv"][b, :n_c]).view(-1, heads, dh).transpose(0, 1)
+            o2 = Fn.scaled_dot_product_attention(q2, Kc, Vc).transpose(0, 1).reshape(-1, C)
+            x1 = x1 + Fn.linear(o2, t(ext["w_o2"]), t(ext["b_o2"]))
+        h2 = Fn.layer_norm(x1, (C,), w["ln2_g"], w["ln2_b"], 1e-6)
+        ys.append(x1 + Fn.linear(Fn.gelu(Fn.linear(h2, w["w_fc1"], w["b_fc1"]), approximate="tanh"), w["w_fc2"], w["b_fc2"]))
+        ks.append(k)
+    return torch.cat(ys).numpy(), torch.cat(ks).numpy()
+
+
+def _run_ext(c, ext, **kw):
+    return oracle.pruned_block_forward_ext(c["w"], 1e-6, c["heads"], c["x"], c["keep_idx"], c["cu"], c["kc"], c["vc"],
+                                           c["lens"], ext, **kw)
+
+
+def test_block_ext_matches_library_composition():
+    rng = np.random.default_rng(5)
+    c = _ext_case(rng)
+    full = c["ext"]
+    subsets = [full,
+               {k: full[k] for k in ("rope_cos", "rope_sin")},
+               {k: full[k] for k in ("qk_gain_q", "qk_gain_k")},
+               {k: full[k] for k in ("lnc_g", "lnc_b", "w_q2", "b_q2", "w_o2", "b_o2", "ck", "cv", "cond_len")}]
+    for ext in subsets:
+        y, k_new, _ = _run_ext(c, ext)
+        wy, wk = _ext_torch(c, ext)
+        assert np.abs(y - wy).max() < 2e-5 and np.abs(k_new - wk).max() < 2e-5
+
+
+def test_block_ext_reductions_and_invariants():
+    rng = np.random.default_rng(6)
+    c = _ext_case(rng)
+    full = c["ext"]
+    plain, k_plain, _ = oracle.pruned_block_forward(c["w"], 1e-6, c["heads"], c["x"], c["keep_idx"], c["cu"], c["kc"],
+                                                    c["vc"], c["lens"])
+    # nothing switched on, and the identity rotation: the plain block, bit for bit
+    y, k_new, _ = _run_ext(c, {})
+    assert np.array_equal(y, plain) and np.array_equal(k_new, k_plain)
+    ident = dict(rope_cos=np.ones_like(full["rope_cos"]), rope_sin=np.zeros_like(full["rope_sin"]))
+    assert np.array_equal(_run_ext(c, ident)[0], plain)
+    # rotation: with no prior keys, turning every position by the same extra angle changes nothing
+    # (scores depend on angle differences only), while the rotated keys themselves do change
+    c0 = dict(c, lens=np.zeros_like(c["lens"]))
+    ang = np.arctan2(full["rope_sin"], full["rope_cos"])
+    a = dict(rope_cos=np.cos(ang).astype(np.float32), rope_sin=np.sin(ang).astype(np.float32))
+    b = dict(rope_cos=np.cos(ang + 0.7).astype(np.float32), rope_sin=np.sin(ang + 0.7).astype(np.float32))
+    ya, ka, _ = _run_ext(c0, a)
+    yb, kb, _ = _run_ext(c0, b)
+    assert np.abs(ya - yb).max() < 1e-5 and np.abs(ka - kb).max() > 0.1
+    assert np.abs(ya - _run_ext(c0, {})[0]).max() > 1e-3                 # and the rotation does act
+    # QK normalisation: the scale of a head's query projection no longer matters
+    qk = {k: full[k] for k in ("qk_gain_q", "qk_gain_k")}
+    w2 = dict(c["w"])
+    w2["w_qkv"] = c["w"]["w_qkv"].copy()
+    w2["b_qkv"] = c["w"]["b_qkv"].copy()
+    w2["w_qkv"][: c["dh"]] *= 3.0
+    w2["b_qkv"][: c["dh"]] *= 3.0
+    y1 = _run_ext(c, qk)[0]
+    y2 = _run_ext(dict(c, w=w2), qk)[0]
+    assert np.abs(y1 - y2).max() < 1e-5
+    assert np.abs(_run_ext(dict(c, w=w2), {})[0] - plain).max() > 1e-3   # without it, it does
+    # unit keys: every transformed key head has norm |gain| when the gain is constant
+    g1 = dict(qk_gain_q=np.full(c["C"], 2.0, np.float32), qk_gain_k=np.full(c["C"], 0.5, np.float32))
+    kn = _run_ext(c, g1)[1].reshape(-1, c["heads"], c["dh"])
+    assert np.allclose(np.linalg.norm(kn, axis=-1), 0.5, atol=1e-6)
+    # cross-attention: a zero output projection leaves the plain block; one condition token adds
+    # exactly its projected value row to the residual stream before the MLP
+    cross = {k: full[k] for k in ("lnc_g", "lnc_b", "w_q2", "b_q2", "w_o2", "b_o2", "ck", "cv", "cond_len")}
+    z = dict(cross, w_o2=np.zeros_like(cross["w_o2"]), b_o2=np.zeros_like(cross["b_o2"]))
+    assert np.array_equal(_run_ext(c, z)[0], plain)
+    one = dict(cross, cond_len=np.ones(c["B"], np.int32))
+    wz = dict(c["w"], w_fc2=np.zeros_like(c["w"]["w_fc2"]), b_fc2=np.zeros_like(c["w"]["b_fc2"]))   # y = x1
+    y_one = _run_ext(dict(c, w=wz), one)[0]
+    y_base = oracle.pruned_block_forward(wz, 1e-6, c["heads"], c["x"], c["keep_idx"], c["cu"], c["kc"], c["vc"], c["lens"])[0]
+    for b_ in range(c["B"]):
+        add = cross["w_o2"].astype(np.float64) @ cross["cv"][b_, 0].astype(np.float64) + cross["b_o2"]
+        rows = slice(c["cu"][b_], c["cu"][b_ + 1])
+        assert np.abs((y_one[rows] - y_base[rows]) - add).max() < 1e-5
+    # row subsets evaluate to the same rows
+    sub = np.array([0, 3, 8], np.int32)
+    assert np.array_equal(_run_ext(c, full, rows=sub)[0], _run_ext(c, full)[0][sub])

@@ -1227,6 +1227,82 @@ def test_selection_on_one_scale_map_gives_nested_sets(ctx):
             assert kept[lo][b] <= kept[hi][b]
 
 
+# ------------------------------------------------------------------ alternative selection scores
+SCORE_TOL = 2e-3          # relative to the largest score: fp32 sums of products of exact bf16 inputs
+
+
+@pytest.mark.parametrize("B,hp,wp,h,w,C", [(2, 13, 13, 16, 16, 1024), (3, 5, 7, 9, 11, 64), (1, 4, 4, 4, 4, 256),
+                                            (4, 48, 48, 64, 64, 2048)])
+def test_score_mse_matches_oracle_and_selects_like_it(ctx, B, hp, wp, h, w, C):
+    """The MSE selection score against the oracle on every token, and the selection it drives: the
+    oracle's top-k on the GPU's scores equals the GPU's index lists."""
+    N = h * w
+    ref = synth.residual_cache(B, hp, wp, C, seed=2, device=DEV)
+    x = synth.activations(B, N, C, seed=1, device=DEV)
+    score = torch.full((B, N), float("nan"), dtype=torch.float32, device=DEV)
+    nova.nova_score_mse(ctx, x, ref, h, w, score)
+    want = oracle.score_mse(f32(x), f32(ref), h, w)
+    got = score.cpu().numpy()
+    assert np.abs(got - want).max() <= SCORE_TOL * np.abs(want).max()
+    ks = [N // 2] * B
+    keep_idx, prune_idx, cu, _ = gpu_select(ctx, score, ks)
+    w_keep, w_prune, w_cu, _ = oracle.select_topk(got, ks)
+    assert np.array_equal(keep_idx.cpu().numpy(), w_keep) and np.array_equal(prune_idx.cpu().numpy(), w_prune)
+    assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("B,N,C,heads,Lmax,kv_lens", [
+    (2, 100, 128, 2, 300, [0, 217]),          # head size 64, ragged tiles, one image without prior keys
+    (2, 256, 256, 2, 680, [424, 424]),        # head size 128, prior keys of the 256 configuration
+    (1, 77, 192, 3, 64, None),                # no cache at all
+    (2, 1024, 1920, 30, 2240, [1216, 1216]),  # the 512 configuration's last scale
+])
+def test_score_attention_mass_matches_oracle(ctx, B, N, C, heads, Lmax, kv_lens):
+    """The attention-mass selection score against the oracle on every token (queries scaled up so that
+    the rows are peaked and the masses differ by orders of magnitude), reproducible bit for bit, and
+    the selection it drives equal to the oracle's on the same scores."""
+    q = (synth.activations(B, N, C, 11, DEV).float() * 1.5).to(torch.bfloat16)
+    k = synth.activations(B, N, C, 12, DEV)
+    if kv_lens is None:
+        k_cache = kv_len = None
+    else:
+        k_cache, _, _ = synth.kv_cache(B, Lmax, max(kv_lens), C, 13, DEV)
+        for b, n in enumerate(kv_lens):
+            k_cache[b, n:] = float("nan")                 # rows past the length are never read
+        kv_len = torch.tensor(kv_lens, dtype=torch.int32, device=DEV)
+    score = torch.full((B, N), float("nan"), dtype=torch.float32, device=DEV)
+    nova.nova_score_attention_mass(ctx, q, k, k_cache, kv_len, heads, score)
+    want = oracle.score_attention_mass(f32(q), f32(k), None if k_cache is None else np.nan_to_num(f32(k_cache)),
+                                       None if kv_lens is None else np.array(kv_lens, np.int32), heads)
+    got = score.cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= SCORE_TOL * np.abs(want).max()
+    assert want.max() - want.min() > 20 * SCORE_TOL * want.max()     # the spread between tokens is far above the tolerance
+    if kv_lens is None or min(kv_lens) == 0:
+        b0 = 0
+        assert abs(float(got[b0].sum()) - 1.0) < 1e-3      # without prior keys all attention stays in the scale
+    score2 = torch.empty_like(score)
+    nova.nova_score_attention_mass(ctx, q, k, k_cache, kv_len, heads, score2)
+    assert torch.equal(score, score2)
+    ks = [N // 4] * B
+    keep_idx, prune_idx, cu, _ = gpu_select(ctx, score, ks)
+    w_keep, w_prune, _, _ = oracle.select_topk(got, ks)
+    assert np.array_equal(keep_idx.cpu().numpy(), w_keep) and np.array_equal(prune_idx.cpu().numpy(), w_prune)
+    assert ctx.device_status() == 0
+
+
+def test_score_bad_args(ctx):
+    x = synth.activations(1, 16, 64, 1, DEV)
+    s = torch.empty((1, 16), dtype=torch.float32, device=DEV)
+    with pytest.raises(nova.NovaError) as ei:             # head size 32
+        nova.nova_score_attention_mass(ctx, x, x, None, None, 2, s)
+    assert ei.value.status == 2
+    x2 = synth.activations(1, 16, 60, 1, DEV)
+    with pytest.raises(nova.NovaError) as ei:             # C not a multiple of 8
+        nova.nova_score_mse(ctx, x2, x2.view(1, 4, 4, 60), 4, 4, s)
+    assert ei.value.status == 2
+
+
 # ------------------------------------------------------------------ bounded device-side waits
 def test_device_wait_runs_into_its_limit_and_context_stays_usable():
     """A wait that nothing will ever satisfy (a diagnostic kernel waits on a barrier without a producer)
