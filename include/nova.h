@@ -321,6 +321,41 @@ nova_status nova_pruned_block_forward_adaln(nova_ctx* ctx, const nova_block_weig
                                             void* k_cache, void* v_cache, int32_t* kv_len,
                                             int append_kv, void* y_kept, int m_on_device, void* stream);
 
+/* ---- Eq. 14 with the parts of the text-conditioned backbones ------------------------------ */
+/*
+ * The text-to-image backbones the paper accelerates (Infinity) differ from the plain block in three
+ * places; the paper names only the layer's parts, so the forms below are the backbones' published
+ * ones. Each group is optional (NULL pointers = absent):
+ *  - QK normalisation: per head, q and k are scaled to unit L2 norm, x / max(||x||, qk_eps), and
+ *    multiplied by a per-channel gain; qk_gain_q, qk_gain_k device bf16 [C] (both or neither).
+ *  - Rotary embedding, after the normalisation: within every head the channel pairs (2i, 2i+1) of
+ *    q and k are rotated, (a, b) -> (a cos - b sin, a sin + b cos), cos and sin taken from rope_cos,
+ *    rope_sin (device f32 [N, dh/2], both or neither) at the token's index in the scale, so the
+ *    caller decides the position scheme (1-D, axial 2-D, ...). Keys enter the cache transformed.
+ *  - Cross-attention after the self-attention residual: q2 = LN(x1; lnc_g, lnc_b) W_q2^T + b_q2
+ *    attends, per head and without mask, to the cond_len[b] rows of the image's condition keys and
+ *    values cond_k, cond_v (device bf16 [B, Lc_max, C], already projected by the caller);
+ *    x1 <- x1 + o2 W_o2^T + b_o2. An image with cond_len 0 receives only b_o2.
+ * mod (adaptive LayerNorm) and m_on_device as in nova_pruned_block_forward_adaln; everything else as
+ * nova_pruned_block_forward. Errors: half-given groups -> INVALID_ARG; misaligned pointers -> ALIGNMENT.
+ */
+typedef struct nova_block_extras {
+    const float *rope_cos, *rope_sin;
+    const void *qk_gain_q, *qk_gain_k;
+    float qk_eps;
+    const void *lnc_g, *lnc_b, *w_q2, *b_q2, *w_o2, *b_o2;
+    const void *cond_k, *cond_v;
+    const int32_t* cond_len;
+    int Lc_max;
+} nova_block_extras;
+
+nova_status nova_pruned_block_forward_ext(nova_ctx* ctx, const nova_block_weights* w,
+                                          const nova_block_modulation* mod, const nova_block_extras* ext,
+                                          const nova_block_shape* s, const void* x_in,
+                                          const int32_t* keep_idx, const int32_t* cu_keep,
+                                          void* k_cache, void* v_cache, int32_t* kv_len,
+                                          int append_kv, void* y_kept, int m_on_device, void* stream);
+
 /* ---- the same block for callers that cannot allocate device memory ------------------ */
 /*
  * (The paper has no counterpart to this call; it exists for deployment.)

@@ -11,6 +11,6 @@ from .binding import (  # noqa: F401
     nova_pruned_block_forward_static, nova_static_scratch_bytes,
     nova_keep_ratios_device, nova_select_topk_device, nova_pruned_block_forward_device,
     nova_restore_from_cache_device, nova_pruned_block_forward_adaln, MODULATION_NAMES,
-    nova_pruned_layer_forward, nova_score_mse, nova_score_attention_mass, nova_scale_entropy_layers, nova_keep_ratios_layers, nova_select_topk_grouped, nova_keep_ratios_layers_device,
+    nova_pruned_layer_forward, nova_pruned_block_forward_ext, EXTRA_NAMES, nova_score_mse, nova_score_attention_mass, nova_scale_entropy_layers, nova_keep_ratios_layers, nova_select_topk_grouped, nova_keep_ratios_layers_device,
     lib_path, STATUS_NAMES,
 )

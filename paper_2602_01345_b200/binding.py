@@ -547,3 +547,47 @@ def nova_score_attention_mass(ctx: Context, q, k, k_cache, kv_len, n_heads, scor
     lse = torch.empty((B, n_heads, N), dtype=torch.float32, device=q.device)
     ctx.check(_lib.nova_score_attention_mass(ctx.handle, _ptr(q), _ptr(k), _ptr(k_cache), _ptr(kv_len), B, N, Cc,
                                              n_heads, Lmax, _ptr(lse), _ptr(score), _stream(stream)))
+
+
+# ---- block with rotary embedding, QK normalisation, cross-attention ----------------------------------
+EXTRA_NAMES = ("rope_cos", "rope_sin", "qk_gain_q", "qk_gain_k", "lnc_g", "lnc_b", "w_q2", "b_q2", "w_o2", "b_o2",
+               "cond_k", "cond_v", "cond_len")
+
+
+class _BlockExtras(C.Structure):
+    _fields_ = [("rope_cos", _vp), ("rope_sin", _vp), ("qk_gain_q", _vp), ("qk_gain_k", _vp), ("qk_eps", C.c_float)] + \
+               [(n, _vp) for n in ("lnc_g", "lnc_b", "w_q2", "b_q2", "w_o2", "b_o2", "cond_k", "cond_v", "cond_len")] + \
+               [("Lc_max", _i)]
+
+
+_lib.nova_pruned_block_forward_ext.argtypes = [_vp, C.POINTER(_BlockWeights), C.POINTER(_BlockModulation),
+                                               C.POINTER(_BlockExtras), C.POINTER(_BlockShape), _vp, _vp, _vp, _vp, _vp,
+                                               _vp, _i, _vp, _i, _vp]
+_lib.nova_pruned_block_forward_ext.restype = _i
+
+
+def nova_pruned_block_forward_ext(ctx: Context, w: BlockWeights, modulation, extras: dict, shape: BlockShape, x_in,
+                                  keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept,
+                                  m_on_device: bool = False, qk_eps: float = 1e-12, stream=None):
+    """nova_pruned_block_forward with the optional parts of the text-conditioned backbones. extras maps
+    names from EXTRA_NAMES to device tensors (missing or None = absent): rope_cos / rope_sin f32 [N, dh/2];
+    qk_gain_q / qk_gain_k bf16 [C]; lnc_g, lnc_b, b_q2, b_o2 bf16 [C], w_q2, w_o2 bf16 [C, C], cond_k / cond_v
+    bf16 [B, Lc_max, C], cond_len int32 [B] for the cross-attention."""
+    e = {n: (extras.get(n) if extras else None) for n in EXTRA_NAMES}
+    dh = shape.C // shape.n_heads
+    for n in ("rope_cos", "rope_sin"):
+        assert e[n] is None or (e[n].dtype == torch.float32 and e[n].shape == (shape.N, dh // 2))
+    Lc = e["cond_k"].shape[1] if e["cond_k"] is not None else 0
+    ce = _BlockExtras(_ptr(e["rope_cos"]), _ptr(e["rope_sin"]), _ptr(e["qk_gain_q"]), _ptr(e["qk_gain_k"]), qk_eps,
+                      *[_ptr(e[n]) for n in ("lnc_g", "lnc_b", "w_q2", "b_q2", "w_o2", "b_o2", "cond_k", "cond_v", "cond_len")],
+                      Lc)
+    ptrs = []
+    for n in MODULATION_NAMES:
+        t = modulation.get(n) if modulation else None
+        ptrs.append(_ptr(t))
+    cm = _BlockModulation(*ptrs)
+    c = shape._c()
+    ctx.check(_lib.nova_pruned_block_forward_ext(
+        ctx.handle, C.byref(w.c), C.byref(cm) if modulation else None, C.byref(ce), C.byref(c), _ptr(x_in), _ptr(keep_idx),
+        _ptr(cu_keep), _ptr(k_cache), _ptr(v_cache), _ptr(kv_len), int(bool(append_kv)), _ptr(y_kept),
+        int(bool(m_on_device)), _stream(stream)))

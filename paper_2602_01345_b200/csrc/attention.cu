@@ -65,6 +65,7 @@ struct AttnParams {
     const int32_t* kv_len;
     __nv_bfloat16* o;
     int B, C, Lmax, n_heads, num_sms;
+    int own_keys;          // 1: keys = cache rows followed by this call's k_b rows; 0: cache rows only (cross-attention)
     float scale_log2e;     // (1 / sqrt(dh)) * log2(e)
     // key-split of a last partial wave: per split item two partial results [2][256 rows][DH + 4]
     // fp32 (unnormalised O row, reference maximum, sum) and a ticket counter; part == NULL: no split
@@ -198,11 +199,19 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     }
     const int rows_valid = min(2 * BQ, k_b - slot * 2 * BQ);
     const bool tile_b_active = rows_valid > BQ;
-    const int n_keys = min(p.kv_len[b] + k_b, p.Lmax);
+    const int n_keys = min(max(p.kv_len[b], 0) + (p.own_keys ? k_b : 0), p.Lmax);
     const int n_tiles_all = (n_keys + BKV - 1) / BKV;
     if (khalf >= 0 && n_tiles_all < 4) {      // too few key tiles to share: the first CTA takes them all
         if (khalf == 1) return;
         khalf = -1;
+    }
+    if (n_keys == 0) {
+        // nothing to attend to (cross-attention with no condition tokens): the output rows are zero
+        for (int i = threadIdx.x; i < rows_valid * (DH / 8); i += kThreads) {
+            const int r = i / (DH / 8), v = i - r * (DH / 8);
+            *(uint4*)(p.o + (long)(q_begin + r) * p.C + head * DH + v * 8) = make_uint4(0, 0, 0, 0);
+        }
+        return;
     }
     // this CTA's key tiles are jt0 .. jt0 + n_tiles - 1; loops below count j from 0
     int jt0 = 0, n_tiles = n_tiles_all;
@@ -642,6 +651,7 @@ nova_status launch(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st)
     p.scale_log2e = (float)((1.0 / sqrt((double)DH)) * 1.4426950408889634);
     p.status = ctx->dev_status;
     p.n_heads = a.n_heads; p.num_sms = ctx->num_sms;
+    p.own_keys = a.cache_only ? 0 : 1;
     // scratch for a key-split last wave: [slots][2][256][DH + 4] fp32; tickets live in the context's
     // status allocation (zero at creation, reset by the CTA that draws the second ticket)
     const size_t slot_bytes = (size_t)2 * 2 * BQ * (DH + 4) * sizeof(float);

@@ -152,6 +152,63 @@ layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, con
     }
 }
 
+// ---- query/key normalisation and rotary embedding -----------------------------------------------
+// After the QKV projection, per kept row r and head: q (in the q buffer) and the row's new key (in
+// its cache row) are, in place, scaled to unit L2 norm times a per-channel gain, then rotated pair by
+// pair by the angle of the token's position in the scale. One warp per (row, head); a lane holds DH / 32
+// consecutive channels, i.e. whole pairs.
+template <int DH>
+__global__ void __launch_bounds__(256)
+qk_transform_kernel(__nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k_cache, const int32_t* __restrict__ kv_row,
+                    const int32_t* __restrict__ keep_idx, int M, const int32_t* __restrict__ m_dev, int C, int n_heads,
+                    const __nv_bfloat16* __restrict__ gain_q, const __nv_bfloat16* __restrict__ gain_k, float eps,
+                    const float* __restrict__ rope_cos, const float* __restrict__ rope_sin)
+{
+    constexpr int PER = DH / 32;          // 2 or 4 channels per lane
+    const int lane = threadIdx.x & 31;
+    const long wid = (long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (m_dev) M = min(M, *m_dev);
+    if (wid >= (long)M * n_heads) return;
+    const int r = (int)(wid / n_heads), hd = (int)(wid - (long)r * n_heads);
+    const int pos = keep_idx[r];
+    const int ch = hd * DH + lane * PER;
+    float cs[PER / 2], sn[PER / 2];
+    if (rope_cos) {
+#pragma unroll
+        for (int i = 0; i < PER / 2; ++i) {
+            cs[i] = rope_cos[(long)pos * (DH / 2) + lane * (PER / 2) + i];
+            sn[i] = rope_sin[(long)pos * (DH / 2) + lane * (PER / 2) + i];
+        }
+    }
+    auto transform = [&](__nv_bfloat16* row, const __nv_bfloat16* gain) {
+        float v[PER];
+#pragma unroll
+        for (int i = 0; i < PER; ++i) v[i] = __bfloat162float(row[ch + i]);
+        if (gain) {
+            float ss = 0.f;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) ss = fmaf(v[i], v[i], ss);
+            ss = warp_sum(ss);
+            const float inv = 1.f / fmaxf(sqrtf(ss), eps);
+#pragma unroll
+            for (int i = 0; i < PER; ++i) v[i] = v[i] * inv * __bfloat162float(gain[ch + i]);
+        }
+        if (rope_cos) {
+#pragma unroll
+            for (int i = 0; i < PER / 2; ++i) {
+                const float a = v[2 * i], b = v[2 * i + 1];
+                v[2 * i] = a * cs[i] - b * sn[i];
+                v[2 * i + 1] = a * sn[i] + b * cs[i];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < PER; ++i) row[ch + i] = __float2bfloat16_rn(v[i]);
+    };
+    transform(q + (long)r * C, gain_q);
+    const int kr = kv_row[r];
+    if (kr >= 0) transform(k_cache + (long)kr * C, gain_k);      // a row of an overflowing image has no cache row
+}
+
 struct Workspace {
     int32_t* src_row;
     int32_t* kv_row;
@@ -246,7 +303,7 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
                                  const int32_t* keep_idx, const int32_t* cu_keep,
                                  void* k_cache, void* v_cache, int32_t* kv_len,
                                  int append_kv, void* y_kept, void* stream, bool m_on_device,
-                                 const ScatterOut* scatter = nullptr)
+                                 const ScatterOut* scatter = nullptr, const nova_block_extras* ext = nullptr)
 {
     if (!ctx) return NOVA_ERR_INVALID_ARG;
     if (!w || !s) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward: null weights or shape");
@@ -265,6 +322,23 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
     Workspace ws = carve(ctx->workspace, s->M, s->C, s->F);
     if (!ctx->workspace || ctx->workspace_bytes < ws.bytes)
         return nova_fail(ctx, NOVA_ERR_WORKSPACE, "nova_pruned_block_forward: workspace missing or too small");
+    const bool rope = ext && (ext->rope_cos || ext->rope_sin);
+    const bool qk_norm = ext && (ext->qk_gain_q || ext->qk_gain_k);
+    const bool cross = ext && ext->w_q2;
+    if (rope && (!ext->rope_cos || !ext->rope_sin)) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward_ext: rope_cos and rope_sin go together");
+    if (qk_norm && (!ext->qk_gain_q || !ext->qk_gain_k)) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward_ext: qk_gain_q and qk_gain_k go together");
+    if (cross) {
+        const void* cp[] = {ext->lnc_g, ext->lnc_b, ext->w_q2, ext->b_q2, ext->w_o2, ext->b_o2, ext->cond_k, ext->cond_v, ext->cond_len};
+        for (const void* ptr : cp)
+            if (!ptr) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward_ext: incomplete cross-attention weights");
+        if (ext->Lc_max < 1) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_block_forward_ext: Lc_max < 1");
+    }
+    if (ext) {
+        const void* ep[] = {ext->rope_cos, ext->rope_sin, ext->qk_gain_q, ext->qk_gain_k, ext->lnc_g, ext->lnc_b, ext->w_q2,
+                            ext->b_q2, ext->w_o2, ext->b_o2, ext->cond_k, ext->cond_v};
+        for (const void* ptr : ep)
+            if (!nova_aligned16(ptr)) return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_pruned_block_forward_ext: tensor not 16-byte aligned");
+    }
     NOVA_DEVICE_GUARD(ctx, "nova_pruned_block_forward");
 
     cudaStream_t st = (cudaStream_t)stream;
@@ -295,6 +369,22 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
     g.epilogue = NOVA_EPI_QKV; g.cat = NOVA_K_GEMM_QKV; g.out = ws.q; g.C = C; g.k_cache = (bf)k_cache; g.v_cache = (bf)v_cache; g.kv_row = ws.kv_row;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
+    if (rope || qk_norm) {
+        // q and the new keys, in place: unit norm times gain, then the rotation of the token's position
+        const long warps = (long)M * s->n_heads;
+        const unsigned blocks = (unsigned)((warps + 7) / 8);
+        typedef const float* cfl;
+        nova_launch_scope scope(ctx, NOVA_K_LAYERNORM, st);
+        if (C / s->n_heads == 64)
+            qk_transform_kernel<64><<<blocks, 256, 0, st>>>(ws.q, (bf)k_cache, ws.kv_row, keep_idx, M, m_dev, C, s->n_heads,
+                                                          (cbf)ext->qk_gain_q, (cbf)ext->qk_gain_k, ext->qk_eps,
+                                                          (cfl)ext->rope_cos, (cfl)ext->rope_sin);
+        else
+            qk_transform_kernel<128><<<blocks, 256, 0, st>>>(ws.q, (bf)k_cache, ws.kv_row, keep_idx, M, m_dev, C, s->n_heads,
+                                                           (cbf)ext->qk_gain_q, (cbf)ext->qk_gain_k, ext->qk_eps,
+                                                           (cfl)ext->rope_cos, (cfl)ext->rope_sin);
+        NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    }
     // o = softmax(q K^T / sqrt(dh)) V
     nova_attn_args a;
     a.q = ws.q; a.k_cache = (cbf)k_cache; a.v_cache = (cbf)v_cache; a.cu_keep = cu_keep; a.kv_len = kv_len;
@@ -303,6 +393,7 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
     // next to each other: together they hold the partial results of a key-split last wave
     a.scratch = ws.x1;
     a.scratch_bytes = (size_t)((char*)ws.f - (char*)ws.x1) + (size_t)((M + 127) / 128) * 128 * (size_t)F * 2;
+    a.cache_only = false;
     rc = nova_launch_attention(ctx, a, st);
     if (rc) return rc;
     // x1 = Xc + o W_o^T + b_o
@@ -312,6 +403,31 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
     g.gate = (cbf)md.gate1; g.img_row = ws.img_row;
     rc = nova_launch_gemm(ctx, g, st);
     if (rc) return rc;
+    if (cross) {
+        // x1 <- x1 + softmax(q2 Kc^T / sqrt(dh)) Vc W_o2^T + b_o2 with q2 = LN(x1) W_q2^T + b_q2: the same
+        // kernels once more, on buffers that are free at this point (h, q, o), the keys and values being
+        // the image's condition tokens and nothing else
+        LnModArgs none_mod = {nullptr, nullptr, ws.img_row};
+        rc = launch_ln(ctx, ws.x1, nullptr, none_mod, (cbf)ext->lnc_g, (cbf)ext->lnc_b, w->eps, M, m_dev, C, ws.h, st);
+        if (rc) return rc;
+        memset(&g, 0, sizeof(g));
+        g.A = ws.h; g.W = (cbf)ext->w_q2; g.bias = (cbf)ext->b_q2; g.M = M; g.m_dev = m_dev; g.N = C; g.K = C;
+        g.epilogue = NOVA_EPI_QKV; g.cat = NOVA_K_GEMM_QKV; g.out = ws.q; g.C = C; g.kv_row = ws.kv_row;   // all columns are q
+        rc = nova_launch_gemm(ctx, g, st);
+        if (rc) return rc;
+        nova_attn_args ca;
+        ca.q = ws.q; ca.k_cache = (cbf)ext->cond_k; ca.v_cache = (cbf)ext->cond_v; ca.cu_keep = cu_keep; ca.kv_len = ext->cond_len;
+        ca.o = ws.o; ca.B = s->B; ca.C = C; ca.n_heads = s->n_heads; ca.Lmax = ext->Lc_max; ca.M = M;
+        ca.scratch = nullptr; ca.scratch_bytes = 0;      // x1 is live: no room for a key-split wave
+        ca.cache_only = true;
+        rc = nova_launch_attention(ctx, ca, st);
+        if (rc) return rc;
+        memset(&g, 0, sizeof(g));
+        g.A = ws.o; g.W = (cbf)ext->w_o2; g.bias = (cbf)ext->b_o2; g.M = M; g.m_dev = m_dev; g.N = C; g.K = C;
+        g.epilogue = NOVA_EPI_BIAS_RES; g.cat = NOVA_K_GEMM_PROJ; g.out = ws.x1; g.res = ws.x1; g.res_row = nullptr;   // in place
+        rc = nova_launch_gemm(ctx, g, st);
+        if (rc) return rc;
+    }
     // h = LN2(x1)
     rc = launch_ln(ctx, ws.x1, nullptr, ln2_mod, (cbf)w->ln2_g, (cbf)w->ln2_b, w->eps, M, m_dev, C, ws.h, st);
     if (rc) return rc;
@@ -368,6 +484,17 @@ extern "C" nova_status nova_pruned_block_forward_adaln(nova_ctx* ctx, const nova
 {
     return block_forward(ctx, w, mod, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream,
                          m_on_device != 0);
+}
+
+extern "C" nova_status nova_pruned_block_forward_ext(nova_ctx* ctx, const nova_block_weights* w,
+                                                     const nova_block_modulation* mod, const nova_block_extras* ext,
+                                                     const nova_block_shape* s, const void* x_in,
+                                                     const int32_t* keep_idx, const int32_t* cu_keep,
+                                                     void* k_cache, void* v_cache, int32_t* kv_len,
+                                                     int append_kv, void* y_kept, int m_on_device, void* stream)
+{
+    return block_forward(ctx, w, mod, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, y_kept, stream,
+                         m_on_device != 0, nullptr, ext);
 }
 
 // Eq. 14 followed by Eq. 15-16 for one layer: the block on the kept rows with its last GEMM writing

@@ -182,6 +182,7 @@ struct nova_attn_args {
     int B, C, n_heads, Lmax, M;
     void* scratch;                 // device memory free during the launch (or NULL) for a key-split last wave
     size_t scratch_bytes;
+    bool cache_only;               // cross-attention: the keys are the kv_len[b] cache rows alone (no rows of this call)
 };
 
 nova_status nova_launch_attention(nova_ctx* ctx, const nova_attn_args& a, cudaStream_t st);

@@ -264,3 +264,111 @@ def test_attention_keys_with_vanishing_probability(ctx, C, heads):
     dead = np.arange(0, 900, 4)
     attention_case(ctx, B=2, N=300, C=C, heads=heads, F=256, Lmax=1400, ks=[300, 77], kv_lens=[900, 900], seed=89,
                    q_gain=2.0, dead_keys=dead, label=f"vanishing probabilities, head size {C // heads}")
+
+
+# ------------------------------------------------- block variants: rotary embedding, QK norm, cross-attention
+def _rope_tables(h, w, dh, seed):
+    """Axial 2-D rotary tables for an h x w token grid: the first half of a head's channel pairs turns
+    with the row index, the second half with the column index, at geometrically spaced frequencies."""
+    n_pairs = dh // 2
+    half = n_pairs // 2
+    freq = 1.0 / (100.0 ** (torch.arange(half, dtype=torch.float64) / half))
+    ys, xs = torch.meshgrid(torch.arange(h, dtype=torch.float64), torch.arange(w, dtype=torch.float64), indexing="ij")
+    ang = torch.cat([ys.reshape(-1, 1) * freq, xs.reshape(-1, 1) * freq], dim=1)          # [N, dh/2]
+    return torch.cos(ang).float().to(DEV), torch.sin(ang).float().to(DEV)
+
+
+@pytest.mark.parametrize("parts", ["rope", "qk_norm", "cross", "all", "all_modulated_device_count"])
+@pytest.mark.parametrize("C,heads", [(256, 2), (256, 4)])
+def test_block_variants_match_oracle(ctx, parts, C, heads):
+    """Rotary embedding, QK normalisation and cross-attention (one at a time and together, also with
+    adaptive-LayerNorm modulation and the kept count left on the device) against the oracle, with the
+    attention branches isolated (identity output projections, no MLP output, small input): the error is
+    taken relative to the attention output, and the transformed keys appended to the cache are compared too."""
+    B, h, w, F, Lmax, Lc = 3, 12, 15, 256, 700, 40
+    N, dh = h * w, C // heads
+    ks, kv_lens, cond_lens = [180, 77, 5], [300, 130, 0], [40, 7, 0]
+    seed = 91
+    wt = probe_weights(C, F, seed, q_gain=1.0 if "qk" in parts or parts.startswith("all") else 4.0)
+    x = (synth.activations(B, N, C, seed + 1, DEV).float() * X_SCALE).to(torch.bfloat16)
+    k_cache, v_cache, _ = synth.kv_cache(B, Lmax, max(kv_lens), C, seed + 2, DEV)
+    use_rope = parts in ("rope", "all", "all_modulated_device_count")
+    use_norm = parts in ("qk_norm", "all", "all_modulated_device_count")
+    use_cross = parts in ("cross", "all", "all_modulated_device_count")
+    ext = {}
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    if use_norm:
+        # unit-norm heads of random directions are nearly orthogonal: a large query gain spreads the scores
+        ext["qk_gain_q"] = (256.0 * (1 + 0.1 * torch.randn(C, generator=g))).to(torch.bfloat16).to(DEV)
+        ext["qk_gain_k"] = (1 + 0.1 * torch.randn(C, generator=g)).to(torch.bfloat16).to(DEV)
+        # prior keys as the cache holds them under this variant: unit heads
+        kc = k_cache.float().view(B, Lmax, heads, dh)
+        k_cache = (kc / kc.norm(dim=-1, keepdim=True).clamp_min(1e-6)).view(B, Lmax, C).to(torch.bfloat16)
+    if use_rope:
+        ext["rope_cos"], ext["rope_sin"] = _rope_tables(h, w, dh, seed)
+    if use_cross:
+        ext["lnc_g"] = synth.randn_bf16((C,), seed + 3, DEV, std=0.02, mean=1.0)
+        ext["lnc_b"] = synth.randn_bf16((C,), seed + 4, DEV, std=0.02)
+        ext["w_q2"] = synth.randn_bf16((C, C), seed + 5, DEV, std=0.08)
+        ext["b_q2"] = synth.randn_bf16((C,), seed + 6, DEV, std=0.02)
+        ext["w_o2"] = torch.eye(C, dtype=torch.bfloat16, device=DEV)
+        ext["b_o2"] = torch.zeros(C, dtype=torch.bfloat16, device=DEV)
+        ext["cond_k"] = synth.randn_bf16((B, Lc, C), seed + 7, DEV)
+        ext["cond_v"] = synth.randn_bf16((B, Lc, C), seed + 8, DEV)
+        for b, n in enumerate(cond_lens):
+            ext["cond_k"][b, n:] = float("nan")
+            ext["cond_v"][b, n:] = float("nan")
+        ext["cond_len"] = torch.tensor(cond_lens, dtype=torch.int32, device=DEV)
+    md = None
+    on_device = parts == "all_modulated_device_count"
+    if on_device:
+        md = {n: (0.3 * torch.randn((B, C), generator=g)).to(torch.bfloat16).to(DEV) for n in nova.MODULATION_NAMES}
+    for b, n in enumerate(kv_lens):
+        k_cache[b, n:] = float("nan")
+        v_cache[b, n:] = float("nan")
+    kv_len = torch.tensor(kv_lens, dtype=torch.int32, device=DEV)
+    ent = torch.rand((B, N), generator=torch.Generator(device="cpu").manual_seed(seed)).to(DEV)
+    M = sum(ks)
+    cap = B * N if on_device else M
+    keep_idx = torch.zeros(cap, dtype=torch.int32, device=DEV)
+    prune_idx = torch.empty(B * N - M, dtype=torch.int32, device=DEV)
+    cu = torch.empty(B + 1, dtype=torch.int32, device=DEV)
+    nova.nova_select_topk(ctx, ent, torch.tensor(ks, dtype=torch.int32), keep_idx[:M], prune_idx, cu, None)
+    shape = nova.BlockShape(B, N, C, heads, F, Lmax, cap)
+    ctx.ensure_workspace(shape)
+    k0, v0 = k_cache.clone(), v_cache.clone()
+    y = torch.full((cap, C), float("nan"), dtype=torch.bfloat16, device=DEV)
+    nova.nova_pruned_block_forward_ext(ctx, nova.BlockWeights(wt, 1e-6), md, ext, shape, x, keep_idx, cu, k_cache, v_cache,
+                                       kv_len, True, y, m_on_device=on_device)
+    assert ctx.device_status() == 0
+
+    wts = {n: f32(t) for n, t in wt.items()}
+    oext = {}
+    for n, t in ext.items():
+        name = {"cond_k": "ck", "cond_v": "cv"}.get(n, n)
+        oext[name] = t.cpu().numpy() if n == "cond_len" else np.nan_to_num(f32(t))
+    ki, cuu = keep_idx[:M].cpu().numpy(), cu.cpu().numpy()
+    lens = np.array(kv_lens, np.int32)
+    mod_np = {n: f32(t) for n, t in md.items()} if md else None
+    wy, wk, _ = oracle.pruned_block_forward_ext(wts, 1e-6, heads, f32(x), ki, cuu, np.nan_to_num(f32(k0)),
+                                                np.nan_to_num(f32(v0)), lens, oext, modulation=mod_np)
+    img = np.searchsorted(cuu, np.arange(M), side="right") - 1
+    x_rows = f32(x)[img, ki]
+    gy = f32(y)[:M]
+    assert np.isfinite(gy).all()
+    err, branch = attn_metric(gy, wy, x_rows)
+    # the variant acts: the plain block's output is far from it in the same metric
+    py, _, _ = oracle.pruned_block_forward(wts, 1e-6, heads, f32(x), ki, cuu, np.nan_to_num(f32(k0)), np.nan_to_num(f32(v0)),
+                                           lens, modulation=mod_np)
+    plain, _ = attn_metric(py, wy, x_rows)
+    print(f"block variant [{parts}, head size {dh}]: err {err:.2e} of max|branches| {branch:.3f}; plain block {plain:.2f}")
+    assert plain > 5 * BLOCK_TOL
+    assert err <= BLOCK_TOL
+    gk = f32(k_cache)
+    for b in range(B):
+        n0, kb = kv_lens[b], ks[b]
+        want_rows = wk[cuu[b]:cuu[b + 1]]
+        assert np.abs(gk[b, n0:n0 + kb] - want_rows).max() <= BLOCK_TOL * np.abs(want_rows).max()
+    if on_device:
+        assert torch.isnan(y[M:].float()).all()
+    assert kv_len.cpu().tolist() == [a + b for a, b in zip(kv_lens, ks)]
