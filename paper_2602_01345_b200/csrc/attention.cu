@@ -302,105 +302,75 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             }
         }
     } else if (warp == 1) {
-        // The whole warp runs this loop in lockstep and one lane issues. Control flow, stage
-        // counters and descriptors are then warp-uniform by construction, which lets the compiler
-        // keep the operands of tcgen05.mma where the instruction takes them from (uniform
-        // registers) instead of moving them there before every issue from a diverged thread; the
-        // tensor core executes an instruction every 64 clocks and accepts them hardly faster, so
-        // every clock of issue overhead is a clock of tensor-core idle time.
-        constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
-        constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
-        // Shared-memory descriptors: (address >> 4) sits in the low 14 bits, so stepping through
-        // a tile or to another stage is an integer add.
-        // tcgen05.mma takes its descriptors and addresses from uniform registers. Everything
-        // they are built from is broadcast from lane 0 once, which tells the compiler that the
-        // values are warp-uniform, so the per-instruction address arithmetic stays in the uniform
-        // datapath instead of being moved there from a lane's registers before every issue.
-        constexpr uint32_t kTileStep = L::kTileBytes >> 4;
-        auto uniform32 = [](uint32_t v) { return __shfl_sync(0xffffffffu, v, 0); };
-        auto uniform64 = [&](uint64_t v) {
-            return ((uint64_t)uniform32((uint32_t)(v >> 32)) << 32) | uniform32((uint32_t)v);
-        };
-        const uint64_t q_desc = uniform64(smem_desc_sw128(smem_u32(q_smem), 16, 1024));
-        const uint64_t k_desc = uniform64(smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024));
-        const uint64_t v_desc = uniform64(smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024));
-        const uint32_t tmem_u = uniform32(tmem_base);
-        const int n_tiles_u = (int)uniform32((uint32_t)n_tiles);     // loop bounds too: uniform control flow
-        const int n_q = (int)uniform32(tile_b_active ? 2u : 1u);
-        const bool issuer = (lane == 0);
-        // S_t = Q_t K^T with K in stage ks
-        auto issue_s = [&](int t, int ks) {
-            const uint64_t qd = q_desc + (uint32_t)t * kTileStep;
-            const uint64_t kd = k_desc + (uint32_t)ks * kTileStep;
-            if (issuer) {
+        // tcgen05.mma issuer: one elected thread serves both query tiles, in the fixed order
+        //     O_A += P_A V_j ; S_A = Q_A K_{j+1}^T ; O_B += P_B V_j ; S_B = Q_B K_{j+1}^T
+        // which is what keeps the two tiles half a period apart (one tile's softmax runs while the
+        // other's 16 instructions execute). Issuing costs the thread about 45 clocks per instruction
+        // against 64 of execution, and the tensor pipe queues only three or four instructions, so every
+        // other clock the thread spends is tensor-core idle time: a barrier wait by one thread costs 65
+        // clocks when already satisfied, the same wait taken by the whole warp with a vote around it
+        // more than 300. Hence a single thread that does nothing but wait and issue.
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
+            constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
+            // Shared-memory descriptors: (address >> 4) sits in the low 14 bits, so stepping through
+            // a tile or to another stage is an integer add.
+            constexpr uint32_t kTileStep = L::kTileBytes >> 4;
+            const uint64_t q_desc = smem_desc_sw128(smem_u32(q_smem), 16, 1024);
+            const uint64_t k_desc = smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024);
+            const uint64_t v_desc = smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024);
+            const int n_q = tile_b_active ? 2 : 1;
+            // S_t = Q_t K^T with K in stage ks
+            auto issue_s = [&](int t, int ks) {
+                const uint64_t qd = q_desc + (uint32_t)t * kTileStep;
+                const uint64_t kd = k_desc + (uint32_t)ks * kTileStep;
 #pragma unroll
                 for (int kk = 0; kk < DH / 16; ++kk) {
                     constexpr uint32_t kSlabStep = kSlabBytes >> 4;
                     const uint32_t off = (kk >> 2) * kSlabStep + (kk & 3) * 2;    // 32 bytes per 16 k
-                    mma_bf16_ss(tmem_u + 128u * t, qd + off, kd + off, idesc_s, kk ? 1u : 0u);
+                    mma_bf16_ss(tmem_base + 128u * t, qd + off, kd + off, idesc_s, kk ? 1u : 0u);
                 }
                 mma_commit(&s_full[t]);
-            }
-            __syncwarp();
-        };
-        // O_t (+)= P_t V with V in stage vs; P_t sits in the first 64 columns of S_t, two keys per column
-        auto issue_pv = [&](int t, int vs, bool first) {
-            const uint64_t vd = v_desc + (uint32_t)vs * kTileStep;
-            if (issuer) {
+            };
+            // O_t (+)= P_t V with V in stage vs; P_t sits in the first 64 columns of S_t, two keys per column
+            auto issue_pv = [&](int t, int vs, bool first) {
+                const uint64_t vd = v_desc + (uint32_t)vs * kTileStep;
 #pragma unroll
                 for (int kk = 0; kk < BKV / 16; ++kk)
-                    mma_bf16_ts(tmem_u + 256u + 128u * t, tmem_u + 128u * t + kk * 8, vd + (uint32_t)(kk * 128),
+                    mma_bf16_ts(tmem_base + 256u + 128u * t, tmem_base + 128u * t + kk * 8, vd + (uint32_t)(kk * 128),
                                 idesc_o, (first && kk == 0) ? 0u : 1u);
-            }
-            __syncwarp();
-        };
-        bool ok = mbar_wait_warp(q_full, 0, abort_flag, p.status);
-        if (ok) ok = mbar_wait_warp(&k_full[0], 0, abort_flag, p.status);
-        if (ok) {
-            tc_fence_after();
-            for (int t = 0; t < n_q; ++t) issue_s(t, 0);
-            if (issuer) mma_commit(&k_empty[0]);
-            __syncwarp();
-        }
-        // ring positions and phase parities, stepped without divisions
-        int vs = 0, ks_next = (kKStages > 1) ? 1 : 0;
-        uint32_t v_par = 0, k_par_next = (kKStages > 1) ? 0u : 1u;
-        for (int j = 0; j < n_tiles_u && ok; ++j) {
-            const bool more = j + 1 < n_tiles_u;
-            // The three barriers this step starts with are tried together, so their shared-memory
-            // round trips overlap; whatever is not complete yet gets a bounded wait of its own.
-            {
-                const bool v_ok = mbar_try_wait(&v_full[vs], v_par);
-                const bool k_ok = more ? mbar_try_wait(&k_full[ks_next], k_par_next) : true;
-                const bool p_ok = mbar_try_wait(&p_full[0], j & 1);
-                if (!__all_sync(0xffffffffu, v_ok && k_ok && p_ok)) {
-                    ok = mbar_wait_warp(&v_full[vs], v_par, abort_flag, p.status);
-                    if (ok && more) ok = mbar_wait_warp(&k_full[ks_next], k_par_next, abort_flag, p.status);
-                    if (ok) ok = mbar_wait_warp(&p_full[0], j & 1, abort_flag, p.status);
-                }
-            }
-            for (int t = 0; t < n_q && ok; ++t) {
-                if (t > 0) ok = mbar_wait_warp(&p_full[t], j & 1, abort_flag, p.status);
-                if (!ok) break;
+            };
+            bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
+            if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag, p.status);
+            if (ok) {
                 tc_fence_after();
-                issue_pv(t, vs, j == 0);
-                if (t == n_q - 1) {
-                    if (issuer) mma_commit(&v_empty[vs]);                 // V_j has no reader left
-                    __syncwarp();
-                }
-                if (more) {
-                    issue_s(t, ks_next);
-                    if (t == n_q - 1) {
-                        if (issuer) mma_commit(&k_empty[ks_next]);        // nor has K_{j+1}
-                        __syncwarp();
+                for (int t = 0; t < n_q; ++t) issue_s(t, 0);
+                mma_commit(&k_empty[0]);
+            }
+            // ring positions and phase parities, stepped without divisions
+            int vs = 0, ks_next = (kKStages > 1) ? 1 : 0;
+            uint32_t v_par = 0, k_par_next = (kKStages > 1) ? 0u : 1u;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const bool more = j + 1 < n_tiles;
+                // V_j and K_{j+1} have usually landed long ago; P is what a step waits for
+                ok = mbar_wait(&v_full[vs], v_par, abort_flag, p.status);
+                if (ok && more) ok = mbar_wait(&k_full[ks_next], k_par_next, abort_flag, p.status);
+                for (int t = 0; t < n_q && ok; ++t) {
+                    ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(t, vs, j == 0);
+                    if (t == n_q - 1) mma_commit(&v_empty[vs]);                 // V_j has no reader left
+                    if (more) {
+                        issue_s(t, ks_next);
+                        if (t == n_q - 1) mma_commit(&k_empty[ks_next]);        // nor has K_{j+1}
                     }
                 }
+                if (++vs == kVStages) { vs = 0; v_par ^= 1u; }
+                if (++ks_next == kKStages) { ks_next = 0; k_par_next ^= 1u; }
             }
-            if (++vs == kVStages) { vs = 0; v_par ^= 1u; }
-            if (++ks_next == kKStages) { ks_next = 0; k_par_next ^= 1u; }
+            if (ok) mma_commit(o_done);
         }
-        if (ok && issuer) mma_commit(o_done);
-        __syncwarp();
     }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsHigh));
@@ -412,10 +382,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             const uint32_t s_addr = tmem_base + lane_off + 128u * t;
             const uint32_t o_addr = tmem_base + lane_off + 256u + 128u * t;
             const float c = p.scale_log2e;
-            // Polynomial share of the exponentials (pairs out of every four pairs of scores): the
-            // special-function unit delivers one exponential per 8 clocks and scheduler, the polynomial
-            // costs about as much in issue slots, so the two pipes share the work.
-            constexpr int kPolyPairs = (DH == 64) ? 1 : 2;
+            // Polynomial share of the exponentials (pairs out of every four pairs of scores). The
+            // special-function unit delivers one exponential per 8 clocks and scheduler; the polynomial
+            // costs a scheduler about as much in issue slots, so it does not replace that unit, it only
+            // works beside it: a quarter of the scores on the polynomial measured best at both head sizes
+            // (6.9 clocks per score and scheduler against 7.5 at a half and 8.2 with none).
+            constexpr int kPolyPairs = 1;
             // The reference maximum starts at a finite floor, not -inf: (-inf) - (-inf) must not appear.
             float m_ref = -1e30f, l_run = 0.f;
             bool ok = true;

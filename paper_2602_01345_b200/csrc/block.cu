@@ -51,8 +51,10 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// Three resident blocks per SM (80 registers): with two (94 registers) a launch of 1024 blocks ran 3.5
+// waves of load-then-compute and sat at 0.41 of the HBM peak.
 template <int VEC, bool MAPS, bool MOD>
-__global__ void __launch_bounds__(kLnWarps * 32)
+__global__ void __launch_bounds__(kLnWarps * 32, 3)
 layernorm_rows(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                float eps, int M, const int32_t* __restrict__ m_dev, int vec_per_row, uint4* __restrict__ out,
                const RowMapArgs maps, const LnModArgs mod)
