@@ -149,3 +149,79 @@ def test_var_d30_512_generation_from_detected_inflection():
     fired = r["act_scale"][r["act_scale"] > 0]
     assert r["first_pruned_scale"] == int(fired.min())                        # pruning begins exactly there
     assert r["pruned_layers"] >= 30 and r["checked"] == 2
+
+
+@pytest.mark.parametrize("cfg,B,keep", [("c4_1024", 1, 0.25), ("c4_1024", 1, 0.5), ("c4_1024", 1, 0.75),
+                                        ("c4_1024", 4, 0.25), ("c4_1024", 4, 0.5), ("c4_1024", 4, 0.75),
+                                        ("c5_2048", 1, 0.2)])
+def test_large_shapes_keep_sweep_through_the_runner(cfg, B, keep):
+    """The 1024x1024 shape at keep ratios 0.25 / 0.5 / 0.75 and batch 1 / 4, and the 2048x2048 shape at
+    keep 0.2: the last scale through the scale runner (two layers resident: the launch shapes are
+    those of the full model), forced activation and keep ratio as the configurations state. Keep
+    counts and index lists of both layers exact; the second layer's block and restore against the
+    oracle on the layer's actual inputs (sampled kept rows, every pruned row)."""
+    ms = synth.CONFIGS[cfg]
+    L, t = 2, len(ms.scales)
+    side, prev = ms.scales[-1], ms.scales[-2]
+    N, P, Lmax, C = side * side, ms.prior_tokens(t), ms.total_tokens, ms.C
+    ctx = nova.Context(0)
+    weights = [synth.block_weights(C, ms.F, 70 + j, DEV) for j in range(L)]
+    k_caches, v_caches = [], []
+    for j in range(L):
+        k, v, _ = synth.kv_cache(B, Lmax, P, C, 80 + 2 * j, DEV)
+        k_caches.append(k)
+        v_caches.append(v)
+    kv_len = torch.full((L, B), P, dtype=torch.int32, device=DEV)
+    cache_prev = [synth.residual_cache(B, prev, prev, C, 90 + j, DEV) for j in range(L)]
+    if cfg == "c5_2048":
+        a = synth.blob_temperature_field(B, side, side, 7, cover=0.2, device=DEV)      # high entropy in blobs covering 20 %
+    else:
+        a = synth.smooth_temperature_field(B, side, side, 7, device=DEV)
+    beta = synth.layer_inverse_temperatures(L, 7)
+    logits = [synth.logits_from_temperature(a * float(beta[j]), synth.V_CODEBOOK, 100 + j) for j in range(L)]
+    x_in = synth.activations(B, N, C, 110, DEV)
+    sched = nova.SchedParams(force_act_scale=t, force_keep_ratio=keep)
+    osched = oracle.SchedParams(force_act_scale=t, force_keep_ratio=keep)
+    hbar = torch.linspace(2.0, 7.0, t).repeat(B, 1).contiguous()
+    runner = pipeline.PrunedScaleRunner(ctx, weights, ms.heads, B, side, side, Lmax, k_caches, v_caches, kv_len,
+                                        cache_prev, fused_restore=True)
+    snap = {}
+
+    def hook(stage, j, info):
+        if j != L - 1:
+            return
+        if stage == "before":
+            snap.update(x_in=info["x_in"].clone(), k=info["k_cache"].clone(), v=info["v_cache"].clone())
+        else:
+            snap.update(x_out=info["x_out"].clone(), cache_out=info["cache_out"].clone())
+
+    x_out, keeps = runner.run_scale(x_in, logits, sched, t, hbar, layer_hook=hook)
+    assert ctx.device_status() == 0
+    k_want = N - int((1.0 - keep) * N)
+    ent_gpu = runner.ent.cpu().numpy()
+    kk, pp, cc = runner.keep_idx.cpu().numpy(), runner.prune_idx.cpu().numpy(), runner.cu_keep.cpu().numpy()
+    for j in range(L):
+        wr = oracle.keep_ratios(osched, t, j + 1, N, hbar.numpy())
+        assert np.array_equal(keeps[j].numpy(), wr["keep"]) and (wr["keep"] == k_want).all()
+        w_keep, w_prune, w_cu, _ = oracle.select_topk(ent_gpu[j], wr["keep"])
+        M = int(w_cu[-1])
+        assert np.array_equal(cc[j], w_cu) and np.array_equal(kk[j, :M], w_keep)
+        assert np.array_equal(pp[j, : B * N - M], w_prune)
+    if cfg == "c5_2048":
+        # the kept tokens are the high-entropy blobs: almost all of them lie where the field is hot
+        hot = (a[0].cpu().numpy() < 1.0)
+        assert hot[w_keep].mean() > 0.9
+    j = L - 1
+    rng = np.random.default_rng(3)
+    rows = np.unique(np.r_[0, M - 1, rng.integers(0, M, 10)]).astype(np.int32)
+    wy, _, _ = oracle.pruned_block_forward({n: f32(v) for n, v in weights[j].items()}, 1e-6, ms.heads, f32(snap["x_in"]),
+                                           w_keep, w_cu, f32(snap["k"]), f32(snap["v"]), np.full(B, P, np.int32), rows=rows)
+    gx, gc = f32(snap["x_out"]), f32(snap["cache_out"])
+    img = np.searchsorted(w_cu, rows, side="right") - 1
+    assert _rel_err(gx[img, w_keep[rows]], wy) <= BLOCK_TOL
+    img_all = np.searchsorted(w_cu, np.arange(M), side="right") - 1
+    wx, wc = oracle.restore_from_cache(f32(snap["x_in"]), gx[img_all, w_keep], w_keep, w_prune, w_cu, f32(cache_prev[j]),
+                                       side, side)
+    assert _bf16_ulp_ok(gx, wx) and _bf16_ulp_ok(gc, wc)
+    assert kv_len.cpu().tolist() == [[P + k_want] * B] * L
+    ctx.close()
