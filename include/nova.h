@@ -71,7 +71,7 @@ const char* nova_status_string(nova_status s);
 
 /* Synchronises `stream`, returns the device status word (NOVA_OK, NOVA_ERR_TIMEOUT,
  * NOVA_ERR_SHAPE for a K/V cache that would overflow, or NOVA_ERR_NONFINITE, in that order of
- * precedence) and clears it. */
+ * precedence; in debug mode also NOVA_ERR_CUDA for a launch that failed) and clears it. */
 nova_status nova_device_status(nova_ctx* ctx, void* stream);
 
 /* ---- bounded device-side waits (no counterpart in the paper) -------------------- */
@@ -84,6 +84,21 @@ nova_status nova_device_status(nova_ctx* ctx, void* stream);
  * leave the context usable. It reads and writes no caller memory. */
 nova_status nova_set_wait_limit_ns(nova_ctx* ctx, unsigned long long ns);
 nova_status nova_debug_wait_probe(nova_ctx* ctx, void* stream);
+
+/* ---- debug mode and tracing (no counterpart in the paper) ------------------------ */
+/* Debug mode is off unless the environment variable NOVA_DEBUG is set (and not "0") when the
+ * context is created; nova_set_debug switches it for the context's later calls. While it is on,
+ *  - every call that reads index lists (nova_pruned_block_forward*, nova_pruned_layer_forward,
+ *    nova_restore_from_cache*) first validates them on the device: cu_keep[0] = 0, 0 <= k_s <= N per
+ *    segment, cu_keep[B] = M (<= M where M is only a bound), every keep_idx / prune_idx entry inside
+ *    [0, N) and ascending within its segment. A list that fails returns NOVA_ERR_INVALID_ARG and
+ *    launches nothing else, so a corrupt index is never dereferenced;
+ *  - the stream is synchronised after every kernel launch, which pins an asynchronous CUDA error to
+ *    the launch that caused it (reported by nova_device_status as NOVA_ERR_CUDA, launch number in
+ *    nova_last_error).
+ * Both cost host synchronisations: not for timed runs. Independently of debug mode every launching
+ * call opens an NVTX range named after itself (no cost unless a tool listens). */
+nova_status nova_set_debug(nova_ctx* ctx, int on);
 
 /* ---- measurement (no counterpart in the paper) --------------------------------- */
 /* Kernels launched by this context since nova_create. */

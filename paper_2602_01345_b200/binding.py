@@ -196,6 +196,12 @@ class Context:
         with torch.cuda.device(self.device):
             self.check(_lib.nova_set_wait_limit_ns(self.handle, int(ns)))
 
+    def set_debug(self, on: bool):
+        """Debug mode: index lists validated on the device before use, every launch synchronised."""
+        _lib.nova_set_debug.argtypes = [_vp, _i]
+        _lib.nova_set_debug.restype = _i
+        self.check(_lib.nova_set_debug(self.handle, 1 if on else 0))
+
     def debug_wait_probe(self, stream=None):
         """Launches the diagnostic kernel whose wait can only end by running into the limit."""
         _lib.nova_debug_wait_probe.argtypes = [_vp, _vp]

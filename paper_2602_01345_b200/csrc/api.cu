@@ -2,6 +2,7 @@
 #include "tc_common.cuh"
 
 #include <math.h>
+#include <stdlib.h>
 #include <new>
 
 extern "C" {
@@ -42,6 +43,9 @@ nova_status nova_create(nova_ctx** out, int device)
     ctx->profiling = false;
     ctx->events_used = 0;
     ctx->wait_limit_ns = 0;
+    const char* dbg = getenv("NOVA_DEBUG");
+    ctx->debug = dbg && dbg[0] && strcmp(dbg, "0") != 0;
+    ctx->debug_failed = false;
     // the allocation is made with `device` current; the caller's current device is put back
     int prev = -1;
     const bool have_prev = (cudaGetDevice(&prev) == cudaSuccess);
@@ -137,7 +141,12 @@ nova_status nova_device_status(nova_ctx* ctx, void* stream)
                                                  sizeof(ctx->wait_limit_ns), cudaMemcpyHostToDevice, st));
         NOVA_CUDA_CHECK(ctx, cudaStreamSynchronize(st));
     }
+    if (ctx->debug_failed) {    // message already in err: a launch failed under debug mode's per-launch synchronisation
+        ctx->debug_failed = false;
+        return NOVA_ERR_CUDA;
+    }
     if (word & NOVA_DEV_TIMEOUT) return nova_fail(ctx, NOVA_ERR_TIMEOUT, "a device-side wait expired");
+    if (word & NOVA_DEV_BAD_INDEX) return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "an index list failed the debug mode's validation");
     if (word & NOVA_DEV_SHAPE) return nova_fail(ctx, NOVA_ERR_SHAPE, "K/V cache overflow on the device");
     if (word & NOVA_DEV_NONFINITE) return nova_fail(ctx, NOVA_ERR_NONFINITE, "non-finite logit");
     return NOVA_OK;
@@ -153,6 +162,65 @@ nova_status nova_set_wait_limit_ns(nova_ctx* ctx, unsigned long long ns)
     NOVA_CUDA_CHECK(ctx, cudaMemcpy(ctx->dev_status + NOVA_WAIT_LIMIT_WORD, &ctx->wait_limit_ns, sizeof(ns), cudaMemcpyHostToDevice));
     return NOVA_OK;
 }
+
+nova_status nova_set_debug(nova_ctx* ctx, int on)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    ctx->debug = on != 0;
+    return NOVA_OK;
+}
+
+}  // extern "C"
+
+// Debug mode: one block per segment validates that segment's slice of the lists. A block touches a
+// list only after its own two prefix-sum entries have passed, so that no read leaves the lists.
+__global__ void check_lists_kernel(const int32_t* __restrict__ keep_idx, const int32_t* __restrict__ prune_idx,
+                                   const int32_t* __restrict__ cu_keep, int N, long m_bound, bool m_exact,
+                                   unsigned int* status)
+{
+    const int s = blockIdx.x;
+    const long c0 = cu_keep[s], c1 = cu_keep[s + 1];
+    bool bad = (s == 0 && c0 != 0) || c0 < 0 || c0 > (long)s * N || c1 < c0 || c1 - c0 > N || c1 > m_bound ||
+               (m_exact && s == (int)gridDim.x - 1 && c1 != m_bound);
+    if (!bad) {
+        if (keep_idx) {
+            for (long i = c0 + threadIdx.x; i < c1; i += blockDim.x) {
+                const int v = keep_idx[i];
+                if (v < 0 || v >= N || (i > c0 && keep_idx[i - 1] >= v)) bad = true;
+            }
+        }
+        if (prune_idx) {
+            const long p0 = (long)s * N - c0, p1 = p0 + N - (c1 - c0);
+            for (long i = p0 + threadIdx.x; i < p1; i += blockDim.x) {
+                const int v = prune_idx[i];
+                if (v < 0 || v >= N || (i > p0 && prune_idx[i - 1] >= v)) bad = true;
+            }
+        }
+    }
+    if (bad) atomicOr(status, NOVA_DEV_BAD_INDEX);
+}
+
+nova_status nova_debug_check_lists(nova_ctx* ctx, const char* who, const int32_t* keep_idx,
+                                   const int32_t* prune_idx, const int32_t* cu_keep,
+                                   int B, int N, long m_bound, bool m_exact, cudaStream_t st)
+{
+    if (!ctx->debug || B <= 0 || !cu_keep) return NOVA_OK;
+    check_lists_kernel<<<B, 256, 0, st>>>(keep_idx, prune_idx, cu_keep, N, m_bound, m_exact, ctx->dev_status);
+    NOVA_CUDA_CHECK(ctx, cudaGetLastError());
+    unsigned int word = 0;
+    NOVA_CUDA_CHECK(ctx, cudaMemcpyAsync(&word, ctx->dev_status, sizeof(word), cudaMemcpyDeviceToHost, st));
+    NOVA_CUDA_CHECK(ctx, cudaStreamSynchronize(st));
+    if (word & NOVA_DEV_BAD_INDEX) {
+        word &= ~NOVA_DEV_BAD_INDEX;
+        NOVA_CUDA_CHECK(ctx, cudaMemcpyAsync(ctx->dev_status, &word, sizeof(word), cudaMemcpyHostToDevice, st));
+        NOVA_CUDA_CHECK(ctx, cudaStreamSynchronize(st));
+        snprintf(ctx->err, sizeof(ctx->err), "%s: keep_idx / prune_idx / cu_keep failed validation (debug mode): nothing launched", who);
+        return NOVA_ERR_INVALID_ARG;
+    }
+    return NOVA_OK;
+}
+
+extern "C" {
 
 // One CTA whose consumer warp waits on a barrier that no producer ever arrives on: the wait runs
 // into the context's limit, records the time-out and the kernel returns normally.

@@ -344,6 +344,11 @@ static nova_status block_forward(nova_ctx* ctx, const nova_block_weights* w, con
     NOVA_DEVICE_GUARD(ctx, "nova_pruned_block_forward");
 
     cudaStream_t st = (cudaStream_t)stream;
+    {
+        const nova_status chk = nova_debug_check_lists(ctx, "nova_pruned_block_forward", keep_idx, nullptr, cu_keep,
+                                                       s->B, s->N, s->M, !m_on_device, st);
+        if (chk != NOVA_OK) return chk;
+    }
     const int M = s->M, C = s->C, F = s->F;
     typedef const __nv_bfloat16* cbf;
     typedef __nv_bfloat16* bf;
@@ -521,6 +526,12 @@ extern "C" nova_status nova_pruned_layer_forward(nova_ctx* ctx, const nova_block
     const bool on_dev = m_on_device != 0;
     if ((s->M < total || on_dev) && (!prune_idx || !cache_prev || hp < 1 || wp < 1))
         return nova_fail(ctx, NOVA_ERR_INVALID_ARG, "nova_pruned_layer_forward: pruned rows need prune_idx and cache_prev");
+    NOVA_DEVICE_GUARD(ctx, "nova_pruned_layer_forward");
+    {   // debug mode: both lists are checked before the block's first kernel, so that a bad pruned list leaves no half-done layer
+        const nova_status chk = nova_debug_check_lists(ctx, "nova_pruned_layer_forward", keep_idx, prune_idx, cu_keep,
+                                                       s->B, s->N, s->M, !on_dev, (cudaStream_t)stream);
+        if (chk != NOVA_OK) return chk;
+    }
     ScatterOut sc = {x_out, cache_out};
     nova_status rc = block_forward(ctx, w, mod, s, x_in, keep_idx, cu_keep, k_cache, v_cache, kv_len, append_kv, nullptr,
                                    stream, on_dev, &sc);

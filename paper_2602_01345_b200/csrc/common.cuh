@@ -8,6 +8,7 @@
 #include <stdio.h>
 #include <string.h>
 #include <vector>
+#include <nvtx3/nvToolsExt.h>
 
 #include "../../include/nova.h"
 
@@ -15,6 +16,7 @@
 #define NOVA_DEV_NONFINITE 1u
 #define NOVA_DEV_TIMEOUT   2u
 #define NOVA_DEV_SHAPE     4u
+#define NOVA_DEV_BAD_INDEX 8u         // set by the debug mode's validation of keep / prune / cu_keep lists
 
 // Layout of the context's one device allocation: NOVA_STATUS_WORDS 32-bit words (word 0 = status
 // flags, a block of tickets for key-split attention items), then one 64-bit accumulator per segment
@@ -48,6 +50,8 @@ struct nova_ctx {
     int num_sms;
     bool attr_select, attr_gemm, attr_attn;   // dynamic shared memory opt-in done on this device
     unsigned long long wait_limit_ns;   // mirrored in the status block (0 = default)
+    bool debug;                 // debug mode: index lists validated before use, every launch synchronised
+    bool debug_failed;          // a launch failed in debug mode (message in err); reported by nova_device_status
     char err[256];
     // measurement: launches since creation, and event pairs around each launch while profiling
     unsigned long long launches;
@@ -83,7 +87,23 @@ struct nova_launch_scope {
     ~nova_launch_scope()
     {
         if (stop) cudaEventRecord(stop, st);
+        if (ctx->debug && !ctx->debug_failed) {
+            // debug mode: an asynchronous failure is pinned to the launch that caused it
+            const cudaError_t e = cudaStreamSynchronize(st);
+            if (e != cudaSuccess) {
+                snprintf(ctx->err, sizeof(ctx->err), "launch %llu failed: %s", ctx->launches, cudaGetErrorString(e));
+                ctx->debug_failed = true;
+            }
+        }
     }
+};
+
+// One NVTX range per C-ABI call (a no-op unless a tool that listens to NVTX is attached).
+struct nova_api_range {
+    explicit nova_api_range(const char* name) { nvtxRangePushA(name); }
+    ~nova_api_range() { nvtxRangePop(); }
+    nova_api_range(const nova_api_range&) = delete;
+    nova_api_range& operator=(const nova_api_range&) = delete;
 };
 
 static inline nova_status nova_fail(nova_ctx* ctx, nova_status s, const char* msg)
@@ -124,11 +144,22 @@ static inline nova_status nova_check_device(nova_ctx* ctx, const char* who)
     }
     return NOVA_OK;
 }
+// Also opens the call's NVTX range, which lasts until the calling function returns.
 #define NOVA_DEVICE_GUARD(ctx, who)                                           \
+    nova_api_range nova_api_range__(who);                                     \
     do {                                                                      \
         const nova_status g__ = nova_check_device((ctx), (who));              \
         if (g__ != NOVA_OK) return g__;                                       \
     } while (0)
+
+// Debug mode only (returns NOVA_OK at once otherwise): checks on the device, before any kernel uses
+// them, that cu_keep is a valid prefix sum (cu_keep[0] = 0, 0 <= k_s <= N, total <= m_bound, or
+// == m_bound when m_exact) and that every keep / prune entry is an in-segment index in [0, N),
+// ascending within its segment. Synchronises the stream. keep_idx or prune_idx may be null (that
+// list is then not looked at).
+nova_status nova_debug_check_lists(nova_ctx* ctx, const char* who, const int32_t* keep_idx,
+                                   const int32_t* prune_idx, const int32_t* cu_keep,
+                                   int B, int N, long m_bound, bool m_exact, cudaStream_t st);
 
 // Kernel launchers implemented in the other translation units.
 

@@ -151,6 +151,12 @@ static nova_status restore(nova_ctx* ctx, const void* x_in, const void* y_kept,
         !nova_aligned16(cache_prev) || !nova_aligned16(cache_out))
         return nova_fail(ctx, NOVA_ERR_ALIGNMENT, "nova_restore_from_cache: tensors must be 16-byte aligned");
     NOVA_DEVICE_GUARD(ctx, "nova_restore_from_cache");
+    {
+        // pruned_only: the kept list is not read (and may be null)
+        const nova_status chk = nova_debug_check_lists(ctx, "nova_restore_from_cache", pruned_only ? nullptr : keep_idx,
+                                                       prune_idx, cu_keep, B, h * w, M, !m_on_device, (cudaStream_t)stream);
+        if (chk != NOVA_OK) return chk;
+    }
     // rows this launch may have to visit: all of them, or only the pruned ones (when the host knows M)
     const long items = (pruned_only && !m_on_device) ? total - M : total;
     if (items == 0) return NOVA_OK;
