@@ -162,6 +162,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     using L = AttnSmem<DH>;
     constexpr int kSlabs = L::kSlabs;
     constexpr int kKStages = L::kKStages, kVStages = L::kVStages;
+    constexpr int kIssuers = (DH == 128) ? 2 : 1;     // threads that issue tcgen05.mma (see the issuer code below)
     constexpr uint32_t kTmemCols = 512;
     // S tile t (fp32) sits at column 128*t; its first 64 columns are reused for P (bf16 pairs).
     // O tile t (fp32, DH columns) sits at column 256 + 128*t.
@@ -228,8 +229,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint64_t* v_empty = v_full + kVStages;            // kVStages
     uint64_t* s_full = v_empty + kVStages;            // 2 (tile A, tile B)
     uint64_t* p_full = s_full + 2;                    // 2, one arrival per softmax warp
-    uint64_t* o_done = p_full + 2;                    // 1
-    uint32_t* tmem_slot = (uint32_t*)(o_done + 1);
+    uint64_t* o_done = p_full + 2;                    // 1, one arrival per issuing thread
+    uint64_t* turn = o_done + 1;                      // 2 counters (not barriers): turns granted to the issuing thread of tile t
+    uint32_t* tmem_slot = (uint32_t*)(turn + 2);
     __shared__ int abort_flag_s;
     __shared__ int ticket_s;
     volatile int* abort_flag = &abort_flag_s;
@@ -239,19 +241,22 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         mbar_init(q_full, 1);
+        // a K or V stage is free once the issuing thread of every active query tile has committed
+        const int n_issuers = (kIssuers == 2 && tile_b_active) ? 2 : 1;
         for (int s = 0; s < kKStages; ++s) {
             mbar_init(&k_full[s], 1);
-            mbar_init(&k_empty[s], 1);
+            mbar_init(&k_empty[s], n_issuers);
         }
         for (int s = 0; s < kVStages; ++s) {
             mbar_init(&v_full[s], 1);
-            mbar_init(&v_empty[s], 1);
+            mbar_init(&v_empty[s], n_issuers);
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&s_full[t], 1);
             mbar_init(&p_full[t], 4);
+            turn[t] = 0;                              // a plain counter, not a barrier
         }
-        mbar_init(o_done, 1);
+        mbar_init(o_done, n_issuers);
         fence_barrier_init();
         prefetch_tmap(&tmap_q);
         prefetch_tmap(&tmap_k);
@@ -301,75 +306,195 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 for (int j = max(0, v_issued - kVStages); j < v_issued; ++j) mbar_drain(&v_full[j % kVStages], (j / kVStages) & 1);
             }
         }
-    } else if (warp == 1) {
-        // tcgen05.mma issuer: one elected thread serves both query tiles, in the fixed order
-        //     O_A += P_A V_j ; S_A = Q_A K_{j+1}^T ; O_B += P_B V_j ; S_B = Q_B K_{j+1}^T
-        // which is what keeps the two tiles half a period apart (one tile's softmax runs while the
-        // other's 16 instructions execute). Issuing costs the thread about 45 clocks per instruction
-        // against 64 of execution, and the tensor pipe queues only three or four instructions, so every
-        // other clock the thread spends is tensor-core idle time: a barrier wait by one thread costs 65
-        // clocks when already satisfied, the same wait taken by the whole warp with a vote around it
-        // more than 300. Hence a single thread that does nothing but wait and issue.
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
-            constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
-            // Shared-memory descriptors: (address >> 4) sits in the low 14 bits, so stepping through
-            // a tile or to another stage is an integer add.
-            constexpr uint32_t kTileStep = L::kTileBytes >> 4;
-            const uint64_t q_desc = smem_desc_sw128(smem_u32(q_smem), 16, 1024);
-            const uint64_t k_desc = smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024);
-            const uint64_t v_desc = smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024);
-            const int n_q = tile_b_active ? 2 : 1;
-            // S_t = Q_t K^T with K in stage ks
-            auto issue_s = [&](int t, int ks) {
-                const uint64_t qd = q_desc + (uint32_t)t * kTileStep;
-                const uint64_t kd = k_desc + (uint32_t)ks * kTileStep;
+    } else if (warp == 1 || warp == 2) {
+        // tcgen05.mma issuers. Per key tile j and query tile t one elected thread issues
+        //     O_t += P_t V_j ; S_t = Q_t K_{j+1}^T          (16 instructions at head size 128)
+        // Issuing costs a thread about 80 clocks per instruction in this kernel (more than the 64 an
+        // instruction executes in) and a satisfied barrier wait 65 to 180.
+        if constexpr (kIssuers == 2) {
+            // Head size 128: one thread serving both tiles was itself the limit (its waits and loop
+            // bookkeeping sat between the two tiles' instruction groups), so each tile has its own thread
+            // (warp 1 for tile A, warp 2 for tile B) and all of that happens while the other thread
+            // issues. The two pass a token so that the groups still alternate A, B, A, B: left to
+            // themselves the tiles drift into phase (both softmaxes at once, then both instruction
+            // groups), which is slower than the alternation, where one tile's softmax runs under the
+            // other tile's instructions. The token orders instruction issue only; no data depends on it.
+            const int t = warp - 1;
+            if (lane == 0 && (t == 0 || tile_b_active)) {
+                constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
+                constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
+                // Shared-memory descriptors: (address >> 4) sits in the low 14 bits, so stepping through
+                // a tile or to another stage is an integer add.
+                constexpr uint32_t kTileStep = L::kTileBytes >> 4;
+                const uint64_t q_desc = smem_desc_sw128(smem_u32(q_smem), 16, 1024) + (uint32_t)t * kTileStep;
+                const uint64_t k_desc = smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024);
+                const uint64_t v_desc = smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024);
+                const uint32_t s_tmem = tmem_base + 128u * t, o_tmem = tmem_base + 256u + 128u * t;
+                const bool paired = tile_b_active;
+                uint32_t turn_par = 0;
+                // S_t = Q_t K^T with K in stage ks
+                auto issue_s = [&](int ks) {
+                    const uint64_t kd = k_desc + (uint32_t)ks * kTileStep;
 #pragma unroll
-                for (int kk = 0; kk < DH / 16; ++kk) {
-                    constexpr uint32_t kSlabStep = kSlabBytes >> 4;
-                    const uint32_t off = (kk >> 2) * kSlabStep + (kk & 3) * 2;    // 32 bytes per 16 k
-                    mma_bf16_ss(tmem_base + 128u * t, qd + off, kd + off, idesc_s, kk ? 1u : 0u);
+                    for (int kk = 0; kk < DH / 16; ++kk) {
+                        constexpr uint32_t kSlabStep = kSlabBytes >> 4;
+                        const uint32_t off = (kk >> 2) * kSlabStep + (kk & 3) * 2;    // 32 bytes per 16 k
+                        mma_bf16_ss(s_tmem, q_desc + off, kd + off, idesc_s, kk ? 1u : 0u);
+                    }
+                    mma_commit(&s_full[t]);
+                };
+                // O_t (+)= P_t V with V in stage vs; P_t sits in the first 64 columns of S_t, two keys per column
+                auto issue_pv = [&](int vs, bool first) {
+                    const uint64_t vd = v_desc + (uint32_t)vs * kTileStep;
+#pragma unroll
+                    for (int kk = 0; kk < BKV / 16; ++kk)
+                        mma_bf16_ts(o_tmem, s_tmem + kk * 8, vd + (uint32_t)(kk * 128), idesc_o, (first && kk == 0) ? 0u : 1u);
+                };
+                // the token: wait for this tile's turn, hand the turn to the other tile once this tile's
+                // instructions are issued (they execute in the order in which they were issued)
+                // (a counter in shared memory polled with plain loads: the waiting thread has nothing else to
+                // do, and a load comes back several times faster than a suspended barrier wait wakes up)
+                volatile uint32_t* turn_ctr = (volatile uint32_t*)turn;      // [2], zeroed with the barriers
+                auto take_turn = [&]() {
+                    if (!paired) return true;
+                    ++turn_par;                                   // number of the turn this thread waits for
+                    if (turn_ctr[t * 2] >= turn_par) return true;
+                    const unsigned long long t0 = global_ns();
+                    uint32_t spins = 0;
+                    while (turn_ctr[t * 2] < turn_par) {
+                        if ((++spins & 255u) == 0) {
+                            if (*abort_flag) return false;
+                            unsigned long long limit = *(volatile const unsigned long long*)(p.status + NOVA_WAIT_LIMIT_WORD);
+                            if (limit == 0) limit = kWaitLimitNs;
+                            if (global_ns() - t0 > limit) {
+                                *abort_flag = 1;
+                                atomicOr(p.status, NOVA_DEV_TIMEOUT);
+                                return false;
+                            }
+                        }
+                    }
+                    return true;
+                };
+                uint32_t passed = 0;
+                auto pass_turn = [&]() {
+                    if (!paired) return;
+                    __threadfence_block();
+                    turn_ctr[(t ^ 1) * 2] = ++passed;
+                };
+                bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
+                if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag, p.status);
+                if (ok && t == 1) ok = take_turn();          // tile A goes first
+                if (ok) {
+                    tc_fence_after();
+                    issue_s(0);
+                    mma_commit(&k_empty[0]);
+                    pass_turn();
                 }
-                mma_commit(&s_full[t]);
-            };
-            // O_t (+)= P_t V with V in stage vs; P_t sits in the first 64 columns of S_t, two keys per column
-            auto issue_pv = [&](int t, int vs, bool first) {
-                const uint64_t vd = v_desc + (uint32_t)vs * kTileStep;
-#pragma unroll
-                for (int kk = 0; kk < BKV / 16; ++kk)
-                    mma_bf16_ts(tmem_base + 256u + 128u * t, tmem_base + 128u * t + kk * 8, vd + (uint32_t)(kk * 128),
-                                idesc_o, (first && kk == 0) ? 0u : 1u);
-            };
-            bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
-            if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag, p.status);
-            if (ok) {
-                tc_fence_after();
-                for (int t = 0; t < n_q; ++t) issue_s(t, 0);
-                mma_commit(&k_empty[0]);
-            }
-            // ring positions and phase parities, stepped without divisions
-            int vs = 0, ks_next = (kKStages > 1) ? 1 : 0;
-            uint32_t v_par = 0, k_par_next = (kKStages > 1) ? 0u : 1u;
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const bool more = j + 1 < n_tiles;
-                // V_j and K_{j+1} have usually landed long ago; P is what a step waits for
-                ok = mbar_wait(&v_full[vs], v_par, abort_flag, p.status);
-                if (ok && more) ok = mbar_wait(&k_full[ks_next], k_par_next, abort_flag, p.status);
-                for (int t = 0; t < n_q && ok; ++t) {
-                    ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
+                // ring positions and phase parities, stepped without divisions
+                int vs = 0, ks_next = (kKStages > 1) ? 1 : 0;
+                uint32_t v_par = 0, k_par_next = (kKStages > 1) ? 0u : 1u;
+                for (int j = 0; j < n_tiles && ok; ++j) {
+                    const bool more = j + 1 < n_tiles;
+                    // V_j and K_{j+1} have usually landed long ago; P is what a step waits for
+                    ok = mbar_wait(&v_full[vs], v_par, abort_flag, p.status);
+                    if (ok && more) ok = mbar_wait(&k_full[ks_next], k_par_next, abort_flag, p.status);
+                    if (ok) {
+                        // polled without suspending: this thread has nothing else to do
+                        const unsigned long long t0 = global_ns();
+                        uint32_t spins = 0;
+                        while (!mbar_test_wait(&p_full[t], j & 1)) {
+                            if ((++spins & 255u) == 0) {
+                                if (*abort_flag) { ok = false; break; }
+                                unsigned long long limit = *(volatile const unsigned long long*)(p.status + NOVA_WAIT_LIMIT_WORD);
+                                if (limit == 0) limit = kWaitLimitNs;
+                                if (global_ns() - t0 > limit) {
+                                    *abort_flag = 1;
+                                    atomicOr(p.status, NOVA_DEV_TIMEOUT);
+                                    ok = false;
+                                    break;
+                                }
+                            }
+                        }
+                    }
+                    if (ok) ok = take_turn();
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(t, vs, j == 0);
-                    if (t == n_q - 1) mma_commit(&v_empty[vs]);                 // V_j has no reader left
+                    issue_pv(vs, j == 0);
+                    mma_commit(&v_empty[vs]);                       // this tile no longer reads V_j
                     if (more) {
-                        issue_s(t, ks_next);
-                        if (t == n_q - 1) mma_commit(&k_empty[ks_next]);        // nor has K_{j+1}
+                        issue_s(ks_next);
+                        mma_commit(&k_empty[ks_next]);              // nor K_{j+1}
                     }
+                    pass_turn();
+                    if (++vs == kVStages) { vs = 0; v_par ^= 1u; }
+                    if (++ks_next == kKStages) { ks_next = 0; k_par_next ^= 1u; }
                 }
-                if (++vs == kVStages) { vs = 0; v_par ^= 1u; }
-                if (++ks_next == kKStages) { ks_next = 0; k_par_next ^= 1u; }
+                if (ok) mma_commit(o_done);
             }
-            if (ok) mma_commit(o_done);
+        } else if (warp == 1) {
+            // Head size 64: the groups are short, the token costs more than it saves, and one thread
+            // serves both tiles in the fixed order A, B.
+            if (lane == 0) {
+                constexpr uint32_t idesc_s = idesc_bf16_f32(BQ, BKV, 0);
+                constexpr uint32_t idesc_o = idesc_bf16_f32(BQ, DH, 1);
+                // Shared-memory descriptors: (address >> 4) sits in the low 14 bits, so stepping through
+                // a tile or to another stage is an integer add.
+                constexpr uint32_t kTileStep = L::kTileBytes >> 4;
+                const uint64_t q_desc = smem_desc_sw128(smem_u32(q_smem), 16, 1024);
+                const uint64_t k_desc = smem_desc_sw128(smem_u32(smem + L::kKOff), 16, 1024);
+                const uint64_t v_desc = smem_desc_sw128(smem_u32(smem + L::kVOff), kSlabBytes, 1024);
+                const int n_q = tile_b_active ? 2 : 1;
+                // S_t = Q_t K^T with K in stage ks
+                auto issue_s = [&](int t, int ks) {
+                    const uint64_t qd = q_desc + (uint32_t)t * kTileStep;
+                    const uint64_t kd = k_desc + (uint32_t)ks * kTileStep;
+#pragma unroll
+                    for (int kk = 0; kk < DH / 16; ++kk) {
+                        constexpr uint32_t kSlabStep = kSlabBytes >> 4;
+                        const uint32_t off = (kk >> 2) * kSlabStep + (kk & 3) * 2;    // 32 bytes per 16 k
+                        mma_bf16_ss(tmem_base + 128u * t, qd + off, kd + off, idesc_s, kk ? 1u : 0u);
+                    }
+                    mma_commit(&s_full[t]);
+                };
+                // O_t (+)= P_t V with V in stage vs; P_t sits in the first 64 columns of S_t, two keys per column
+                auto issue_pv = [&](int t, int vs, bool first) {
+                    const uint64_t vd = v_desc + (uint32_t)vs * kTileStep;
+#pragma unroll
+                    for (int kk = 0; kk < BKV / 16; ++kk)
+                        mma_bf16_ts(tmem_base + 256u + 128u * t, tmem_base + 128u * t + kk * 8, vd + (uint32_t)(kk * 128),
+                                    idesc_o, (first && kk == 0) ? 0u : 1u);
+                };
+                bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
+                if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag, p.status);
+                if (ok) {
+                    tc_fence_after();
+                    for (int t = 0; t < n_q; ++t) issue_s(t, 0);
+                    mma_commit(&k_empty[0]);
+                }
+                // ring positions and phase parities, stepped without divisions
+                int vs = 0, ks_next = (kKStages > 1) ? 1 : 0;
+                uint32_t v_par = 0, k_par_next = (kKStages > 1) ? 0u : 1u;
+                for (int j = 0; j < n_tiles && ok; ++j) {
+                    const bool more = j + 1 < n_tiles;
+                    // V_j and K_{j+1} have usually landed long ago; P is what a step waits for
+                    ok = mbar_wait(&v_full[vs], v_par, abort_flag, p.status);
+                    if (ok && more) ok = mbar_wait(&k_full[ks_next], k_par_next, abort_flag, p.status);
+                    for (int t = 0; t < n_q && ok; ++t) {
+                        ok = mbar_wait(&p_full[t], j & 1, abort_flag, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(t, vs, j == 0);
+                        if (t == n_q - 1) mma_commit(&v_empty[vs]);                 // V_j has no reader left
+                        if (more) {
+                            issue_s(t, ks_next);
+                            if (t == n_q - 1) mma_commit(&k_empty[ks_next]);        // nor has K_{j+1}
+                        }
+                    }
+                    if (++vs == kVStages) { vs = 0; v_par ^= 1u; }
+                    if (++ks_next == kKStages) { ks_next = 0; k_par_next ^= 1u; }
+                }
+                if (ok) mma_commit(o_done);
+            }
         }
     }
     } else {
@@ -477,10 +602,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 }
                 l_run += lsum;
                 tmem_st_wait();
-                if (t == 0 && cols_valid < BKV) {
+                if ((t == 0 || kIssuers == 2) && cols_valid < BKV) {
                     // ragged last tile: rows of V past the last key may hold anything (even NaN);
-                    // zero them so that 0 * garbage cannot poison the accumulator (tile A's O += P V
-                    // is issued before tile B's, so tile A's softmax warps do it for both)
+                    // zero them so that 0 * garbage cannot poison the accumulator. With one issuing
+                    // thread tile A's O += P V is issued before tile B's, so tile A's softmax warps do it
+                    // for both; with a thread per tile each tile's warps do it before their own hand-over
+                    // (zeros written over zeros are harmless)
                     const int s = j % kVStages;
                     ok = mbar_wait_warp(&v_full[s], (j / kVStages) & 1, abort_flag, p.status);
                     if (!ok) break;
