@@ -378,8 +378,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 uint32_t passed = 0;
                 auto pass_turn = [&]() {
                     if (!paired) return;
-                    __threadfence_block();
-                    turn_ctr[(t ^ 1) * 2] = ++passed;
+                    turn_ctr[(t ^ 1) * 2] = ++passed;      // no fence: the token orders issue in time, no data hangs on it
                 };
                 bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
                 if (ok) ok = mbar_wait(&k_full[0], 0, abort_flag, p.status);
@@ -398,7 +397,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     // V_j and K_{j+1} have usually landed long ago; P is what a step waits for
                     ok = mbar_wait(&v_full[vs], v_par, abort_flag, p.status);
                     if (ok && more) ok = mbar_wait(&k_full[ks_next], k_par_next, abort_flag, p.status);
-                    if (ok) {
+                    if (ok && !mbar_test_wait(&p_full[t], j & 1)) {
                         // polled without suspending: this thread has nothing else to do
                         const unsigned long long t0 = global_ns();
                         uint32_t spins = 0;
