@@ -46,9 +46,10 @@ constexpr float kHugeSum = 1.0995116e12f;   // 2^40
 
 template <int DH>
 struct AttnSmem {
-    // K tiles are released right after the last S = Q K^T that reads them, V tiles only after
-    // O += P V one softmax later, so the two rings run separately; head size 128 fills the
-    // 227 KB with two Q tiles, three K stages and two V stages.
+    // K_{j+1} is last read by S = Q K_{j+1}^T in step j, V_j by O += P V_j in the same step, one
+    // softmax after V_j's own scores, so the two rings have different depths and one release (after
+    // the step's last instruction) serves both; head size 128 fills the 227 KB with two Q tiles,
+    // three K stages and two V stages.
     static constexpr int kKStages = (DH == 64) ? 4 : 3;
     static constexpr int kVStages = (DH == 64) ? 4 : 2;
     static constexpr int kSlabs = DH / 64;
@@ -226,8 +227,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint64_t* k_full = bars + 1;                      // kKStages
     uint64_t* k_empty = k_full + kKStages;            // kKStages
     uint64_t* v_full = k_empty + kKStages;            // kVStages
-    uint64_t* v_empty = v_full + kVStages;            // kVStages
-    uint64_t* s_full = v_empty + kVStages;            // 2 (tile A, tile B)
+    uint64_t* s_full = v_full + kVStages;             // 2 (tile A, tile B)
     uint64_t* p_full = s_full + 2;                    // 2, one arrival per softmax warp
     uint64_t* o_done = p_full + 2;                    // 1, one arrival per issuing thread
     uint64_t* turn = o_done + 1;                      // 2 counters (not barriers): turns granted to the issuing thread of tile t
@@ -247,10 +247,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             mbar_init(&k_full[s], 1);
             mbar_init(&k_empty[s], n_issuers);
         }
-        for (int s = 0; s < kVStages; ++s) {
-            mbar_init(&v_full[s], 1);
-            mbar_init(&v_empty[s], n_issuers);
-        }
+        for (int s = 0; s < kVStages; ++s) mbar_init(&v_full[s], 1);
         for (int t = 0; t < 2; ++t) {
             mbar_init(&s_full[t], 1);
             mbar_init(&p_full[t], 4);
@@ -293,7 +290,16 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 for (int sl = 0; sl < kSlabs; ++sl)
                     tma_load_3d(k_dst + sl * kSlabBytes, &tmap_k, &k_full[ks], head * DH + sl * 64, (jt0 + j) * BKV, b);
                 k_issued = j + 1;
-                if (j >= kVStages && !mbar_wait(&v_empty[vs], ((j / kVStages) - 1) & 1, abort_flag, p.status)) break;
+                // The slot of V_j held V_{j-kVStages}, whose last reader is step j-kVStages. That step ends with
+                // S = Q K_{j-kVStages+1}^T, and the commit that releases that K tile (k_empty) follows every
+                // instruction of the step, O += P V included: it releases the V tile as well. (The K slot is
+                // not released again before K_{j-kVStages+1+kKStages} has been loaded, which comes after
+                // this wait since kKStages + 1 > kVStages: the phase waited for cannot be overtaken twice.)
+                static_assert(kKStages + 1 > kVStages, "the K release that stands for the V release must not be overtaken");
+                if (j >= kVStages) {
+                    const int kj = j - kVStages + 1;
+                    if (!mbar_wait(&k_empty[kj % kKStages], (kj / kKStages) & 1, abort_flag, p.status)) break;
+                }
                 uint8_t* v_dst = smem + L::kVOff + vs * L::kTileBytes;
                 mbar_arrive_expect_tx(&v_full[vs], L::kTileBytes);
                 for (int sl = 0; sl < kSlabs; ++sl)
@@ -419,10 +425,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     if (!ok) break;
                     tc_fence_after();
                     issue_pv(vs, j == 0);
-                    mma_commit(&v_empty[vs]);                       // this tile no longer reads V_j
                     if (more) {
                         issue_s(ks_next);
-                        mma_commit(&k_empty[ks_next]);              // nor K_{j+1}
+                        mma_commit(&k_empty[ks_next]);              // this tile no longer reads K_{j+1}, nor V_j
                     }
                     pass_turn();
                     if (++vs == kVStages) { vs = 0; v_par ^= 1u; }
@@ -483,10 +488,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         if (!ok) break;
                         tc_fence_after();
                         issue_pv(t, vs, j == 0);
-                        if (t == n_q - 1) mma_commit(&v_empty[vs]);                 // V_j has no reader left
                         if (more) {
                             issue_s(t, ks_next);
-                            if (t == n_q - 1) mma_commit(&k_empty[ks_next]);        // nor has K_{j+1}
+                            if (t == n_q - 1) mma_commit(&k_empty[ks_next]);        // K_{j+1} and V_j have no reader left
                         }
                     }
                     if (++vs == kVStages) { vs = 0; v_par ^= 1u; }
