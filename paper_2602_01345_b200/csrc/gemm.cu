@@ -561,53 +561,44 @@ gemm_bf16_tn_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
         }
     } else if (warp == 1) {
-        if (rank == 0) {
-            // The whole warp runs the loop in lockstep and lane 0 issues. tcgen05.mma takes its
-            // descriptors and addresses from uniform registers; with the bases broadcast from lane 0
-            // (which tells the compiler they are warp-uniform), ring counters instead of divisions
-            // and warp-uniform control flow, the per-instruction address arithmetic stays in the
-            // uniform datapath. Issue is close to synchronous with execution, so every clock of
-            // issue overhead is a clock the tensor core idles.
+        if (rank == 0 && lane == 0) {
+            // One elected thread of the leader CTA does nothing but wait and issue. Per 64-wide k-block
+            // the tensor core works 512 clocks (four M=256, N=256, K=16 instructions); the thread spends
+            // about 80 clocks per instruction, 50 on the commit and 65 on a wait that is already
+            // satisfied, which leaves a margin. The earlier form, the whole warp in lockstep with every
+            // lane polling the barrier and a vote after it, paid about 300 clocks per wait and made the
+            // issuing warp, not the tensor core, the limit of the main loop (tensor pipe 75 % active).
             constexpr uint32_t idesc_whole = idesc_bf16_f32(kPairBM, BN, 0);
             constexpr uint32_t idesc_half = idesc_bf16_f32(kPairBM, BN / 2, 0);
-            auto uniform32 = [](uint32_t v) { return __shfl_sync(0xffffffffu, v, 0); };
-            const uint64_t desc0 = smem_desc_sw128(smem_u32(smem), 16, 1024);
-            const uint64_t a_desc = ((uint64_t)uniform32((uint32_t)(desc0 >> 32)) << 32) | uniform32((uint32_t)desc0);
-            const uint32_t tmem_u = uniform32(tmem_base);
-            const int first_tile = (int)uniform32((uint32_t)pair), step = (int)uniform32((uint32_t)num_pairs);
-            const bool issuer = (lane == 0);
+            const uint64_t a_desc = smem_desc_sw128(smem_u32(smem), 16, 1024);
             int s = 0;                 // ring position and phase parity of the next k-block
             uint32_t par = 0;
             int local = 0;
             bool ok = true;
             for (; ok; ++local) {
-                const int tile = pair_entry(local, first_tile, step, num_tiles, group);
+                const int tile = pair_entry(local, pair, num_pairs, num_tiles, group);
                 if (tile < 0) break;
                 const int a = local & 1;
                 if (local >= 2) {
-                    ok = mbar_wait_warp(&acc_empty[a], (uint32_t)((local >> 1) - 1) & 1, abort_flag, p.status);
+                    ok = mbar_wait(&acc_empty[a], (uint32_t)((local >> 1) - 1) & 1, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
                 }
-                const uint32_t d_tmem = tmem_u + (uint32_t)(a * BN);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * BN);
                 const uint32_t idesc = (tile < tiles_full) ? idesc_whole : idesc_half;
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    ok = mbar_wait_warp(&full_bar[s], par, abort_flag, p.status);
+                    ok = mbar_wait(&full_bar[s], par, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
                     const uint64_t ad = a_desc + (uint32_t)s * (uint32_t)(L::kStageBytes >> 4);
                     const uint64_t bd = ad + (uint32_t)(L::kABytes >> 4);
-                    if (issuer) {
 #pragma unroll
-                        for (int kk = 0; kk < BK / 16; ++kk)
-                            mma_bf16_ss_pair(d_tmem, ad + (uint32_t)(kk * 2), bd + (uint32_t)(kk * 2), idesc, (kb | kk) ? 1u : 0u);
-                        mma_commit_pair(&empty_bar[s], 3);      // frees the stage in both CTAs
-                    }
-                    __syncwarp();
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        mma_bf16_ss_pair(d_tmem, ad + (uint32_t)(kk * 2), bd + (uint32_t)(kk * 2), idesc, (kb | kk) ? 1u : 0u);
+                    mma_commit_pair(&empty_bar[s], 3);      // frees the stage in both CTAs
                     if (++s == STAGES) { s = 0; par ^= 1u; }
                 }
-                if (ok && issuer) mma_commit_pair(&acc_full[a], 3);    // accumulator complete in both CTAs
-                __syncwarp();
+                if (ok) mma_commit_pair(&acc_full[a], 3);    // accumulator complete in both CTAs
             }
         }
     } else {
