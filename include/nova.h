@@ -106,9 +106,13 @@ unsigned long long nova_launch_count(const nova_ctx* ctx);
 /* Per-kernel timing: between nova_profile_begin and nova_profile_end every kernel launch is
  * bracketed by CUDA events on its stream. nova_profile_end waits for them and fills
  * ms[c] / launches[c] (host arrays of n >= nova_profile_categories() entries) with the summed
- * device time and the launch count of category c; nova_profile_category_name(c) names it. */
+ * device time and the launch count of category c; nova_profile_category_name(c) names it.
+ * nova_profile_select restricts the brackets to the categories whose bit is set in category_mask
+ * (bit c = category c; all by default): each bracket costs two event records on the stream, which
+ * shows in a step of a few hundred launches. */
 int         nova_profile_categories(void);
 const char* nova_profile_category_name(int cat);
+nova_status nova_profile_select(nova_ctx* ctx, unsigned long long category_mask);
 nova_status nova_profile_begin(nova_ctx* ctx);
 nova_status nova_profile_end(nova_ctx* ctx, double* ms, long long* launches, int n);
 

@@ -41,6 +41,7 @@ nova_status nova_create(nova_ctx** out, int device)
     ctx->err[0] = 0;
     ctx->launches = 0;
     ctx->profiling = false;
+    ctx->prof_mask = ~0ull;
     ctx->events_used = 0;
     ctx->wait_limit_ns = 0;
     const char* dbg = getenv("NOVA_DEBUG");
@@ -95,6 +96,13 @@ const char* nova_profile_category_name(int cat)
         "entropy_rows", "entropy_mean", "select_topk", "layernorm", "gemm_qkv",
         "attention", "gemm_proj", "gemm_fc1", "gemm_fc2", "restore", "keep_ratios", "selection_score"};
     return (cat >= 0 && cat < NOVA_K_COUNT) ? names[cat] : "?";
+}
+
+nova_status nova_profile_select(nova_ctx* ctx, unsigned long long category_mask)
+{
+    if (!ctx) return NOVA_ERR_INVALID_ARG;
+    ctx->prof_mask = category_mask;
+    return NOVA_OK;
 }
 
 nova_status nova_profile_begin(nova_ctx* ctx)

@@ -56,6 +56,7 @@ struct nova_ctx {
     // measurement: launches since creation, and event pairs around each launch while profiling
     unsigned long long launches;
     bool profiling;
+    unsigned long long prof_mask;             // categories that get event brackets while profiling (bit c = category c)
     std::vector<nova_prof_rec> prof_recs;     // records of the current profiling window
     std::vector<cudaEvent_t> event_pool;      // events created so far (reused across windows)
     size_t events_used;
@@ -70,7 +71,7 @@ struct nova_launch_scope {
     nova_launch_scope(nova_ctx* c, int cat, cudaStream_t s) : ctx(c), st(s), stop(nullptr)
     {
         ctx->launches++;
-        if (!ctx->profiling) return;
+        if (!ctx->profiling || !((ctx->prof_mask >> cat) & 1ull)) return;
         while (ctx->event_pool.size() < ctx->events_used + 2) {
             cudaEvent_t e;
             if (cudaEventCreate(&e) != cudaSuccess) return;

@@ -326,9 +326,31 @@ def launch_count(ctx: nv.Context) -> int:
     return int(nv._lib.nova_launch_count(ctx.handle))
 
 
-def profile_begin(ctx: nv.Context):
-    nv._lib.nova_profile_begin.argtypes = [C.c_void_p]
-    ctx.check(nv._lib.nova_profile_begin(ctx.handle))
+def profile_begin(ctx: nv.Context, categories=None):
+    """Starts a profiling window. categories: names of the kernel categories to bracket with events
+    (None = all)."""
+    lib = nv._lib
+    lib.nova_profile_select.argtypes = [C.c_void_p, C.c_ulonglong]
+    mask = (1 << 64) - 1
+    if categories is not None:
+        lib.nova_profile_categories.restype = C.c_int
+        lib.nova_profile_category_name.restype = C.c_char_p
+        lib.nova_profile_category_name.argtypes = [C.c_int]
+        names = [lib.nova_profile_category_name(i).decode() for i in range(lib.nova_profile_categories())]
+        unknown = set(categories) - set(names)
+        assert not unknown, f"unknown kernel categories {sorted(unknown)}"
+        mask = sum(1 << names.index(c) for c in set(categories))
+    ctx.check(lib.nova_profile_select(ctx.handle, mask))
+    lib.nova_profile_begin.argtypes = [C.c_void_p]
+    ctx.check(lib.nova_profile_begin(ctx.handle))
+
+
+def profile_category_names(ctx: nv.Context) -> list:
+    lib = nv._lib
+    lib.nova_profile_categories.restype = C.c_int
+    lib.nova_profile_category_name.restype = C.c_char_p
+    lib.nova_profile_category_name.argtypes = [C.c_int]
+    return [lib.nova_profile_category_name(i).decode() for i in range(lib.nova_profile_categories())]
 
 
 def profile_end(ctx: nv.Context) -> dict:
