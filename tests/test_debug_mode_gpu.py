@@ -1,4 +1,4 @@
-"""Debug mode and guard bands.
+"""Debug mode, guard bands and the selection of profiled kernel categories.
 
 Debug mode (nova_set_debug): index lists are validated on the device before any kernel uses them,
 so a corrupt list comes back as NOVA_ERR_INVALID_ARG with nothing dereferenced, and every launch is
@@ -238,3 +238,25 @@ def test_guard_bands_around_every_output(ctx):
     for b in range(B):
         n1 = c["kv_lens"][b] + ks[b]
         assert torch.equal(kc.t[b, n1:], c["k_cache"][b, n1:]) and torch.equal(vc.t[b, n1:], c["v_cache"][b, n1:])
+
+
+def test_profile_select_brackets_only_the_selected_categories(ctx):
+    """nova_profile_select: only launches of the selected kernel categories get event brackets; the
+    launch counter counts every launch either way."""
+    from paper_2602_01345_b200 import pipeline
+    c = _case()
+    keep_idx, prune_idx, cu = _lists(ctx, c)
+    n0 = pipeline.launch_count(ctx)
+    pipeline.profile_begin(ctx, ["attention", "restore"])
+    _layer(ctx, c, keep_idx, prune_idx, cu)
+    prof = pipeline.profile_end(ctx)
+    per_layer = pipeline.launch_count(ctx) - n0
+    assert per_layer >= 8                                   # two LayerNorms, four GEMMs, attention, restore
+    assert prof["attention"][1] == 1 and prof["restore"][1] == 1 and prof["attention"][0] > 0.0
+    assert all(v[1] == 0 for k, v in prof.items() if k not in ("attention", "restore"))
+    pipeline.profile_begin(ctx)                             # all categories again
+    _layer(ctx, c, keep_idx, prune_idx, cu)
+    prof = pipeline.profile_end(ctx)
+    assert sum(v[1] for v in prof.values()) == per_layer
+    with pytest.raises(AssertionError):
+        pipeline.profile_begin(ctx, ["no_such_kernel"])
