@@ -184,6 +184,16 @@ def test_attention_small_ragged(ctx, C, heads):
                    seed=3, q_gain=4.0, label=f"ragged, head size {C // heads}")
 
 
+@pytest.mark.parametrize("C,heads", [(256, 2), (128, 2)])
+def test_attention_partly_filled_query_blocks_over_many_key_tiles(ctx, C, heads):
+    """Both head sizes (at 128 each query tile has its own issuing thread, at 64 one thread serves
+    both): a 300-row image whose second query block has 44 rows (second tile unused), a 129-row image
+    whose second tile has a single row, and a 256-row image with both tiles full, over 8 to 11 key
+    tiles with ragged ends."""
+    attention_case(ctx, B=3, N=320, C=C, heads=heads, F=256, Lmax=1400, ks=[300, 129, 256], kv_lens=[1000, 517, 777],
+                   seed=13, q_gain=4.0, label=f"partly filled query blocks, head size {C // heads}")
+
+
 def test_attention_q_zero_gives_mean_of_values(ctx):
     """Zero queries: every score is 0, the softmax is uniform, the output is the mean of all value
     rows (prior ones and the kept tokens' own)."""
